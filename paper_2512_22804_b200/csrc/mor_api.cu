@@ -1,0 +1,446 @@
+// Host side of the C boundary: argument checks, workspace layout, grouping of tensors by
+// partition kind and launch sequence.  No device code lives here.
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "mor_internal.h"
+
+namespace mor {
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+struct Shape {
+    int kind;
+    uint32_t nbc, nbr, n_units, n_tiles, amax_tiles;
+    uint64_t n_blocks;
+};
+
+// Partition geometry of one descriptor; MOR_OK or the reason it cannot run.
+mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
+{
+    if (d.rows < 0 || d.cols < 0) return MOR_ERR_INVALID_ARG;
+    if (d.block_rows == 0 && d.block_cols == 0) s.kind = KIND_TENSOR;
+    else if (d.block_rows == 1 && d.block_cols == 128) s.kind = KIND_ROW128;
+    else if (d.block_rows == 128 && d.block_cols == 128) s.kind = KIND_BLK128;
+    else return MOR_ERR_UNSUPPORTED;
+    const bool empty = d.rows == 0 || d.cols == 0;
+    const uint64_t nbc = empty ? 0 : (uint64_t)(d.cols + 127) / 128;
+    const uint64_t nbr = empty ? 0 : (uint64_t)(d.rows + 127) / 128;
+    const uint64_t segs = empty ? 0 : (uint64_t)d.rows * nbc;
+    if (segs >= (1ull << 31) || nbc >= (1ull << 24)) return MOR_ERR_UNSUPPORTED;
+    s.nbc = (uint32_t)nbc;
+    s.nbr = (uint32_t)nbr;
+    s.amax_tiles = (uint32_t)((segs + kSegsPerTile - 1) / kSegsPerTile);
+    if (s.kind == KIND_BLK128) {
+        s.n_units = (uint32_t)(nbr * nbc);
+        s.n_tiles = s.n_units;
+        s.n_blocks = s.n_units;
+    } else {
+        s.n_units = (uint32_t)segs;
+        s.n_tiles = s.amax_tiles;
+        s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
+    }
+    return MOR_OK;
+}
+
+mor_status_t check_desc(const mor_tensor_desc_t& d, Shape& s)
+{
+    mor_status_t st = shape_of(d, s);
+    if (st != MOR_OK) return st;
+    if (d.ld < d.cols) return MOR_ERR_INVALID_ARG;
+    if (d.ld % 8 != 0) return MOR_ERR_ALIGNMENT;
+    const bool empty = d.rows == 0 || d.cols == 0;
+    if (!empty && d.x == nullptr) return MOR_ERR_INVALID_ARG;
+    if (!aligned(d.x, 16)) return MOR_ERR_ALIGNMENT;
+    if (d.n_formats == 2) {
+        if (d.formats[0] != MOR_FMT_E4M3 || d.formats[1] != MOR_FMT_BF16) return MOR_ERR_UNSUPPORTED;
+    } else if (d.n_formats == 3) {
+        if (d.formats[0] != MOR_FMT_E4M3 || d.formats[1] != MOR_FMT_E5M2 || d.formats[2] != MOR_FMT_BF16)
+            return MOR_ERR_UNSUPPORTED;
+        // the paper defines the E5M2 metric (Eq. 4) only after the Eq. 3 test, per block;
+        // a per-tensor block would need its codes rewritten after the last tile
+        if (d.criterion != MOR_CRIT_BLOCK_VS_E5M2 || s.kind == KIND_TENSOR) return MOR_ERR_UNSUPPORTED;
+    } else {
+        return MOR_ERR_INVALID_ARG;
+    }
+    if (d.criterion < MOR_CRIT_TENSOR_MEAN_REL || d.criterion > MOR_CRIT_BLOCK_MEAN_REL) return MOR_ERR_INVALID_ARG;
+    if (d.scale_mode < MOR_SCALE_GAM || d.scale_mode > MOR_SCALE_FP32_AMAX) return MOR_ERR_INVALID_ARG;
+    if (!(d.threshold >= 0.0f) || std::isinf(d.threshold)) return MOR_ERR_INVALID_ARG;
+    if (d.flags & ~(uint32_t)(MOR_FLAG_STRICT_TIES | MOR_FLAG_RANGE_MIN_INCLUDES_ZERO)) return MOR_ERR_INVALID_ARG;
+    if (d.group_amax && !aligned(d.group_amax, 4)) return MOR_ERR_ALIGNMENT;
+    return MOR_OK;
+}
+
+mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_outputs_t& o, bool store)
+{
+    if (o.tensor_stats == nullptr) return MOR_ERR_INVALID_ARG;
+    if (!aligned(o.tensor_stats, 8) || !aligned(o.block_stats, 4) || !aligned(o.scale_f32, 4)) return MOR_ERR_ALIGNMENT;
+    const bool empty = d.rows == 0 || d.cols == 0;
+    if (store) {
+        if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
+        if (o.codes_ld < (int64_t)round_up((size_t)d.cols, 16)) return MOR_ERR_INVALID_ARG;
+        if (o.codes_ld % 16 != 0 || !aligned(o.codes, 16)) return MOR_ERR_ALIGNMENT;
+        if (d.scale_mode == MOR_SCALE_FP32_AMAX && o.scale_f32 == nullptr && s.n_blocks) return MOR_ERR_INVALID_ARG;
+        if (o.bf16_fallback) {
+            if (s.kind == KIND_TENSOR || d.criterion == MOR_CRIT_TENSOR_MEAN_REL) return MOR_ERR_UNSUPPORTED;
+            if (!aligned(o.bf16_fallback, 16)) return MOR_ERR_ALIGNMENT;
+        }
+    }
+    return MOR_OK;
+}
+
+struct Layout {
+    size_t amax_off, nonf_off, partial_off, total;
+};
+
+Layout layout_of(int n, uint64_t tiles)
+{
+    Layout l;
+    l.amax_off = 0;
+    l.nonf_off = (size_t)n * sizeof(float);
+    l.partial_off = round_up(2 * (size_t)n * sizeof(float), kAlign);
+    l.total = l.partial_off + round_up((size_t)tiles * sizeof(Partial), kAlign);
+    return l;
+}
+
+struct Item {
+    const mor_tensor_desc_t* d;
+    mor_outputs_t o;
+    Shape s;
+    MainVariant v;
+    uint32_t tile_begin;
+    int index;
+};
+
+void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
+{
+    const mor_tensor_desc_t& d = *it.d;
+    r.x = static_cast<const uint16_t*>(d.x);
+    r.codes = it.o.codes;
+    r.scale_e8m0 = it.o.scale_e8m0;
+    r.sel = it.o.sel;
+    r.scale_f32 = it.o.scale_f32;
+    r.fallback = static_cast<uint16_t*>(it.o.bf16_fallback);
+    r.block_stats = it.o.block_stats;
+    r.tensor_stats = it.o.tensor_stats;
+    r.amax = d.group_amax ? d.group_amax : reinterpret_cast<const float*>(ws + l.amax_off) + it.index;
+    r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
+    r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
+    r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
+    r.tile_begin = it.tile_begin;
+    r.criterion = d.criterion; r.scale_mode = d.scale_mode; r.n_formats = d.n_formats;
+    r.flags = d.flags; r.threshold = d.threshold;
+}
+
+inline bool same_variant(const MainVariant& a, const MainVariant& b)
+{
+    return a.kind == b.kind && a.yard == b.yard && a.three == b.three && a.store == b.store;
+}
+
+// The launch sequence shared by every entry point.
+mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                 const mor_stage_events_t* ev = nullptr)
+{
+    auto record = [&](void* e) -> bool {
+        return e == nullptr || cudaEventRecord(static_cast<cudaEvent_t>(e), stream) == cudaSuccess;
+    };
+    const int n = (int)items.size();
+    uint64_t tiles = 0;
+    for (Item& it : items) { it.tile_begin = (uint32_t)tiles; tiles += it.s.n_tiles; }
+    if (tiles >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
+    const Layout l = layout_of(n, tiles);
+    if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign)) return MOR_ERR_ALIGNMENT;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    Partial* partials = reinterpret_cast<Partial*>(ws + l.partial_off);
+
+    // 1. Algorithm 1, group amax, for the tensors whose caller did not supply it
+    if (ev && !record(ev->amax_begin)) return MOR_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, l.partial_off, stream) != cudaSuccess) return MOR_ERR_CUDA;
+    {
+        BatchParams bp;
+        bp.n = 0;
+        uint32_t t_end = 0;
+        auto flush = [&]() -> bool {
+            if (bp.n == 0) return true;
+            const bool ok = launch_amax(bp, t_end, stream) == cudaSuccess;
+            bp.n = 0; t_end = 0;
+            return ok;
+        };
+        for (const Item& it : items) {
+            if (it.d->group_amax || it.s.amax_tiles == 0) continue;
+            TensorRec& r = bp.t[bp.n];
+            fill_rec(it, ws, l, r);
+            r.n_units = (uint32_t)((uint64_t)it.d->rows * it.s.nbc);   // row pieces, whatever the partition
+            r.n_tiles = it.s.amax_tiles;
+            t_end += r.n_tiles;
+            bp.tile_end[bp.n++] = t_end;
+            if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
+        }
+        if (!flush()) return MOR_ERR_CUDA;
+    }
+
+    // 2. main kernels, one launch per (variant, chunk of tensors); 3. their finalise kernels
+    struct Chunk { BatchParams bp; int kind; };
+    std::vector<Chunk> chunks;
+    if (ev && !record(ev->main_begin)) return MOR_ERR_CUDA;
+    std::vector<char> done(n, 0);
+    for (int i = 0; i < n; ++i) {
+        if (done[i]) continue;
+        const MainVariant v = items[i].v;
+        BatchParams bp;
+        bp.n = 0;
+        uint32_t t_end = 0;
+        auto flush = [&]() -> bool {
+            if (bp.n == 0) return true;
+            const bool ok = launch_main(v, bp, partials, t_end, stream) == cudaSuccess;
+            chunks.push_back(Chunk{bp, v.kind});
+            bp.n = 0; t_end = 0;
+            return ok;
+        };
+        for (int j = i; j < n; ++j) {
+            if (done[j] || !same_variant(items[j].v, v)) continue;
+            done[j] = 1;
+            fill_rec(items[j], ws, l, bp.t[bp.n]);
+            t_end += items[j].s.n_tiles;
+            bp.tile_end[bp.n++] = t_end;
+            if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
+        }
+        if (!flush()) return MOR_ERR_CUDA;
+    }
+    if (ev && !record(ev->main_end)) return MOR_ERR_CUDA;
+    for (const Chunk& c : chunks)
+        if (launch_finalise(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
+    if (ev && !record(ev->finalise_end)) return MOR_ERR_CUDA;
+    return MOR_OK;
+}
+
+mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool store, int index, Item& it)
+{
+    if (d == nullptr) return MOR_ERR_INVALID_ARG;
+    mor_status_t st = check_desc(*d, it.s);
+    if (st != MOR_OK) return st;
+    st = check_out(*d, it.s, o, store);
+    if (st != MOR_OK) return st;
+    it.d = d;
+    it.o = o;
+    it.index = index;
+    it.v.kind = it.s.kind;
+    it.v.three = d->n_formats == 3;
+    it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
+    it.v.store = store;
+    return MOR_OK;
+}
+
+}  // namespace
+}  // namespace mor
+
+using namespace mor;
+
+extern "C" {
+
+size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n)
+{
+    if (host_descs == nullptr || n <= 0) return 0;
+    uint64_t tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        Shape s;
+        if (shape_of(host_descs[i], s) != MOR_OK) return 0;
+        tiles += s.n_tiles;
+    }
+    return layout_of(n, tiles).total;
+}
+
+mor_status_t mor_analyze_quantize_batched_ex(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
+                                             int n, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                                             const mor_stage_events_t* host_events)
+{
+    if (host_descs == nullptr || host_outs == nullptr || n < 0) return MOR_ERR_INVALID_ARG;
+    if (n == 0) return MOR_OK;
+    std::vector<Item> items((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        mor_status_t st = make_item(&host_descs[i], host_outs[i], true, i, items[i]);
+        if (st != MOR_OK) return st;
+    }
+    return run(items, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream), host_events);
+}
+
+mor_status_t mor_analyze_quantize_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
+                                          int n, void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    return mor_analyze_quantize_batched_ex(host_descs, host_outs, n, workspace, workspace_bytes, cuda_stream, nullptr);
+}
+
+mor_status_t mor_analyze_quantize(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    return mor_analyze_quantize_batched(host_desc, host_out, 1, workspace, workspace_bytes, cuda_stream);
+}
+
+mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_block_stats_t* block_stats,
+                              mor_tensor_stats_t* tensor_stats, uint8_t* sel, uint8_t* scale_e8m0,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    mor_outputs_t o;
+    std::memset(&o, 0, sizeof(o));
+    o.block_stats = block_stats;
+    o.tensor_stats = tensor_stats;
+    o.sel = sel;
+    o.scale_e8m0 = scale_e8m0;
+    std::vector<Item> items(1);
+    mor_status_t st = make_item(host_desc, o, false, 0, items[0]);
+    if (st != MOR_OK) return st;
+    return run(items, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* amax_out,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (host_descs == nullptr || n < 0 || (n > 0 && amax_out == nullptr)) return MOR_ERR_INVALID_ARG;
+    if (n == 0) return MOR_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const Layout l = layout_of(n, 0);
+    if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
+    if (!aligned(workspace, kAlign) || !aligned(amax_out, 4)) return MOR_ERR_ALIGNMENT;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    if (cudaMemsetAsync(ws, 0, l.partial_off, stream) != cudaSuccess) return MOR_ERR_CUDA;
+    BatchParams bp;
+    bp.n = 0;
+    uint32_t t_end = 0;
+    for (int i = 0; i < n; ++i) {
+        Item it;
+        mor_tensor_desc_t d = host_descs[i];
+        d.group_amax = nullptr;
+        mor_status_t st = check_desc(d, it.s);
+        if (st != MOR_OK) return st;
+        std::memset(&it.o, 0, sizeof(it.o));
+        it.d = &d; it.index = i; it.tile_begin = 0;
+        if (it.s.amax_tiles) {
+            TensorRec& r = bp.t[bp.n];
+            fill_rec(it, ws, l, r);
+            r.n_units = (uint32_t)((uint64_t)d.rows * it.s.nbc);
+            r.n_tiles = it.s.amax_tiles;
+            t_end += r.n_tiles;
+            bp.tile_end[bp.n++] = t_end;
+        }
+        if (bp.n == kMaxBatch || (i == n - 1 && bp.n)) {
+            if (launch_amax(bp, t_end, stream) != cudaSuccess) return MOR_ERR_CUDA;
+            bp.n = 0; t_end = 0;
+        }
+    }
+    if (cudaMemcpyAsync(amax_out, ws + l.amax_off, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return MOR_ERR_CUDA;
+    return MOR_OK;
+}
+
+// ---- host-memory variant: staging layout [x | codes | scale | sel | scale_f32 | block_stats | tensor_stats | workspace]
+
+namespace {
+struct Staging {
+    size_t x, codes, scale, sel, sf32, bstats, tstats, ws, ws_bytes, total;
+};
+bool staging_of(const mor_tensor_desc_t& d, int64_t codes_ld, Staging& g)
+{
+    Shape s;
+    if (shape_of(d, s) != MOR_OK) return false;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += round_up(bytes ? bytes : 1, kAlign); return o; };
+    g.x = take((size_t)d.rows * (size_t)d.ld * 2);
+    g.codes = take((size_t)d.rows * (size_t)codes_ld);
+    g.scale = take((size_t)s.n_blocks);
+    g.sel = take((size_t)s.n_blocks);
+    g.sf32 = take((size_t)s.n_blocks * 4);
+    g.bstats = take((size_t)s.n_blocks * sizeof(mor_block_stats_t));
+    g.tstats = take(sizeof(mor_tensor_stats_t));
+    g.ws_bytes = layout_of(1, s.n_tiles).total;
+    g.ws = take(g.ws_bytes);
+    g.total = off;
+    return true;
+}
+}  // namespace
+
+size_t mor_host_staging_bytes(const mor_tensor_desc_t* host_desc)
+{
+    if (host_desc == nullptr || host_desc->cols < 0 || host_desc->rows < 0) return 0;
+    Staging g;
+    if (!staging_of(*host_desc, (int64_t)round_up((size_t)host_desc->cols, 16), g)) return 0;
+    return g.total;
+}
+
+mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+                                       void* device_staging, size_t staging_bytes, void* cuda_stream)
+{
+    if (host_desc == nullptr || host_out == nullptr) return MOR_ERR_INVALID_ARG;
+    if (host_desc->group_amax != nullptr) return MOR_ERR_INVALID_ARG;
+    if (host_out->bf16_fallback != nullptr) return MOR_ERR_UNSUPPORTED;   // the fallback is the caller's own host tensor
+    if (host_desc->rows < 0 || host_desc->cols < 0 || host_desc->ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int64_t dev_codes_ld = (int64_t)round_up((size_t)host_desc->cols, 16);
+    if (host_out->codes_ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
+    Staging g;
+    if (!staging_of(*host_desc, dev_codes_ld, g)) return MOR_ERR_UNSUPPORTED;
+    if (device_staging == nullptr || staging_bytes < g.total) return MOR_ERR_WORKSPACE;
+    if (!aligned(device_staging, kAlign)) return MOR_ERR_ALIGNMENT;
+    unsigned char* base = static_cast<unsigned char*>(device_staging);
+
+    mor_tensor_desc_t d = *host_desc;
+    d.x = base + g.x;
+    mor_outputs_t o;
+    std::memset(&o, 0, sizeof(o));
+    o.codes = base + g.codes;
+    o.codes_ld = dev_codes_ld;
+    o.scale_e8m0 = base + g.scale;
+    o.sel = base + g.sel;
+    o.scale_f32 = reinterpret_cast<float*>(base + g.sf32);
+    o.block_stats = host_out->block_stats ? reinterpret_cast<mor_block_stats_t*>(base + g.bstats) : nullptr;
+    o.tensor_stats = reinterpret_cast<mor_tensor_stats_t*>(base + g.tstats);
+
+    std::vector<Item> items(1);
+    mor_status_t st = make_item(&d, o, true, 0, items[0]);
+    if (st != MOR_OK) return st;
+    if (host_out->tensor_stats == nullptr) return MOR_ERR_INVALID_ARG;
+    const Shape& s = items[0].s;
+    const size_t xbytes = (size_t)d.rows * (size_t)d.ld * 2;
+    if (xbytes && host_desc->x == nullptr) return MOR_ERR_INVALID_ARG;
+    if (xbytes && cudaMemcpyAsync(base + g.x, host_desc->x, xbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return MOR_ERR_CUDA;
+    st = run(items, base + g.ws, g.ws_bytes, stream);
+    if (st != MOR_OK) return st;
+    bool ok = true;
+    if (host_out->codes && d.rows && d.cols)
+        ok = ok && cudaMemcpy2DAsync(host_out->codes, (size_t)host_out->codes_ld, o.codes, (size_t)dev_codes_ld,
+                                     (size_t)d.cols, (size_t)d.rows, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_out->scale_e8m0 && s.n_blocks)
+        ok = ok && cudaMemcpyAsync(host_out->scale_e8m0, o.scale_e8m0, (size_t)s.n_blocks, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_out->sel && s.n_blocks)
+        ok = ok && cudaMemcpyAsync(host_out->sel, o.sel, (size_t)s.n_blocks, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_out->scale_f32 && s.n_blocks)
+        ok = ok && cudaMemcpyAsync(host_out->scale_f32, o.scale_f32, (size_t)s.n_blocks * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (host_out->block_stats && s.n_blocks)
+        ok = ok && cudaMemcpyAsync(host_out->block_stats, o.block_stats, (size_t)s.n_blocks * sizeof(mor_block_stats_t),
+                                   cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(host_out->tensor_stats, o.tensor_stats, sizeof(mor_tensor_stats_t), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    return ok ? MOR_OK : MOR_ERR_CUDA;
+}
+
+const char* mor_status_string(mor_status_t status)
+{
+    switch (status) {
+        case MOR_OK: return "ok";
+        case MOR_ERR_INVALID_ARG: return "invalid argument";
+        case MOR_ERR_UNSUPPORTED: return "unsupported recipe or block shape";
+        case MOR_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+        case MOR_ERR_WORKSPACE: return "workspace missing or too small";
+        case MOR_ERR_CUDA: return "CUDA runtime error";
+        case MOR_ERR_TIMEOUT: return "device-side wait expired";
+    }
+    return "unknown status";
+}
+
+int mor_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,118 @@
+"""The C boundary without a GPU: the library loads, exports what the header declares, and
+rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2512_22804_b200 import binding as mb
+from paper_2512_22804_b200 import build as mbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    mbuild.build()
+    return mb.load()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "mor.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mor_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_entry_point_is_exported(lib):
+    names = declared_functions()
+    assert set(names) == set(mb.EXPORTS), "binding and header list the same entry points"
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert mb.mor_version() >= 100
+    seen = {mb.mor_status_string(s) for s in range(0, 7)}
+    assert len(seen) == 7 and "ok" in seen
+
+
+def desc(rows=256, cols=256, ld=None, block=(128, 128), formats=(0, 2), crit=mb.MOR_CRIT_BLOCK_VS_E5M2, x=0x1000):
+    r = mb.Recipe(block, formats, crit)
+    return mb.make_desc(x, rows, cols, cols if ld is None else ld, r)
+
+
+def test_workspace_bytes(lib):
+    assert mb.mor_workspace_bytes([desc(64 * 128, 64 * 128)]) >= 64 * 64 * 40
+    small, big = mb.mor_workspace_bytes([desc(128, 128)]), mb.mor_workspace_bytes([desc(8192, 4096)])
+    assert 0 < small < big and small % 256 == 0
+    both = mb.mor_workspace_bytes([desc(128, 128), desc(8192, 4096, block=(1, 128))])
+    assert both >= big
+    assert mb.mor_workspace_bytes([desc(0, 128)]) > 0                     # empty tensors still get their slots
+    assert lib.mor_workspace_bytes(None, 1) == 0
+    assert mb.mor_workspace_bytes([desc(128, 128, block=(64, 64))]) == 0  # unsupported block shape
+
+
+def out_struct(codes=0x2000, codes_ld=256, ts=0x3000):
+    o = mb.mor_outputs_t()
+    o.codes, o.codes_ld, o.tensor_stats = codes, codes_ld, ts
+    o.scale_e8m0, o.sel = 0x4000, 0x5000
+    return o
+
+
+@pytest.mark.parametrize("d,o,want", [
+    (desc(block=(64, 64)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(block=(128, 1)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(formats=(1, 0, 2)), out_struct(), mb.MOR_ERR_UNSUPPORTED),       # order is fixed: E4M3 first
+    (desc(formats=(0, 1)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(formats=(0, 1, 2), crit=mb.MOR_CRIT_TENSOR_MEAN_REL), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(formats=(0, 1, 2), block=(0, 0)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(rows=-1), out_struct(), mb.MOR_ERR_INVALID_ARG),
+    (desc(ld=128), out_struct(), mb.MOR_ERR_INVALID_ARG),                  # ld < cols
+    (desc(ld=260), out_struct(), mb.MOR_ERR_ALIGNMENT),                    # ld not a multiple of 8
+    (desc(x=0x1002), out_struct(), mb.MOR_ERR_ALIGNMENT),
+    (desc(x=0), out_struct(), mb.MOR_ERR_INVALID_ARG),
+    (desc(crit=7), out_struct(), mb.MOR_ERR_INVALID_ARG),
+    (desc(), out_struct(ts=0), mb.MOR_ERR_INVALID_ARG),
+    (desc(), out_struct(codes=0), mb.MOR_ERR_INVALID_ARG),
+    (desc(), out_struct(codes_ld=250), mb.MOR_ERR_INVALID_ARG),
+    (desc(cols=250, ld=256), out_struct(codes_ld=250), mb.MOR_ERR_INVALID_ARG),   # codes_ld below roundup(cols, 16)
+    (desc(), out_struct(codes=0x2004), mb.MOR_ERR_ALIGNMENT),
+    (desc(), out_struct(), mb.MOR_ERR_WORKSPACE),                          # valid, but no workspace given
+])
+def test_bad_arguments_are_reported_before_any_launch(lib, d, o, want):
+    assert mb.mor_analyze_quantize(d, o, 0, 0) == want
+
+
+def test_threshold_and_flags_are_checked(lib):
+    d = desc()
+    d.threshold = float("nan")
+    assert mb.mor_analyze_quantize(d, out_struct(), 0, 0) == mb.MOR_ERR_INVALID_ARG
+    d = desc()
+    d.flags = 8
+    assert mb.mor_analyze_quantize(d, out_struct(), 0, 0) == mb.MOR_ERR_INVALID_ARG
+    d = desc()
+    d.scale_mode = mb.MOR_SCALE_FP32_AMAX                                   # needs the scale_f32 output
+    assert mb.mor_analyze_quantize(d, out_struct(), 0, 0) == mb.MOR_ERR_INVALID_ARG
+
+
+def test_misaligned_workspace_is_rejected(lib):
+    d = desc()
+    need = mb.mor_workspace_bytes([d])
+    assert mb.mor_analyze_quantize(d, out_struct(), 0x10010, need) == mb.MOR_ERR_ALIGNMENT
+    assert mb.mor_analyze_quantize(d, out_struct(), 0x10000, need - 1) == mb.MOR_ERR_WORKSPACE
+
+
+def test_null_descriptors(lib):
+    assert lib.mor_analyze_quantize(None, None, None, 0, None) == mb.MOR_ERR_INVALID_ARG
+    assert lib.mor_analyze_quantize_batched(None, None, 3, None, 0, None) == mb.MOR_ERR_INVALID_ARG
+    assert lib.mor_select_stats(None, None, None, None, None, None, 0, None) == mb.MOR_ERR_INVALID_ARG
+    assert lib.mor_group_amax(None, 2, None, None, 0, None) == mb.MOR_ERR_INVALID_ARG
+    assert lib.mor_host_staging_bytes(None) == 0
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(mb, "_lib", None)
+    monkeypatch.setattr(mb, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        mb.load()

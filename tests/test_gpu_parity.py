@@ -1,0 +1,296 @@
+"""Parity of the CUDA path (through the C boundary) with the CPU oracle.  Needs a B200."""
+import numpy as np
+import pytest
+
+from oracle import mor_oracle as orc
+from paper_2512_22804_b200 import binding as mb
+from paper_2512_22804_b200 import workloads as wl
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+TWO = (mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16)
+THREE = (mb.MOR_FMT_E4M3, mb.MOR_FMT_E5M2, mb.MOR_FMT_BF16)
+KINDS = [(0, 0), (1, 128), (128, 128)]
+
+
+def recipe(block, formats=TWO, criterion=mb.MOR_CRIT_BLOCK_VS_E5M2, threshold=0.045, scale_mode=mb.MOR_SCALE_GAM, flags=0):
+    return mb.Recipe(tuple(block), tuple(formats), criterion, threshold, scale_mode, flags)
+
+
+# ------------------------------------------------------------ the benchmark configurations, reduced
+
+@pytest.mark.parametrize("cfg,scale", [(0, 1), (0, 4), (1, 8), (2, 8), (3, 8), (4, 16)])
+def test_configs_reduced(cfg, scale):
+    total = exempt = 0
+    for case in wl.config_case(cfg, scale=scale):
+        rep = parity.run_and_compare(case.bits, parity.recipe_from_case(case))
+        total += rep.n_blocks
+        exempt += rep.n_exempt
+    assert exempt <= max(1, total // 1000), f"{exempt} of {total} blocks within the tolerance band"
+
+
+@pytest.mark.parametrize("block", KINDS)
+@pytest.mark.parametrize("crit", [mb.MOR_CRIT_TENSOR_MEAN_REL, mb.MOR_CRIT_BLOCK_VS_E5M2, mb.MOR_CRIT_BLOCK_MEAN_REL])
+def test_every_partition_with_every_criterion(block, crit):
+    x = wl.activation_like(384, 640, seed=41)
+    parity.run_and_compare(x, recipe(block, TWO, crit))
+    g = wl.gradient_like(256, 512, seed=42)
+    parity.run_and_compare(g, recipe(block, TWO, crit, threshold=0.2))
+
+
+@pytest.mark.parametrize("block", [(1, 128), (128, 128)])
+@pytest.mark.parametrize("flags", [0, mb.MOR_FLAG_STRICT_TIES, mb.MOR_FLAG_RANGE_MIN_INCLUDES_ZERO,
+                                   mb.MOR_FLAG_STRICT_TIES | mb.MOR_FLAG_RANGE_MIN_INCLUDES_ZERO])
+def test_three_way_with_flags(block, flags):
+    g = wl.gradient_like(384, 1024, seed=43)
+    rep = parity.run_and_compare(g, recipe(block, THREE, flags=flags))
+    assert rep.n_exempt <= 2
+    # all three formats are exercised by this workload at 1x128
+    if block == (1, 128) and flags == 0:
+        ref = orc.run(g, block, list(THREE), orc.CRIT_BLOCK_VS_E5M2)
+        assert ref.tensor["n_e4m3"] > 0 and ref.tensor["n_e5m2"] > 0 and ref.tensor["n_bf16"] > 0
+
+
+@pytest.mark.parametrize("block", KINDS)
+@pytest.mark.parametrize("mode", [mb.MOR_SCALE_GAM, mb.MOR_SCALE_E8M0, mb.MOR_SCALE_FP32_AMAX])
+def test_scale_modes(block, mode):
+    x = wl.weight_like(256, 384, seed=44)
+    parity.run_and_compare(x, recipe(block, TWO, scale_mode=mode))
+
+
+# ------------------------------------------------------------ ragged, padded, tiny and empty shapes
+
+@pytest.mark.parametrize("block", KINDS)
+@pytest.mark.parametrize("shape", [(1, 1), (1, 128), (3, 127), (129, 129), (200, 300), (127, 1000), (257, 8), (5, 2049)])
+def test_ragged_shapes(block, shape):
+    x = wl.activation_like(shape[0], shape[1], n_outlier_cols=min(4, shape[1]), seed=45)
+    ld = (shape[1] + 7) // 8 * 8 + 8
+    parity.run_and_compare(x, recipe(block, THREE if block != (0, 0) else TWO), pad_to=ld)
+
+
+@pytest.mark.parametrize("block", KINDS)
+@pytest.mark.parametrize("shape", [(0, 128), (128, 0), (0, 0)])
+def test_empty_tensors(block, shape):
+    import torch
+
+    x = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
+    out = mb.analyze_quantize(x, recipe(block))
+    ts = out.tensor_stats_dict()
+    assert ts["n_blocks"] == 0 and ts["nnz"] == 0 and ts["mean_rel_e4m3"] == 0.0
+    assert ts["tensor_format"] == mb.MOR_FMT_E4M3 and ts["group_amax"] == 0.0 and ts["group_mantissa"] == 0
+
+
+# ------------------------------------------------------------ degenerate contents
+
+@pytest.mark.parametrize("block", KINDS)
+def test_degenerate_blocks(block):
+    a = np.zeros((256, 256))
+    a[:128, :128] = 0.3                                            # constant block: exact tie in Eq. 3
+    a[128:, :128] = np.tile([448.0, 224.0, 14.0, -320.0, 0.0, 0.5, -448.0, 112.0], (128, 16)) / 256.0   # FP8-exact
+    a[128:, 128:] = 2.0 ** -20 * 1.3                               # flushed by E4M3 next to the value below
+    a[128:, 128] = 1.0
+    a[0, 200] = -0.0                                               # all-zero block with a negative zero
+    x = wl.to_bf16_bits(a)
+    for flags in (0, mb.MOR_FLAG_STRICT_TIES):
+        fm = THREE if block != (0, 0) else TWO
+        rep = parity.run_and_compare(x, recipe(block, fm, flags=flags))
+        assert rep.n_exempt == 0
+
+
+def test_values_below_binary32_normal_range_after_scaling():
+    # a block amax near the top of BF16's range makes the scale tiny; BF16 subnormals times that
+    # scale fall below 2^-126 or vanish: they still count as fully flushed non-zeros
+    a = np.zeros((4, 256), dtype=np.float64)
+    bits = wl.to_bf16_bits(a)
+    bits[:, :] = 0x0001                                            # smallest BF16 subnormal
+    bits[0, 0] = 0x7F00                                            # 1.7e38
+    bits[1, 5] = 0x7E80
+    bits[2, 128:] = 0x0040
+    bits[2, 130] = 0x7F7F                                          # largest finite BF16
+    for block in KINDS:
+        fm = THREE if block != (0, 0) else TWO
+        rep = parity.run_and_compare(bits, recipe(block, fm))
+        assert rep.n_exempt == 0
+
+
+@pytest.mark.parametrize("block", KINDS)
+def test_nonfinite_inputs(block):
+    x = wl.activation_like(256, 384, seed=46)
+    x[3, 7] = 0x7FC0; x[3, 8] = 0xFFC1; x[130, 200] = 0x7F80; x[255, 383] = 0xFF80; x[131, 0] = 0x7FFF
+    fm = THREE if block != (0, 0) else TWO
+    parity.run_and_compare(x, recipe(block, fm))
+    parity.run_and_compare(x, recipe(block, TWO, mb.MOR_CRIT_TENSOR_MEAN_REL))
+
+
+# ------------------------------------------------------------ the cast itself, exhaustively
+
+@pytest.mark.parametrize("amax_bits", [0x3F80, 0x4049, 0x3C23, 0x4B12, 0x0090, 0x7F00, 0x2D5A])
+def test_every_bf16_pattern_through_the_cast(amax_bits):
+    """All 65,536 BF16 patterns under several scales, per-tensor partition with the group amax
+    supplied (so values above it exercise saturation); NaN/inf patterns included."""
+    import torch
+
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16).reshape(512, 128)
+    amax = float(wl.bf16_bits_to_float(np.array([amax_bits], dtype=np.uint16))[0])
+    for clean in (False, True):
+        b = bits.copy()
+        if clean:
+            b[(b & 0x7F80) == 0x7F80] = 0
+        for block, fm in (((0, 0), TWO), ((1, 128), THREE), ((128, 128), THREE)):
+            r = recipe(block, fm)
+            ref = orc.run(b, r.block, list(r.formats), r.criterion, r.threshold, group_amax=amax)
+            ga = torch.tensor([amax], dtype=torch.float32, device="cuda")
+            out = mb.analyze_quantize(parity.to_device(b), r, group_amax=ga, block_stats=True, scale_f32=True)
+            parity.compare(b, r, out, ref)
+
+
+# ------------------------------------------------------------ API behaviour
+
+def test_supplied_group_amax_and_group_amax_entry_point():
+    import torch
+
+    xs = [wl.weight_like(256, 256, seed=50), wl.activation_like(130, 200, seed=51), wl.gradient_like(64, 1024, seed=52)]
+    dev = [parity.to_device(np.pad(x, ((0, 0), (0, (-x.shape[1]) % 8)))) for x in xs]
+    dev = [d[:, :x.shape[1]] for d, x in zip(dev, xs)]
+    got = mb.group_amax(dev).cpu().numpy()
+    for g, x in zip(got, xs):
+        assert g == orc.tensor_amax(x)
+    rep = parity.run_and_compare(xs[0], recipe((128, 128)), group_amax_supplied=True)
+    assert rep.n_blocks == 4
+
+
+def test_select_stats_matches_analyze_quantize():
+    import torch
+
+    g = wl.gradient_like(256, 1024, seed=53)
+    x = parity.to_device(g)
+    for block in [(1, 128), (128, 128)]:
+        r = recipe(block, THREE)
+        a = mb.analyze_quantize(x, r, block_stats=True)
+        s = mb.select_stats(x, r)
+        torch.cuda.synchronize()
+        assert a.tensor_stats_dict() == s.tensor_stats_dict()
+        assert torch.equal(a.sel, s.sel) and torch.equal(a.scale_e8m0, s.scale_e8m0)
+        assert (a.block_stats_array() == s.block_stats_array()).all()
+        ref = orc.run(g, r.block, list(r.formats), r.criterion, r.threshold)
+        parity.compare(g, r, s, ref)
+
+
+def test_bf16_fallback_copies_only_rejected_blocks():
+    import torch
+
+    g = wl.gradient_like(300, 1000, seed=54)
+    host = np.zeros((300, 1008), dtype=np.uint16); host[:, :1000] = g
+    x = parity.to_device(host)
+    for block in [(1, 128), (128, 128)]:
+        r = recipe(block, THREE)
+        out = mb.analyze_quantize(x, r, cols=1000, fallback=True)
+        torch.cuda.synchronize()
+        fb = out.bf16_fallback.view(torch.int16).cpu().numpy().view(np.uint16)
+        sel = out.sel.cpu().numpy()
+        assert (sel == mb.MOR_FMT_BF16).any() and (sel != mb.MOR_FMT_BF16).any()
+        br, bc = block
+        for bi in range(sel.shape[0]):
+            for bj in range(sel.shape[1]):
+                sl = (slice(bi * br, min((bi + 1) * br, 300)), slice(bj * bc, min((bj + 1) * bc, 1000)))
+                want = host[sl] if sel[bi, bj] == mb.MOR_FMT_BF16 else 0
+                assert (fb[sl] == want).all()
+        assert (fb[:, 1000:] == 0).all()
+
+
+def test_batched_call_equals_single_calls():
+    import torch
+
+    cases = wl.llama_layer_cases(scale=16)
+    cases += wl.config_case(0, scale=2) + wl.config_case(3, scale=16)
+    xs = [parity.to_device(c.bits) for c in cases]
+    recipes = [parity.recipe_from_case(c) for c in cases]
+    plan = mb.BatchPlan(xs, recipes, block_stats=True)
+    plan.run()
+    torch.cuda.synchronize()
+    for c, x, r, o in zip(cases, xs, recipes, plan.outs):
+        single = mb.analyze_quantize(x, r, block_stats=True)
+        torch.cuda.synchronize()
+        assert o.tensor_stats_dict() == single.tensor_stats_dict(), c.name
+        assert torch.equal(o.codes, single.codes) and torch.equal(o.sel, single.sel)
+        assert torch.equal(o.scale_e8m0, single.scale_e8m0)
+        ref = orc.run(c.bits, r.block, list(r.formats), r.criterion, r.threshold)
+        parity.compare(c.bits, r, o, ref)
+
+
+def test_many_tensors_exceeding_one_launch():
+    import torch
+
+    rng = np.random.default_rng(60)
+    bits = [wl.weight_like(int(rng.integers(1, 300)), int(rng.integers(1, 40)) * 8, seed=61 + i) for i in range(47)]
+    xs = [parity.to_device(b) for b in bits]
+    recipes = [recipe(KINDS[i % 3]) for i in range(47)]
+    plan = mb.BatchPlan(xs, recipes)
+    plan.run()
+    torch.cuda.synchronize()
+    for b, r, o in zip(bits, recipes, plan.outs):
+        ref = orc.run(b, r.block, list(r.formats), r.criterion, r.threshold)
+        parity.compare(b, r, o, ref)
+
+
+def test_runs_are_deterministic():
+    import torch
+
+    g = wl.gradient_like(512, 2048, seed=55)
+    x = parity.to_device(g)
+    for block in KINDS:
+        r = recipe(block, THREE if block != (0, 0) else TWO)
+        a = mb.analyze_quantize(x, r, block_stats=True)
+        b = mb.analyze_quantize(x, r, block_stats=True)
+        torch.cuda.synchronize()
+        assert torch.equal(a.codes, b.codes) and torch.equal(a.sel, b.sel) and torch.equal(a.tensor_stats, b.tensor_stats)
+        assert torch.equal(a.block_stats, b.block_stats)
+
+
+def test_host_memory_entry_point():
+    import ctypes as C
+    import torch
+
+    g = wl.gradient_like(300, 1000, seed=56)
+    host = np.zeros((300, 1008), dtype=np.uint16); host[:, :1000] = g
+    r = recipe((1, 128), THREE)
+    hx = torch.from_numpy(host.view(np.int16)).pin_memory()
+    d = mb.make_desc(hx.data_ptr(), 300, 1000, 1008, r)
+    grid = mb.grid_of(300, 1000, r.block)
+    codes = torch.zeros((300, 1000), dtype=torch.uint8).pin_memory()
+    scale = torch.zeros(grid, dtype=torch.uint8).pin_memory()
+    sel = torch.zeros(grid, dtype=torch.uint8).pin_memory()
+    ts = torch.zeros((mb.TENSOR_STATS_DTYPE.itemsize,), dtype=torch.uint8).pin_memory()
+    o = mb.mor_outputs_t()
+    o.codes, o.codes_ld, o.scale_e8m0, o.sel, o.tensor_stats = codes.data_ptr(), 1000, scale.data_ptr(), sel.data_ptr(), ts.data_ptr()
+    nbytes = mb.mor_host_staging_bytes(d)
+    staging = torch.empty((nbytes,), dtype=torch.uint8, device="cuda")
+    st = mb.mor_analyze_quantize_host(d, o, staging.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream)
+    assert st == mb.MOR_OK
+    torch.cuda.synchronize()
+    ref = orc.run(host, r.block, list(r.formats), r.criterion, r.threshold, cols=1000)
+    np.testing.assert_array_equal(codes.numpy(), ref.codes)
+    np.testing.assert_array_equal(sel.numpy().reshape(-1), ref.sel)
+    np.testing.assert_array_equal(scale.numpy().reshape(-1), ref.scale_e8m0)
+    rec = ts.numpy().view(mb.TENSOR_STATS_DTYPE)[0]
+    assert rec["nnz"] == ref.tensor["nnz"] and rec["group_mantissa"] == ref.tensor["group_mantissa"]
+
+
+def test_invalid_arguments_launch_nothing():
+    import torch
+
+    x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mb.MorError) as e:
+        mb.analyze_quantize(x, recipe((64, 64)))
+    assert e.value.status == mb.MOR_ERR_UNSUPPORTED
+    with pytest.raises(mb.MorError) as e:
+        mb.analyze_quantize(x, recipe((1, 128), (mb.MOR_FMT_E5M2, mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16)))
+    assert e.value.status == mb.MOR_ERR_UNSUPPORTED
+    with pytest.raises(mb.MorError) as e:
+        mb.analyze_quantize(x[:, 1:], recipe((1, 128)))                     # misaligned base, odd leading dimension
+    assert e.value.status == mb.MOR_ERR_ALIGNMENT
+    d = mb.desc_for(x, recipe((1, 128)))
+    o = mb.alloc_outputs(128, 256, recipe((1, 128)), x.device)
+    assert mb.mor_analyze_quantize(d, o.c_struct, 0, 0) == mb.MOR_ERR_WORKSPACE
+    torch.cuda.synchronize()
