@@ -194,14 +194,14 @@ def main():
     # ---- timed region: K steps, CUDA events on the launching stream, stage events around the main kernel
     K = args.steps
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(K)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     stage = []
     for a, b in ev:
+        a.record(stream); b.record(stream)       # torch creates the CUDA event on first record
         s = mb.mor_stage_events_t()
         s.main_begin, s.main_end = a.cuda_event, b.cuda_event
+        assert s.main_begin and s.main_end
         stage.append(s)
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for a, b in ev:          # events must exist before their handles are passed down
-        a.record(stream); b.record(stream)
     sync_all()
     sampler = ClockSampler(local_rank)
     sampler.start()

@@ -93,9 +93,12 @@ typedef struct mor_tensor_desc {
     float   threshold;      /* th of Eq. 2 as a fraction (0.045 = the paper's 4.5 %)         */
     int32_t scale_mode;     /* mor_scale_mode_t                                              */
     uint32_t flags;         /* MOR_FLAG_*                                                    */
-    const float* group_amax;/* DEVICE, optional.  max|x| over the tensor if the caller has
-                               it already (GAM only); NULL = the library computes it with
-                               one extra read of the tensor                                  */
+    const float* group_amax;/* DEVICE, optional.  g_amax of Algorithm 1 if the caller has it
+                               already: it fixes the shared mantissa; block amaxes are still
+                               taken from the data, so a stale value cannot cause saturation.
+                               NULL = the library computes it with one extra read of the
+                               tensor (always done for the (0,0) partition, whose block amax
+                               is the tensor amax)                                           */
 } mor_tensor_desc_t;
 
 /* Per-block quantities behind the decisions (Eq. 3 sums, Eq. 4 range). */

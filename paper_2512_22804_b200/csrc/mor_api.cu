@@ -127,7 +127,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.fallback = static_cast<uint16_t*>(it.o.bf16_fallback);
     r.block_stats = it.o.block_stats;
     r.tensor_stats = it.o.tensor_stats;
-    r.amax = d.group_amax ? d.group_amax : reinterpret_cast<const float*>(ws + l.amax_off) + it.index;
+    r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
+    r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
@@ -172,7 +173,9 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
             return ok;
         };
         for (const Item& it : items) {
-            if (it.d->group_amax || it.s.amax_tiles == 0) continue;
+            // a supplied group amax only fixes the shared mantissa; the per-tensor partition still
+            // needs its block amax, which is the tensor amax, from the data (Algorithm 1)
+            if ((it.d->group_amax && it.s.kind != KIND_TENSOR) || it.s.amax_tiles == 0) continue;
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);
             r.n_units = (uint32_t)((uint64_t)it.d->rows * it.s.nbc);   // row pieces, whatever the partition

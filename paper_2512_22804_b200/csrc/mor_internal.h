@@ -38,7 +38,8 @@ struct TensorRec {
     uint16_t* fallback;
     mor_block_stats_t* block_stats;
     mor_tensor_stats_t* tensor_stats;
-    const float* amax;            // tensor amax on the device (workspace slot or the caller's)
+    const float* amax;            // group amax on the device (workspace slot or the caller's)
+    float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
     int64_t rows, cols, ld, codes_ld;
     uint32_t nbc;                 // segments per row = ceil(cols / 128)

@@ -188,70 +188,124 @@ __device__ __forceinline__ void load_tile_async(const TensorRec& R, const TileSh
     }
 }
 
-// max over |x| of a thread's 64 elements as BF16 bits; NaN and inf win (they compare above
-// every finite pattern), which is how a non-finite input is noticed
-__device__ __forceinline__ uint32_t raw_amax_half_segment(const unsigned char* half, int t)
+// Block statistics of a thread's 64 elements in one pass over packed BF16 pairs:
+//   mx  per-halfword max of the |x| bit patterns.  NaN and inf compare above every finite
+//       pattern, which is how a non-finite input is noticed.
+//   mn  per-halfword min of (|x| bits - 1) mod 2^16: zeros wrap to 0xFFFF and drop out, so
+//       mn + 1 is the smallest non-zero |x| (Eq. 4, and the check for values that leave
+//       binary32's normal range after scaling).
+__device__ __forceinline__ void scan_half_segment(const unsigned char* half, int t, uint32_t& amax_bits, uint32_t& minm1_bits)
 {
-    __nv_bfloat162 m = __float2bfloat162_rn(0.0f);
+    uint32_t mx = 0u, mn = 0xFFFFFFFFu;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const uint4 v = lds128(half + (((j + t) & 7) << 4));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&w[i]);
-            m = __hmax2_nan(m, __habs2(a));
-        }
+        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+        mx = __vimax3_u16x2(mx, a0, a1);
+        mx = __vimax3_u16x2(mx, a2, a3);
+        mn = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn);
+        mn = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn);
+        mn = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn);
+        mn = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn);
     }
-    const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m);
-    return max(mb & 0xFFFFu, mb >> 16);
+    amax_bits = max(mx & 0xFFFFu, mx >> 16);
+    minm1_bits = min(mn & 0xFFFFu, mn >> 16);
 }
 
 // the same over finite elements only (used once a non-finite element has been seen)
-__device__ __forceinline__ uint32_t finite_amax_half_segment(const unsigned char* half, int t)
+__device__ __forceinline__ void scan_half_segment_finite(const unsigned char* half, int t, uint32_t& amax_bits, uint32_t& minm1_bits)
 {
-    uint32_t m = 0;
+    uint32_t m = 0u, n = 0xFFFFu;
 #pragma unroll 1
     for (int j = 0; j < 8; ++j) {
         const uint4 v = lds128(half + (((j + t) & 7) << 4));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
         for (int i = 0; i < 4; ++i) {
             const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
-            if (lo < kBf16Inf) m = max(m, lo);
-            if (hi < kBf16Inf) m = max(m, hi);
+            if (lo < kBf16Inf) { m = max(m, lo); n = min(n, (lo - 1u) & 0xFFFFu); }
+            if (hi < kBf16Inf) { m = max(m, hi); n = min(n, (hi - 1u) & 0xFFFFu); }
         }
     }
-    return m;
+    amax_bits = m;
+    minm1_bits = n;
 }
 
 struct Acc {
     float a43[4], a52[4];
-    uint32_t nnz, nbig, nonfinite, mn;   // mn: min over non-zeros of (|x| bits << 16) - 1
+    uint32_t nnz, nbig, nonfinite;
 };
 
-// One BF16 pair -> two E4M3 codes (and two E5M2 codes), with its terms of Eq. 1-3.
-//   y = fl32(x * scale); c = RNE-saturating cast; q = value of c; term = |y - q| / |y|.
-// Terms are accumulated only where |y| is a normal binary32; the few non-zero elements
-// below that (they are flushed by both formats, term = 1) are added from the counts
-// nnz - nbig by the caller.
-template <bool YARD, bool THREE, bool SLOW>
-__device__ __forceinline__ void convert_pair(uint32_t w, float s4, float s5, int lane, Acc& A,
-                                             uint32_t& c4, uint32_t& c5)
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+// two IEEE binary32 multiplies in one instruction (each lane rounds to nearest even)
+__device__ __forceinline__ void mul_f32x2(unsigned long long a, unsigned long long b, float& lo, float& hi)
+{
+    unsigned long long r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ float rcp_ftz(float a)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+
+// Fast path for one BF16 pair: two E4M3 codes (and two E5M2 codes) with their terms of
+// Eq. 1-3.   y = fl32(x * scale); c = RNE-saturating cast; q = value of c;
+// term = |y - q| / |y|, formed as |y - q| * rcp(|y| + 2^-126).  The caller guarantees that
+// the block holds no NaN/inf and that every non-zero |y| is at least 2^-100, so the added
+// constant changes a term by less than 2^-26 relative, and a zero element gives 0 * finite.
+template <bool YARD>
+__device__ __forceinline__ void convert_pair_fast(uint32_t w, unsigned long long s4x2, unsigned long long s5x2, int lane,
+                                                  float (&a43)[4], float (&a52)[4], __nv_bfloat162& cnt,
+                                                  uint32_t& c4, uint32_t& c5)
+{
+    const __nv_bfloat162 xb = *reinterpret_cast<const __nv_bfloat162*>(&w);
+    cnt = __hadd2(cnt, __hneu2(xb, __float2bfloat162_rn(0.0f)));          // non-zero count, exact up to 256 per half
+    const unsigned long long x2 = pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    float ylo, yhi;
+    mul_f32x2(x2, s4x2, ylo, yhi);
+    c4 = cvt_e4m3x2(yhi, ylo);
+    const uint32_t q4 = e4m3x2_to_f16x2(c4);
+    const float dlo = diff_f16_f32(static_cast<uint16_t>(q4 & 0xFFFFu), ylo);
+    const float dhi = diff_f16_f32(static_cast<uint16_t>(q4 >> 16), yhi);
+    const float rlo = rcp_ftz(fabsf(ylo) + FLT_MIN), rhi = rcp_ftz(fabsf(yhi) + FLT_MIN);
+    a43[lane] = fmaf(fabsf(dlo), rlo, a43[lane]);
+    a43[lane] = fmaf(fabsf(dhi), rhi, a43[lane]);
+    if (YARD) {
+        float zlo, zhi;
+        mul_f32x2(x2, s5x2, zlo, zhi);
+        c5 = cvt_e5m2x2(zhi, zlo);
+        const uint32_t q5 = e5m2x2_to_f16x2(c5);
+        const float elo = diff_f16_f32(static_cast<uint16_t>(q5 & 0xFFFFu), zlo);
+        const float ehi = diff_f16_f32(static_cast<uint16_t>(q5 >> 16), zhi);
+        // |z - q'| / |z| = |z - q'| * (1/|y|) * (scale4/scale5); the power-of-two ratio is applied once per block
+        a52[lane] = fmaf(fabsf(elo), rlo, a52[lane]);
+        a52[lane] = fmaf(fabsf(ehi), rhi, a52[lane]);
+    } else {
+        c5 = 0;
+    }
+}
+
+// Careful path for one BF16 pair: handles NaN/inf elements (stated reading: ignored by
+// every count and sum, NaN -> 0x7F, +-inf -> +-largest finite) and non-zero elements whose
+// scaled value leaves binary32's normal range (flushed by both formats: term 1, added by
+// the caller from the counts nnz - nbig).
+template <bool YARD>
+__device__ __forceinline__ void convert_pair_careful(uint32_t w, float s4, float s5, int lane, Acc& A,
+                                                     uint32_t& c4, uint32_t& c5)
 {
     const uint32_t blo = w << 16, bhi = w & 0xFFFF0000u;
     const uint32_t alo = blo & 0x7FFFFFFFu, ahi = bhi & 0x7FFFFFFFu;
     const float xlo = __uint_as_float(blo), xhi = __uint_as_float(bhi);
-    bool uselo = true, usehi = true;
-    if (SLOW) {
-        uselo = alo < 0x7F800000u;
-        usehi = ahi < 0x7F800000u;
-        A.nonfinite += (uselo ? 0u : 1u) + (usehi ? 0u : 1u);
-    }
+    const bool uselo = alo < 0x7F800000u, usehi = ahi < 0x7F800000u;
+    A.nonfinite += (uselo ? 0u : 1u) + (usehi ? 0u : 1u);
     A.nnz += ((alo != 0u && uselo) ? 1u : 0u) + ((ahi != 0u && usehi) ? 1u : 0u);
-    if (THREE) {
-        if (uselo) A.mn = min(A.mn, alo - 1u);
-        if (usehi) A.mn = min(A.mn, ahi - 1u);
-    }
 
     const float ylo = __fmul_rn(xlo, s4), yhi = __fmul_rn(xhi, s4);
     c4 = cvt_e4m3x2(yhi, ylo);
@@ -270,67 +324,99 @@ __device__ __forceinline__ void convert_pair(uint32_t w, float s4, float s5, int
         const uint32_t q5 = e5m2x2_to_f16x2(c5);
         const float elo = diff_f16_f32(static_cast<uint16_t>(q5 & 0xFFFFu), zlo);
         const float ehi = diff_f16_f32(static_cast<uint16_t>(q5 >> 16), zhi);
-        // |z - q'| / |z| = |z - q'| * (1/|y|) * (scale4/scale5); the power-of-two ratio is
-        // applied once per block
         if (biglo) A.a52[lane] = fmaf(fabsf(elo), rlo, A.a52[lane]);
         if (bighi) A.a52[lane] = fmaf(fabsf(ehi), rhi, A.a52[lane]);
     } else {
         c5 = 0;
     }
-
-    if (SLOW) {
-        // stated reading for non-finite inputs: NaN -> 0x7F, +-inf -> +-largest finite
-        if (!uselo) {
-            const bool nan = (alo & 0x007F0000u) != 0u;
-            const uint32_t sg = (blo >> 24) & 0x80u;
-            c4 = (c4 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Eu));
-            c5 = (c5 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Bu));
-        }
-        if (!usehi) {
-            const bool nan = (ahi & 0x007F0000u) != 0u;
-            const uint32_t sg = (bhi >> 24) & 0x80u;
-            c4 = (c4 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Eu)) << 8);
-            c5 = (c5 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Bu)) << 8);
-        }
+    if (!uselo) {
+        const bool nan = (alo & 0x007F0000u) != 0u;
+        const uint32_t sg = (blo >> 24) & 0x80u;
+        c4 = (c4 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Eu));
+        c5 = (c5 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Bu));
+    }
+    if (!usehi) {
+        const bool nan = (ahi & 0x007F0000u) != 0u;
+        const uint32_t sg = (bhi >> 24) & 0x80u;
+        c4 = (c4 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Eu)) << 8);
+        c5 = (c5 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Bu)) << 8);
     }
 }
 
 // A thread's 64 elements.  E4M3 codes go to shared memory at once unless the recipe is
 // three-way, where both code sets wait in registers for the block's decision.
-template <bool YARD, bool THREE, bool SLOW, bool STORE>
+// Results: e43 = the thread's sum of E4M3 terms, complete; e52 = its sum of E5M2 terms still
+// to be multiplied by scale4/scale5 and then increased by `tiny` (the count of non-zeros
+// flushed below binary32's normal range, already inside e43); nnz; nonfinite.
+template <bool YARD, bool THREE, bool CAREFUL, bool STORE>
 __device__ __forceinline__ void convert_half_segment(const unsigned char* half_in, unsigned char* half_out, int t,
-                                                     float s4, float s5, Acc& A, uint2 (&k4)[8], uint2 (&k5)[8])
+                                                     float s4, float s5, float& e43, float& e52, float& tiny,
+                                                     uint32_t& nnz, uint32_t& nonfinite, uint2 (&k4)[8], uint2 (&k5)[8])
 {
+    Acc A;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { A.a43[i] = 0.0f; A.a52[i] = 0.0f; }
+    A.nnz = A.nbig = A.nonfinite = 0u;
+    __nv_bfloat162 cnt = __float2bfloat162_rn(0.0f);
+    const unsigned long long s4x2 = pack_f32x2(s4, s4), s5x2 = pack_f32x2(s5, s5);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int kk = (j + t) & 7;
         const uint4 v = lds128(half_in + (kk << 4));
         uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-        convert_pair<YARD, THREE, SLOW>(v.x, s4, s5, 0, A, a0, b0);
-        convert_pair<YARD, THREE, SLOW>(v.y, s4, s5, 1, A, a1, b1);
-        convert_pair<YARD, THREE, SLOW>(v.z, s4, s5, 2, A, a2, b2);
-        convert_pair<YARD, THREE, SLOW>(v.w, s4, s5, 3, A, a3, b3);
-        const uint2 c4 = make_uint2(a0 | (a1 << 16), a2 | (a3 << 16));
+        if (CAREFUL) {
+            convert_pair_careful<YARD>(v.x, s4, s5, 0, A, a0, b0);
+            convert_pair_careful<YARD>(v.y, s4, s5, 1, A, a1, b1);
+            convert_pair_careful<YARD>(v.z, s4, s5, 2, A, a2, b2);
+            convert_pair_careful<YARD>(v.w, s4, s5, 3, A, a3, b3);
+        } else {
+            convert_pair_fast<YARD>(v.x, s4x2, s5x2, 0, A.a43, A.a52, cnt, a0, b0);
+            convert_pair_fast<YARD>(v.y, s4x2, s5x2, 1, A.a43, A.a52, cnt, a1, b1);
+            convert_pair_fast<YARD>(v.z, s4x2, s5x2, 2, A.a43, A.a52, cnt, a2, b2);
+            convert_pair_fast<YARD>(v.w, s4x2, s5x2, 3, A.a43, A.a52, cnt, a3, b3);
+        }
+        const uint2 c4 = make_uint2(__byte_perm(a0, a1, 0x5410), __byte_perm(a2, a3, 0x5410));
         if (THREE) {
             k4[j] = c4;
-            k5[j] = make_uint2(b0 | (b1 << 16), b2 | (b3 << 16));
+            k5[j] = make_uint2(__byte_perm(b0, b1, 0x5410), __byte_perm(b2, b3, 0x5410));
         } else if (STORE) {
             *reinterpret_cast<uint2*>(half_out + (kk << 3)) = c4;
         }
     }
+    tiny = 0.0f;
+    if (CAREFUL) {
+        nnz = A.nnz;
+        nonfinite = A.nonfinite;
+        tiny = (float)(A.nnz - A.nbig);
+    } else {
+        nnz = (uint32_t)(__low2float(cnt) + __high2float(cnt));
+        nonfinite = 0u;
+    }
+    e43 = ((A.a43[0] + A.a43[1]) + (A.a43[2] + A.a43[3])) + tiny;
+    e52 = (A.a52[0] + A.a52[1]) + (A.a52[2] + A.a52[3]);
 }
-
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;
 }
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
+{
+    return minm1_bits == 0xFFFFu ? __uint_as_float(0x7F800000u) : __uint_as_float((minm1_bits + 1u) << 16);
+}
 
 // Algorithm 2 for one block with the per-block metrics (M_1 = Eq. 3, M_2 = Eq. 4, or
 // Eq. 1-2 on the block alone).
 __device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43, double e52, uint32_t nnz,
-                                                 uint32_t nonfinite, uint32_t amax_bits, uint32_t mn,
+                                                 uint32_t nonfinite, uint32_t amax_bits, uint32_t minm1_bits,
                                                  uint32_t n_elems)
 {
     if (nonfinite) return MOR_FMT_BF16;
@@ -339,7 +425,7 @@ __device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43,
         if (ok) return MOR_FMT_E4M3;
         if (R.n_formats == 3) {
             // max|b| < (57344 * 2^14) * min|b|, exact in binary32 (11 significant bits)
-            float mnv = (mn == 0xFFFFFFFFu) ? __uint_as_float(0x7F800000u) : __uint_as_float(mn + 1u);
+            float mnv = minnz_value(minm1_bits);
             if ((R.flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) && nnz < n_elems) mnv = 0.0f;
             const float amax = __uint_as_float(amax_bits << 16);
             if (amax < 939524096.0f * mnv) return MOR_FMT_E5M2;
@@ -383,68 +469,77 @@ mor_main_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ par
     const unsigned char* half_in = s_in + seg * 256 + (t & 1) * 128;
     unsigned char* half_out = s_out + seg * 128 + (t & 1) * 64;
 
-    // ---- block amax (Algorithm 1) ----
-    uint32_t amax_bits = raw_amax_half_segment(half_in, t);
-    bool slow;
+    // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
+    uint32_t amax_bits, minm1;
+    scan_half_segment(half_in, t, amax_bits, minm1);
+    bool nonfin;
     if (KIND == KIND_ROW128) {
         amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, 1));
-        slow = __any_sync(0xFFFFFFFFu, amax_bits >= kBf16Inf);
-        if (slow) {
-            amax_bits = finite_amax_half_segment(half_in, t);
+        minm1 = min(minm1, __shfl_xor_sync(0xFFFFFFFFu, minm1, 1));
+        nonfin = __any_sync(0xFFFFFFFFu, amax_bits >= kBf16Inf);          // warp-uniform
+        if (nonfin) {
+            scan_half_segment_finite(half_in, t, amax_bits, minm1);
             amax_bits = max(amax_bits, __shfl_xor_sync(0xFFFFFFFFu, amax_bits, 1));
+            minm1 = min(minm1, __shfl_xor_sync(0xFFFFFFFFu, minm1, 1));
         }
     } else {
         amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
-        if (lane == 0) sh.wmax[warp] = amax_bits;
+        minm1 = __reduce_min_sync(0xFFFFFFFFu, minm1);
+        if (lane == 0) sh.wmax[warp] = (amax_bits << 16) | (0xFFFFu - minm1);   // both halves reduce with max
         __syncthreads();
-        amax_bits = sh.wmax[0];
+        uint32_t hi = 0u, lo = 0u;
 #pragma unroll
-        for (int i = 1; i < kThreads / 32; ++i) amax_bits = max(amax_bits, sh.wmax[i]);
-        slow = amax_bits >= kBf16Inf;
-        if (slow) {                                         // CTA-uniform
+        for (int i = 0; i < kThreads / 32; ++i) { hi = max(hi, sh.wmax[i] >> 16); lo = max(lo, sh.wmax[i] & 0xFFFFu); }
+        amax_bits = hi; minm1 = 0xFFFFu - lo;
+        nonfin = amax_bits >= kBf16Inf;                                   // CTA-uniform
+        if (nonfin) {
             __syncthreads();
-            amax_bits = __reduce_max_sync(0xFFFFFFFFu, finite_amax_half_segment(half_in, t));
-            if (lane == 0) sh.wmax[warp] = amax_bits;
+            scan_half_segment_finite(half_in, t, amax_bits, minm1);
+            amax_bits = __reduce_max_sync(0xFFFFFFFFu, amax_bits);
+            minm1 = __reduce_min_sync(0xFFFFFFFFu, minm1);
+            if (lane == 0) sh.wmax[warp] = (amax_bits << 16) | (0xFFFFu - minm1);
             __syncthreads();
-            amax_bits = sh.wmax[0];
-            for (int i = 1; i < kThreads / 32; ++i) amax_bits = max(amax_bits, sh.wmax[i]);
+            hi = 0u; lo = 0u;
+            for (int i = 0; i < kThreads / 32; ++i) { hi = max(hi, sh.wmax[i] >> 16); lo = max(lo, sh.wmax[i] & 0xFFFFu); }
+            amax_bits = hi; minm1 = 0xFFFFu - lo;
         }
     }
-    // per-tensor partition: the block is the tensor, its amax is the group amax
-    const float b_amax = (KIND == KIND_TENSOR) ? g_amax : __uint_as_float(amax_bits << 16);
-    if (KIND == KIND_TENSOR) amax_bits = __float_as_uint(g_amax) >> 16;
+    // per-tensor partition: the block is the tensor, its amax was reduced by the pre-pass
+    const float b_amax = (KIND == KIND_TENSOR) ? *R.amax_slot : __uint_as_float(amax_bits << 16);
+    if (KIND == KIND_TENSOR) amax_bits = __float_as_uint(b_amax) >> 16;
 
     uint32_t s4b, s5b;
     block_scale(b_amax, m_g, R.scale_mode, s4b, s5b);
     const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
 
-    // ---- cast and error terms ----
-    Acc A;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { A.a43[i] = 0.0f; A.a52[i] = 0.0f; }
-    A.nnz = A.nbig = A.nonfinite = 0u;
-    A.mn = 0xFFFFFFFFu;
-    uint2 k4[8], k5[8];
-    if (slow) convert_half_segment<YARD, THREE, true, STORE>(half_in, half_out, t, s4, s5, A, k4, k5);
-    else      convert_half_segment<YARD, THREE, false, STORE>(half_in, half_out, t, s4, s5, A, k4, k5);
+    // The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_pair_fast).
+    // minm1 covers this thread's block (ROW128), this tile (BLK128, TENSOR).
+    bool careful = nonfin;
+    if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), s4) >= 7.888609052210118e-31f);
+    if (KIND == KIND_ROW128) careful = __any_sync(0xFFFFFFFFu, careful);
 
-    const float tiny = (float)(A.nnz - A.nbig);             // non-zeros below binary32's normal range: term 1
-    float e43 = ((A.a43[0] + A.a43[1]) + (A.a43[2] + A.a43[3])) + tiny;
+    // ---- cast and error terms ----
+    float e43, e52, tiny;
+    uint32_t nnz, nonf;
+    uint2 k4[8], k5[8];
+    if (careful) convert_half_segment<YARD, THREE, true, STORE>(half_in, half_out, t, s4, s5, e43, e52, tiny, nnz, nonf, k4, k5);
+    else         convert_half_segment<YARD, THREE, false, STORE>(half_in, half_out, t, s4, s5, e43, e52, tiny, nnz, nonf, k4, k5);
     // scale4 / scale5 = 2^(e4 - e5)
     const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);
-    float e52 = YARD ? ((A.a52[0] + A.a52[1]) + (A.a52[2] + A.a52[3])) * ratio + tiny : 0.0f;
+    e52 = YARD ? e52 * ratio + tiny : 0.0f;
 
     // ---- block sums, decision, per-tile partial ----
-    WarpPart wp;
     uint32_t sel = MOR_FMT_E4M3;
+    float w43, w52;                 // what this thread adds to the tile's sums
+    uint32_t wcnt = 0u;             // n_e4m3 | n_e5m2 << 8 | n_bf16 << 16 (at most 128 blocks per tile)
+    uint32_t wnz = nnz | (nonf << 16);   // at most 64 per thread, 16384 per tile
     if (KIND == KIND_ROW128) {
         e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
         e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
-        const uint32_t nnz = A.nnz + __shfl_xor_sync(0xFFFFFFFFu, A.nnz, 1);
-        const uint32_t nonf = A.nonfinite + __shfl_xor_sync(0xFFFFFFFFu, A.nonfinite, 1);
-        const uint32_t mn = min(A.mn, __shfl_xor_sync(0xFFFFFFFFu, A.mn, 1));
+        const uint32_t pz = wnz + __shfl_xor_sync(0xFFFFFFFFu, wnz, 1);
+        const uint32_t bnnz = pz & 0xFFFFu, bnonf = pz >> 16;
         const int n_el = sh.seg_n[seg];
-        sel = decide_block(R, (double)e43, (double)e52, nnz, nonf, amax_bits, mn, (uint32_t)n_el);
+        sel = decide_block(R, (double)e43, (double)e52, bnnz, bnonf, amax_bits, minm1, (uint32_t)n_el);
         const bool lead = (t & 1) == 0 && n_el > 0;
         if (lead) {
             const uint32_t b = local * (uint32_t)kSegsPerTile + (uint32_t)seg;
@@ -455,34 +550,32 @@ mor_main_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ par
             if (R.block_stats) {
                 mor_block_stats_t bs;
                 bs.amax = b_amax;
-                bs.min_abs_nz = (mn == 0xFFFFFFFFu) ? __uint_as_float(0x7F800000u) : __uint_as_float(mn + 1u);
-                bs.nnz = nnz; bs.n_nonfinite = nonf; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
+                bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                bs.nnz = bnnz; bs.n_nonfinite = bnonf; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
                 R.block_stats[b] = bs;
             }
             sh.blk_sel[seg] = (uint8_t)sel;
+            wcnt = 1u << (8 * sel);
         }
-        wp.s43 = lead ? (double)e43 : 0.0;
-        wp.s52 = lead ? (double)e52 : 0.0;
-        wp.nnz = lead ? nnz : 0u;
-        wp.nonfinite = lead ? nonf : 0u;
-        wp.n4 = (lead && sel == MOR_FMT_E4M3) ? 1u : 0u;
-        wp.n5 = (lead && sel == MOR_FMT_E5M2) ? 1u : 0u;
-        wp.nb = (lead && sel == MOR_FMT_BF16) ? 1u : 0u;
-        wp.mn = mn;
+        w43 = lead ? e43 : 0.0f;
+        w52 = lead ? e52 : 0.0f;
     } else {
-        wp.s43 = (double)e43; wp.s52 = (double)e52;
-        wp.nnz = A.nnz; wp.nonfinite = A.nonfinite;
-        wp.n4 = wp.n5 = wp.nb = 0u;
-        wp.mn = A.mn;
+        w43 = e43; w52 = e52;
     }
-    wp.s43 = warp_sum(wp.s43);
-    wp.s52 = warp_sum(wp.s52);
-    wp.nnz = __reduce_add_sync(0xFFFFFFFFu, wp.nnz);
-    wp.nonfinite = __reduce_add_sync(0xFFFFFFFFu, wp.nonfinite);
-    wp.n4 = __reduce_add_sync(0xFFFFFFFFu, wp.n4);
-    wp.n5 = __reduce_add_sync(0xFFFFFFFFu, wp.n5);
-    wp.nb = __reduce_add_sync(0xFFFFFFFFu, wp.nb);
-    wp.mn = __reduce_min_sync(0xFFFFFFFFu, wp.mn);
+    WarpPart wp;
+    if (KIND == KIND_ROW128) {
+        // block sums are binary32 already; add them up in binary32 inside the warp
+        wp.s43 = (double)warp_sum(w43);
+        wp.s52 = (double)warp_sum(w52);
+    } else {
+        wp.s43 = warp_sum((double)w43);
+        wp.s52 = warp_sum((double)w52);
+    }
+    wnz = __reduce_add_sync(0xFFFFFFFFu, wnz);
+    wcnt = __reduce_add_sync(0xFFFFFFFFu, wcnt);
+    wp.nnz = wnz & 0xFFFFu; wp.nonfinite = wnz >> 16;
+    wp.n4 = wcnt & 0xFFu; wp.n5 = (wcnt >> 8) & 0xFFu; wp.nb = wcnt >> 16;
+    wp.mn = (KIND == KIND_ROW128) ? __reduce_min_sync(0xFFFFFFFFu, minm1) : minm1;
     if (lane == 0) sh.wp[warp] = wp;
     __syncthreads();
 
@@ -497,7 +590,7 @@ mor_main_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ par
             const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
             const long long rr = R.rows - (long long)bi * 128, cc = R.cols - (long long)bj * 128;
             const uint32_t n_el = (uint32_t)((rr < 128 ? rr : 128) * (cc < 128 ? cc : 128));
-            const uint32_t bsel = decide_block(R, tot.s43, tot.s52, tot.nnz, tot.nonfinite, amax_bits, tot.mn, n_el);
+            const uint32_t bsel = decide_block(R, tot.s43, tot.s52, tot.nnz, tot.nonfinite, amax_bits, minm1, n_el);
             const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
             if (R.sel) R.sel[local] = (uint8_t)bsel;
             if (R.scale_e8m0) R.scale_e8m0[local] = (uint8_t)(sb >> 23);
@@ -505,7 +598,7 @@ mor_main_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ par
             if (R.block_stats) {
                 mor_block_stats_t bs;
                 bs.amax = b_amax;
-                bs.min_abs_nz = (tot.mn == 0xFFFFFFFFu) ? __uint_as_float(0x7F800000u) : __uint_as_float(tot.mn + 1u);
+                bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
                 bs.nnz = tot.nnz; bs.n_nonfinite = tot.nonfinite;
                 bs.sum_rel_e4m3 = (float)tot.s43; bs.sum_rel_e5m2 = (float)tot.s52;
                 R.block_stats[local] = bs;
@@ -592,7 +685,8 @@ mor_amax_kernel(const __grid_constant__ BatchParams p, float* __restrict__ amax_
             const uint16_t* src = R.x + s_off[seg] + 8 * k;
             uint16_t e[8] = {0, 0, 0, 0, 0, 0, 0, 0};
             for (int i = 0; i < left; ++i) e[i] = src[i];
-            v[j] = make_uint4(e[0] | (e[1] << 16), e[2] | (e[3] << 16), e[4] | (e[5] << 16), e[6] | (e[7] << 16));
+            v[j] = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
+                              e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
         }
     }
     __nv_bfloat162 m = __float2bfloat162_rn(0.0f);
@@ -622,7 +716,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p, float* __restrict__ amax_
     if (t == 0) {
         for (int i = 1; i < kThreads / 32; ++i) { amax = max(amax, s_wmax[i]); nf += s_wnf[i]; }
         // non-negative binary32 patterns order like the values
-        atomicMax(reinterpret_cast<unsigned int*>(const_cast<float*>(R.amax)), amax << 16);
+        atomicMax(reinterpret_cast<unsigned int*>(R.amax_slot), amax << 16);
         if (nf) atomicAdd(R.nonfinite_slot, nf);
     }
 }
@@ -642,7 +736,7 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
 
     WarpPart a;
-    a.s43 = a.s52 = 0.0; a.nnz = a.nonfinite = a.n4 = a.n5 = a.nb = 0u; a.mn = 0xFFFFFFFFu;
+    a.s43 = a.s52 = 0.0; a.nnz = a.nonfinite = a.n4 = a.n5 = a.nb = 0u; a.mn = 0xFFFFu;
     unsigned long long nnz64 = 0, nonf64 = 0, n4 = 0, n5 = 0, nb = 0;
     for (uint32_t i = t; i < R.n_tiles; i += kThreads) {
         const Partial P = partials[R.tile_begin + i];
@@ -690,14 +784,15 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
             c[2] = (n_blocks && bsel == MOR_FMT_E4M3); c[3] = 0; c[4] = (n_blocks && bsel == MOR_FMT_BF16);
             if (n_blocks && blockIdx.y == 0) {
                 uint32_t s4b, s5b;
-                block_scale(g_amax, m_g, R.scale_mode, s4b, s5b);
+                const float b_amax = *R.amax_slot;
+                block_scale(b_amax, m_g, R.scale_mode, s4b, s5b);
                 if (R.sel) R.sel[0] = (uint8_t)bsel;
                 if (R.scale_e8m0) R.scale_e8m0[0] = (uint8_t)(s4b >> 23);
                 if (R.scale_f32) R.scale_f32[0] = __uint_as_float(s4b);
                 if (R.block_stats) {
                     mor_block_stats_t bs;
-                    bs.amax = g_amax;
-                    bs.min_abs_nz = (tot.mn == 0xFFFFFFFFu) ? __uint_as_float(0x7F800000u) : __uint_as_float(tot.mn + 1u);
+                    bs.amax = b_amax;
+                    bs.min_abs_nz = minnz_value(tot.mn);
                     bs.nnz = (uint32_t)(c[0] > 0xFFFFFFFFull ? 0xFFFFFFFFull : c[0]);
                     bs.n_nonfinite = (uint32_t)(c[1] > 0xFFFFFFFFull ? 0xFFFFFFFFull : c[1]);
                     bs.sum_rel_e4m3 = (float)tot.s43; bs.sum_rel_e5m2 = (float)tot.s52;

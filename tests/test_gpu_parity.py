@@ -180,7 +180,7 @@ def test_select_stats_matches_analyze_quantize():
 def test_bf16_fallback_copies_only_rejected_blocks():
     import torch
 
-    g = wl.gradient_like(300, 1000, seed=54)
+    g = np.concatenate([wl.gradient_like(150, 1000, seed=54), wl.weight_like(150, 1000, seed=57)])
     host = np.zeros((300, 1008), dtype=np.uint16); host[:, :1000] = g
     x = parity.to_device(host)
     for block in [(1, 128), (128, 128)]:
