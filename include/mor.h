@@ -35,7 +35,9 @@ typedef enum {
     MOR_ERR_ALIGNMENT = 3,     /* base pointer or leading dimension not aligned as stated     */
     MOR_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than mor_workspace_bytes()        */
     MOR_ERR_CUDA = 5,          /* a CUDA runtime call failed (launch, copy)                   */
-    MOR_ERR_TIMEOUT = 6        /* reserved: a bounded device-side wait expired                */
+    MOR_ERR_TIMEOUT = 6,       /* reserved: a bounded device-side wait expired                */
+    MOR_ERR_STATIC_SCRATCH = 7 /* mor_analyze_quantize_static: the tensor needs more scratch than
+                                  the built-in array holds                                    */
 } mor_status_t;
 
 /* Representation types (Section 3: ordered "from most aggressive (e.g. E4M3) to least
@@ -204,6 +206,25 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
 size_t mor_host_staging_bytes(const mor_tensor_desc_t* host_desc);
 mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                        void* device_staging, size_t staging_bytes, void* cuda_stream);
+
+/* No counterpart in the paper: a packaging variant of mor_analyze_quantize for callers that cannot
+ * allocate device memory where they run (a plug-in inside a runtime that owns all device memory, a
+ * latency-critical loop that must avoid the synchronisation an allocation implies, a process with a
+ * memory budget fixed at start-up).  Inputs and outputs are the caller's as before; the scratch
+ * comes from an array of MOR_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU
+ * that loads the library holds that much memory until the process exits.  The call makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Limit: mor_workspace_bytes(host_desc, 1) must not exceed MOR_STATIC_SCRATCH_BYTES (512 KiB:
+ *     about 13,000 tiles of 128 x 128 elements, i.e. tensors up to roughly 214 M elements);
+ *     larger tensors are refused with MOR_ERR_STATIC_SCRATCH and nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array, and it keeps what the previous call left in it; the call
+ *     clears the part that has to start at zero.  Two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them.  */
+#define MOR_STATIC_SCRATCH_BYTES (512 * 1024)
+mor_status_t mor_analyze_quantize_static(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+                                         void* cuda_stream);
 
 const char* mor_status_string(mor_status_t status);
 int mor_version(void);

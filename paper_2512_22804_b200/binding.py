@@ -26,7 +26,8 @@ LIB_PATH = os.path.join(_HERE, "libmor_b200.so")
 
 MOR_OK = 0
 (MOR_ERR_INVALID_ARG, MOR_ERR_UNSUPPORTED, MOR_ERR_ALIGNMENT, MOR_ERR_WORKSPACE, MOR_ERR_CUDA,
- MOR_ERR_TIMEOUT) = range(1, 7)
+ MOR_ERR_TIMEOUT, MOR_ERR_STATIC_SCRATCH) = range(1, 8)
+MOR_STATIC_SCRATCH_BYTES = 512 * 1024
 MOR_FMT_E4M3, MOR_FMT_E5M2, MOR_FMT_BF16 = 0, 1, 2
 MOR_SCALE_GAM, MOR_SCALE_E8M0, MOR_SCALE_FP32_AMAX = 0, 1, 2
 MOR_CRIT_TENSOR_MEAN_REL, MOR_CRIT_BLOCK_VS_E5M2, MOR_CRIT_BLOCK_MEAN_REL = 0, 1, 2
@@ -109,6 +110,8 @@ def load():
         L.mor_host_staging_bytes.argtypes = [pd]
         L.mor_analyze_quantize_host.restype = C.c_int
         L.mor_analyze_quantize_host.argtypes = [pd, po, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.mor_analyze_quantize_static.restype = C.c_int
+        L.mor_analyze_quantize_static.argtypes = [pd, po, C.c_void_p]
         L.mor_status_string.restype = C.c_char_p
         L.mor_status_string.argtypes = [C.c_int]
         L.mor_version.restype = C.c_int
@@ -119,8 +122,8 @@ def load():
 
 EXPORTS = ["mor_workspace_bytes", "mor_analyze_quantize", "mor_analyze_quantize_batched",
            "mor_analyze_quantize_batched_ex", "mor_select_stats",
-           "mor_group_amax", "mor_host_staging_bytes", "mor_analyze_quantize_host", "mor_status_string",
-           "mor_version"]
+           "mor_group_amax", "mor_host_staging_bytes", "mor_analyze_quantize_host",
+           "mor_analyze_quantize_static", "mor_status_string", "mor_version"]
 
 
 # ------------------------------------------------------------------ C entry points ----
@@ -182,6 +185,12 @@ def mor_host_staging_bytes(desc: mor_tensor_desc_t) -> int:
 def mor_analyze_quantize_host(desc: mor_tensor_desc_t, out: mor_outputs_t, staging_ptr: int, staging_bytes: int,
                               stream_ptr: int = 0) -> int:
     return load().mor_analyze_quantize_host(C.byref(desc), C.byref(out), staging_ptr, staging_bytes, stream_ptr)
+
+
+def mor_analyze_quantize_static(desc: mor_tensor_desc_t, out: mor_outputs_t, stream_ptr: int = 0) -> int:
+    """mor_analyze_quantize with the library's built-in scratch array: no workspace to pass, no
+    device allocation made; tensors that need more than MOR_STATIC_SCRATCH_BYTES are refused."""
+    return load().mor_analyze_quantize_static(C.byref(desc), C.byref(out), stream_ptr)
 
 
 # ------------------------------------------------------------------------- helpers ----

@@ -440,6 +440,7 @@ const char* mor_status_string(mor_status_t status)
         case MOR_ERR_WORKSPACE: return "workspace missing or too small";
         case MOR_ERR_CUDA: return "CUDA runtime error";
         case MOR_ERR_TIMEOUT: return "device-side wait expired";
+        case MOR_ERR_STATIC_SCRATCH: return "tensor needs more scratch than the built-in array holds";
     }
     return "unknown status";
 }

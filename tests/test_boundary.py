@@ -33,8 +33,8 @@ def test_every_declared_entry_point_is_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert mb.mor_version() >= 100
-    seen = {mb.mor_status_string(s) for s in range(0, 7)}
-    assert len(seen) == 7 and "ok" in seen
+    seen = {mb.mor_status_string(s) for s in range(0, 8)}
+    assert len(seen) == 8 and "ok" in seen
 
 
 def desc(rows=256, cols=256, ld=None, block=(128, 128), formats=(0, 2), crit=mb.MOR_CRIT_BLOCK_VS_E5M2, x=0x1000):
