@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmor_b200.so")
-SOURCES = ["mor_api.cu", "mor_kernels.cu", "mor_static.cu"]
+SOURCES = ["mor_api.cu", "mor_kernels.cu", "mor_main.cu", "mor_static.cu"]
 
 
 def nvcc_path() -> str:

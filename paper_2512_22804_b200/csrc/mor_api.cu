@@ -35,13 +35,12 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     s.nbc = (uint32_t)nbc;
     s.nbr = (uint32_t)nbr;
     s.amax_tiles = (uint32_t)((segs + kSegsPerTile - 1) / kSegsPerTile);
+    s.n_tiles = (uint32_t)(nbr * nbc);       // the main kernel works on 128 x 128 tiles whatever the partition
     if (s.kind == KIND_BLK128) {
-        s.n_units = (uint32_t)(nbr * nbc);
-        s.n_tiles = s.n_units;
+        s.n_units = s.n_tiles;
         s.n_blocks = s.n_units;
     } else {
         s.n_units = (uint32_t)segs;
-        s.n_tiles = s.amax_tiles;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
     return MOR_OK;
@@ -93,8 +92,53 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
     return MOR_OK;
 }
 
+// ---- TMA descriptors (cuTensorMapEncodeTiled, reached through the runtime so that the library
+// does not link against the driver library)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// One descriptor for the BF16 input [rows, cols] with row pitch ld (box 128 x 128 elements; elements
+// past the edge read as zero) and one for the codes [rows, cols] bytes with row pitch codes_ld (box
+// 128 x 128 bytes; the part of a box past the edge is not written).
+bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store, CUtensorMap& in_map, CUtensorMap& out_map)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)d.cols, (cuuint64_t)d.rows};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileCols, (cuuint32_t)kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    const cuuint64_t in_stride[1] = {(cuuint64_t)d.ld * 2};
+    if (enc(&in_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.x), dims, in_stride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    if (store) {
+        const cuuint64_t out_stride[1] = {(cuuint64_t)o.codes_ld};
+        if (enc(&out_map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, o.codes, dims, out_stride, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    return true;
+}
+
 struct Layout {
-    size_t amax_off, nonf_off, partial_off, total;
+    size_t amax_off, nonf_off, status_off, partial_off, total;
 };
 
 Layout layout_of(int n, uint64_t tiles)
@@ -102,7 +146,8 @@ Layout layout_of(int n, uint64_t tiles)
     Layout l;
     l.amax_off = 0;
     l.nonf_off = (size_t)n * sizeof(float);
-    l.partial_off = round_up(2 * (size_t)n * sizeof(float), kAlign);
+    l.status_off = 2 * (size_t)n * sizeof(float);
+    l.partial_off = round_up(l.status_off + sizeof(uint32_t), kAlign);
     l.total = l.partial_off + round_up((size_t)tiles * sizeof(Partial), kAlign);
     return l;
 }
@@ -130,6 +175,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
+    r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.tile_begin = it.tile_begin;
@@ -192,15 +238,18 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     std::vector<Chunk> chunks;
     if (ev && !record(ev->main_begin)) return MOR_ERR_CUDA;
     std::vector<char> done(n, 0);
+    MainParams mp;
+    mp.device_status = reinterpret_cast<uint32_t*>(ws + l.status_off);
     for (int i = 0; i < n; ++i) {
         if (done[i]) continue;
         const MainVariant v = items[i].v;
-        BatchParams bp;
+        BatchParams& bp = mp.b;
         bp.n = 0;
         uint32_t t_end = 0;
         auto flush = [&]() -> bool {
             if (bp.n == 0) return true;
-            const bool ok = launch_main(v, bp, partials, t_end, stream) == cudaSuccess;
+            mp.total_tiles = t_end;
+            const bool ok = launch_main(v, mp, partials, stream) == cudaSuccess;
             chunks.push_back(Chunk{bp, v.kind});
             bp.n = 0; t_end = 0;
             return ok;
@@ -208,9 +257,16 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         for (int j = i; j < n; ++j) {
             if (done[j] || !same_variant(items[j].v, v)) continue;
             done[j] = 1;
-            fill_rec(items[j], ws, l, bp.t[bp.n]);
-            t_end += items[j].s.n_tiles;
-            bp.tile_end[bp.n++] = t_end;
+            if (items[j].s.n_tiles == 0) {
+                // an empty tensor has no tiles; its summary is still written by the finalise kernel
+                fill_rec(items[j], ws, l, bp.t[bp.n]);
+                bp.tile_end[bp.n++] = t_end;
+            } else {
+                fill_rec(items[j], ws, l, bp.t[bp.n]);
+                if (!encode_maps(*items[j].d, items[j].o, v.store, mp.in_map[bp.n], mp.out_map[bp.n])) return MOR_ERR_CUDA;
+                t_end += items[j].s.n_tiles;
+                bp.tile_end[bp.n++] = t_end;
+            }
             if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
         }
         if (!flush()) return MOR_ERR_CUDA;

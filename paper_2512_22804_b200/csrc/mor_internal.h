@@ -1,7 +1,9 @@
 // Internal contract between the host entry points (mor_api.cu) and the kernels
-// (mor_kernels.cu).  Not part of the C boundary.
+// (mor_kernels.cu: amax pre-pass and finalise; mor_main.cu: the fused main kernel).
+// Not part of the C boundary.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -9,14 +11,18 @@
 
 namespace mor {
 
-// A tile is 128 segments of 128 contiguous BF16 elements (32 KiB), handled by one CTA of
-// 256 threads, two threads per segment.  What a segment is depends on the partition:
-//   KIND_TENSOR / KIND_ROW128  consecutive 128-element pieces of the rows, row-major
-//   KIND_BLK128                the 128 rows of one 128x128 block
+// The main kernel works on tiles of 128 rows x 128 columns (32 KiB of BF16), whatever the
+// partition: a tile is one 128x128 block, or 128 one-row blocks of 128 elements, or a piece of
+// the single block of the per-tensor partition.  Tiles are numbered row-major over the tile
+// grid [ceil(rows/128), ceil(cols/128)].  The amax pre-pass has its own tiling: 128
+// consecutive 128-element row pieces per CTA.
+constexpr int kTileRows = 128;
+constexpr int kTileCols = 128;
 constexpr int kSegsPerTile = 128;
 constexpr int kSegElems = 128;
-constexpr int kThreads = 256;
-constexpr int kMaxBatch = 20;   // tensors per launch; the records travel as kernel parameters
+constexpr int kThreads = 256;          // amax and finalise kernels; compute threads of the main kernel
+constexpr int kMainThreads = 320;      // 8 compute warps + load warp + store warp
+constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor maps travel as kernel parameters
 
 enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2 };
 
@@ -25,7 +31,7 @@ struct Partial {
     double   sum43, sum52;        // relative-error sums of the tile (E4M3, E5M2)
     uint32_t nnz, nonfinite;
     uint32_t n_e4m3, n_e5m2, n_bf16;
-    uint32_t min_nz_bits;         // min |x| over non-zeros as BF16 bits, 0xFFFF if none (three-way only)
+    uint32_t min_nz_bits;         // min |x| over non-zeros as BF16 bits minus one, 0xFFFF if none
 };
 static_assert(sizeof(Partial) == 40, "Partial layout");
 
@@ -41,10 +47,11 @@ struct TensorRec {
     const float* amax;            // group amax on the device (workspace slot or the caller's)
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
+    const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     int64_t rows, cols, ld, codes_ld;
-    uint32_t nbc;                 // segments per row = ceil(cols / 128)
-    uint32_t nbr;                 // KIND_BLK128: block rows = ceil(rows / 128)
-    uint32_t n_units;             // KIND_BLK128: blocks; otherwise segments = rows * nbc
+    uint32_t nbc;                 // tile columns = ceil(cols / 128)
+    uint32_t nbr;                 // tile rows = ceil(rows / 128)
+    uint32_t n_units;             // blocks of the partition (KIND_TENSOR: row pieces, used by the pre-pass)
     uint32_t n_tiles;
     uint32_t tile_begin;          // index of the tensor's first Partial
     int32_t criterion, scale_mode, n_formats;
@@ -58,6 +65,16 @@ struct BatchParams {
     TensorRec t[kMaxBatch];
 };
 
+// Parameters of the main kernel: the records plus one TMA descriptor per tensor for the BF16
+// input (box 128 x 128 elements) and one for the code output (box 128 x 128 bytes).
+struct alignas(64) MainParams {
+    CUtensorMap in_map[kMaxBatch];
+    CUtensorMap out_map[kMaxBatch];
+    BatchParams b;
+    uint32_t total_tiles;
+    uint32_t* device_status;
+};
+
 struct MainVariant {
     int kind;        // Kind
     bool yard;       // evaluate E5M2 as well (Eq. 3, or statistics asked for)
@@ -66,9 +83,7 @@ struct MainVariant {
 };
 
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
-cudaError_t launch_main(const MainVariant& v, const BatchParams& p, Partial* partials,
-                        uint32_t total_tiles, cudaStream_t s);
+cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s);
-cudaError_t launch_copy_amax(const BatchParams& p, float* out, cudaStream_t s);
 
 }  // namespace mor

@@ -1,0 +1,904 @@
+// The fused main kernel of the MoR analyse-and-quantise pass for sm_100a.
+//
+// Per 128 x 128 tile: block amax and GAM scale (Algorithm 1), cast to E4M3 and E5M2,
+// relative-error sums (Eq. 1-3), range statistics (Eq. 4), per-block decision (Algorithm 2),
+// codes, scale bytes, selection bytes and a per-tile partial for the tensor-wide aggregate.
+//
+// Structure: persistent CTAs (two per SM), ten warps each.
+//   load warp      one thread walks the CTA's tiles and brings each one in with a TMA tile load
+//                  (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) into a two-stage
+//                  ring of 32 KiB buffers, signalling an mbarrier per stage;
+//   compute warps  8 warps, two threads per tile row.  A thread copies its 64 elements from the
+//                  stage to registers (the stage is handed back to the load warp at once), scans
+//                  them for amax / smallest non-zero, derives the scale, converts and accumulates
+//                  the error terms from the registers, and writes its codes to a 16 KiB staging
+//                  buffer;
+//   store warp     waits for the staging buffer, issues the TMA tile store of the codes (clipped
+//                  at the tensor's edge by the hardware), adds up the threads' sums in a fixed
+//                  order, and writes the tile's partial and, for 128x128 blocks, the block's
+//                  decision and metadata.
+// Every wait on an mbarrier is bounded; a wait that runs out sets a status word that the
+// finalise kernel copies into mor_tensor_stats_t.status, and the CTA winds down.
+//
+// Arithmetic that must be exact: amax (integer compare of BF16 bit patterns), the scale (IEEE
+// binary32 division, looked up by the 7 mantissa bits of the BF16 amax from a table that each
+// CTA fills with that same division), the scaled value (one IEEE binary32 multiply) and the FP8
+// codes (cvt.rn.satfinite).  The error ratio uses an approximate reciprocal; it only feeds
+// sums that are compared with a tolerance.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <float.h>
+
+#include "mor_internal.h"
+
+namespace mor {
+namespace {
+
+constexpr int kStages = 2;
+constexpr int kInBytes = kTileRows * kTileCols * 2;      // 32768
+constexpr int kOutBytes = kTileRows * kTileCols;         // 16384
+constexpr int kComputeWarps = kThreads / 32;             // 8
+constexpr int kLoadWarp = kComputeWarps;                 // warp 8
+constexpr int kStoreWarp = kComputeWarps + 1;            // warp 9
+constexpr uint32_t kBf16Inf = 0x7F80u;
+constexpr uint32_t kSpinLimit = 1u << 17;                // x 20 us suspend hint: a few seconds at most
+constexpr uint32_t kSelNone = 3u;                        // entry of a tile row outside the tensor
+
+// What the load warp tells the other warps about the tile in a stage.
+struct TileMeta {
+    int32_t ti;            // tensor index within the launch, -1 = no more tiles
+    uint32_t local;        // tile index within the tensor
+    int32_t row0, col0;    // first row / column of the tile
+    int32_t vrows, vcols;  // rows / columns of the tile inside the tensor (1..128)
+    uint32_t blk_base;     // ROW128: index of the block of the tile's first row
+    uint32_t pad;
+};
+
+// What a compute thread hands to the store warp: its (ROW128: its block's) sums and counts.
+struct __align__(16) Entry {
+    float e43, e52;
+    uint32_t nnz_nonf;     // non-zeros | non-finites << 16
+    uint32_t sel_min;      // selection (kSelNone: not a block) | (smallest non-zero bits - 1) << 16
+};
+
+struct Control {
+    unsigned long long full[kStages], empty[kStages];   // input ring
+    unsigned long long out_full[2], out_empty[2];       // code staging + entries
+    unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
+    unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
+    TileMeta meta[kStages];
+    Entry entry[2][kThreads];
+    uint32_t wmax[2][2][kComputeWarps];                  // BLK128: per tile parity, per pass: warp amax | inverted min
+    uint32_t tile_scale[2][2];                           // BLK128: scale bits (E4M3, E5M2) of the tile
+    uint32_t tile_key[2];                                // BLK128: amax bits << 16 | 0xFFFF - (min - 1)
+    uint32_t dec_sel[2];
+    uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
+    volatile uint32_t abort;
+};
+
+constexpr int kSmemBytes = 1024 + kStages * kInBytes + 2 * kOutBytes + (int)sizeof(Control);
+
+// ------------------------------------------------------------------ PTX helpers ----
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity; false when the limit ran out or (with a flag
+// given) another thread of the CTA has given up already.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, const volatile uint32_t* abort_flag)
+{
+    const uint32_t a = smem_addr(bar);
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        uint32_t done;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(done) : "r"(a), "r"(parity), "r"(20000u) : "memory");
+        if (done) return true;
+        if (abort_flag != nullptr && *abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, void* bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, int x, int y, const void* src)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(smem_addr(src)) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// barrier over the compute threads that also ORs a predicate
+__device__ __forceinline__ bool compute_bar_or(bool v)
+{
+    uint32_t r;
+    asm volatile("{ .reg .pred p, q; setp.ne.u32 p, %1, 0; barrier.cta.red.or.pred q, 1, %2, p; selp.u32 %0, 1, 0, q; }"
+                 : "=r"(r) : "r"((uint32_t)v), "n"(kThreads) : "memory");
+    return r != 0;
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts64(uint32_t a, uint2 v)
+{
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
+}
+
+// {hi, lo} -> two FP8 codes, `lo` in the low byte (round to nearest even, saturate to the largest finite)
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t cvt_e5m2x2(float hi, float lo)
+{
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// two FP8 codes -> f16x2 (exact: every E4M3 and E5M2 value is a binary16 number)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t c)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(static_cast<uint16_t>(c)));
+    return r;
+}
+__device__ __forceinline__ uint32_t e5m2x2_to_f16x2(uint32_t c)
+{
+    uint32_t r;
+    asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(r) : "h"(static_cast<uint16_t>(c)));
+    return r;
+}
+// (q.lo - ylo, q.hi - yhi) with q binary16 and y binary32, each one binary32 operation; exact
+// here because q is the FP8 neighbour of y
+__device__ __forceinline__ void diff_f16x2_f32(uint32_t q, float ylo, float yhi, float& dlo, float& dhi)
+{
+    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; sub.f32.f16 %0, l, %3; sub.f32.f16 %1, h, %4; }"
+        : "=f"(dlo), "=f"(dhi) : "r"(q), "f"(ylo), "f"(yhi));
+}
+__device__ __forceinline__ float rcp_ftz(float a)
+{
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+__device__ __forceinline__ float rcp_approx(float a)
+{
+    float r;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
+{
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// two IEEE binary32 multiplies / fused multiply-adds in one instruction (each lane rounds to nearest even)
+__device__ __forceinline__ unsigned long long mul_f32x2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
+{
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+// ------------------------------------------------------------------ Algorithm 1 ----
+
+// "ideal FP32 scaling factor" 448 / amax by one IEEE division; a quotient above the largest
+// finite binary32 is replaced by it
+__device__ __forceinline__ uint32_t ideal_scale_bits_div(float amax)
+{
+    return __float_as_uint(fminf(__fdiv_rn(448.0f, amax), FLT_MAX));
+}
+
+// The same for an amax that is a finite non-zero BF16 value, given as its 15 magnitude bits:
+// 448 / (2^e * (1 + m/128)) = (448 / (1 + m/128)) * 2^-e, and scaling by a power of two is exact
+// as long as the result stays a normal binary32 (it always does at the small end; at the large end,
+// and for subnormal amax, the exponent test finds the overflow).
+__device__ __forceinline__ uint32_t ideal_scale_bits_tab(uint32_t a, const uint32_t* rtab)
+{
+    const int32_t e = (int32_t)(a >> 7);
+    const uint32_t t = rtab[a & 127u];
+    const int32_t ef = (int32_t)(t >> 23) + 127 - e;
+    return ef > 254 ? 0x7F7FFFFFu : t + (uint32_t)((127 - e) * (1 << 23));
+}
+
+// Algorithm 1, group part: mantissa of 448 / g_amax (0 for an all-zero tensor, and for the
+// scale modes that have no shared mantissa)
+__device__ __forceinline__ uint32_t group_mantissa(float g_amax, int scale_mode)
+{
+    if (scale_mode != MOR_SCALE_GAM || !(g_amax > 0.0f)) return 0u;
+    return ideal_scale_bits_div(g_amax) & 0x7FFFFFu;
+}
+
+// Algorithm 1, block part: exponent of 448 / b_amax, lowered by one when the group mantissa
+// exceeds the block's; the scale is the shared mantissa joined to that exponent.  The E5M2
+// scale is 7 binades higher (57344 = 448 * 2^7), capped at exponent field 254.
+__device__ __forceinline__ void block_scale(uint32_t amax_bits, uint32_t m_g, int scale_mode, const uint32_t* rtab,
+                                            uint32_t& s4_bits, uint32_t& s5_bits)
+{
+    uint32_t e = 127u, m = (scale_mode == MOR_SCALE_FP32_AMAX) ? 0u : m_g;
+    if (amax_bits != 0u) {
+        const uint32_t sb = ideal_scale_bits_tab(amax_bits, rtab);
+        const uint32_t m_b = sb & 0x7FFFFFu;
+        e = sb >> 23;
+        if (scale_mode == MOR_SCALE_FP32_AMAX) m = m_b;
+        else if (m_g > m_b) e -= 1u;
+    }
+    const uint32_t e5 = min(e + 7u, 254u);
+    s4_bits = (e << 23) | m;
+    s5_bits = (e5 << 23) | m;
+}
+
+__device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
+{
+    return minm1_bits == 0xFFFFu ? __uint_as_float(0x7F800000u) : __uint_as_float((minm1_bits + 1u) << 16);
+}
+
+// ------------------------------------------------------------------ scan ----
+
+// Block statistics of a thread's 64 elements in one pass over packed BF16 pairs, returned as
+// one word: amax bits << 16 | 0xFFFF - (smallest non-zero bits - 1), so that both combine with
+// a packed 16-bit maximum.
+//   amax  per-halfword max of the |x| bit patterns.  NaN and inf compare above every finite
+//         pattern, which is how a non-finite input is noticed.
+//   min   per-halfword min of (|x| bits - 1) mod 2^16: zeros wrap to 0xFFFF and drop out.
+__device__ __forceinline__ uint32_t scan_words(const uint32_t (&w)[32])
+{
+    uint32_t mx = 0u, mn = 0xFFFFFFFFu;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const uint32_t a0 = w[i] & 0x7FFF7FFFu, a1 = w[i + 1] & 0x7FFF7FFFu;
+        mx = __vimax3_u16x2(mx, a0, a1);
+        mn = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn);
+        mn = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn);
+    }
+    const uint32_t amax = max(mx & 0xFFFFu, mx >> 16), minm1 = min(mn & 0xFFFFu, mn >> 16);
+    return (amax << 16) | (0xFFFFu - minm1);
+}
+
+// the same over finite elements only (used once a non-finite element has been seen)
+__device__ __noinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
+{
+    uint32_t m = 0u, n = 0xFFFFu;
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i) {
+        const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
+        if (lo < kBf16Inf) { m = max(m, lo); n = min(n, (lo - 1u) & 0xFFFFu); }
+        if (hi < kBf16Inf) { m = max(m, hi); n = min(n, (hi - 1u) & 0xFFFFu); }
+    }
+    return (m << 16) | (0xFFFFu - n);
+}
+
+__device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
+
+// ------------------------------------------------------------------ conversion ----
+
+// Fast path for one BF16 pair: two E4M3 codes (and two E5M2 codes) with their terms of
+// Eq. 1-3.   y = fl32(x * scale); c = RNE-saturating cast; q = value of c;
+// term = |y - q| / |y|, formed as |y - q| * |rcp(y + 2^-126)| (the sum inside a fused
+// multiply-add).  The caller guarantees that the block holds no NaN/inf and that every non-zero
+// |y| is at least 2^-100, so the added constant changes a term by less than 2^-26 relative, and a
+// zero element gives 0 * 2^126.  The same reciprocal counts the non-zeros: y * rcp is 1 for a
+// non-zero element (within 2^-22) and 0 for a zero.
+template <bool YARD>
+__device__ __forceinline__ void convert_pair_fast(uint32_t w, unsigned long long s4x2, unsigned long long s5x2,
+                                                  unsigned long long tiny2, float& a43, float& a52,
+                                                  unsigned long long& cnt2, uint32_t& c4, uint32_t& c5)
+{
+    const unsigned long long x2 = pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    const unsigned long long y2 = mul_f32x2(x2, s4x2);
+    float ylo, yhi, ulo, uhi;
+    unpack_f32x2(y2, ylo, yhi);
+    unpack_f32x2(fma_f32x2(x2, s4x2, tiny2), ulo, uhi);
+    const float rlo = rcp_ftz(ulo), rhi = rcp_ftz(uhi);
+    cnt2 = fma_f32x2(y2, pack_f32x2(rlo, rhi), cnt2);
+    c4 = cvt_e4m3x2(yhi, ylo);
+    float dlo, dhi;
+    diff_f16x2_f32(e4m3x2_to_f16x2(c4), ylo, yhi, dlo, dhi);
+    a43 = fmaf(fabsf(dlo), fabsf(rlo), a43);
+    a43 = fmaf(fabsf(dhi), fabsf(rhi), a43);
+    if (YARD) {
+        float zlo, zhi, elo, ehi;
+        unpack_f32x2(mul_f32x2(x2, s5x2), zlo, zhi);
+        c5 = cvt_e5m2x2(zhi, zlo);
+        diff_f16x2_f32(e5m2x2_to_f16x2(c5), zlo, zhi, elo, ehi);
+        // |z - q'| / |z| = |z - q'| * (1/|y|) * (scale4/scale5); the power-of-two ratio is applied once per block
+        a52 = fmaf(fabsf(elo), fabsf(rlo), a52);
+        a52 = fmaf(fabsf(ehi), fabsf(rhi), a52);
+    } else {
+        c5 = 0;
+    }
+}
+
+struct CarefulAcc {
+    float a43, a52;
+    uint32_t nnz, nbig, nonfinite;
+};
+
+// Careful path for one BF16 pair: handles NaN/inf elements (stated reading: ignored by
+// every count and sum, NaN -> 0x7F, +-inf -> +-largest finite) and non-zero elements whose
+// scaled value leaves binary32's normal range (flushed by both formats: term 1, added by
+// the caller from the counts nnz - nbig).
+template <bool YARD>
+__device__ __forceinline__ void convert_pair_careful(uint32_t w, float s4, float s5, CarefulAcc& A, uint32_t& c4, uint32_t& c5)
+{
+    const uint32_t blo = w << 16, bhi = w & 0xFFFF0000u;
+    const uint32_t alo = blo & 0x7FFFFFFFu, ahi = bhi & 0x7FFFFFFFu;
+    const float xlo = __uint_as_float(blo), xhi = __uint_as_float(bhi);
+    const bool uselo = alo < 0x7F800000u, usehi = ahi < 0x7F800000u;
+    A.nonfinite += (uselo ? 0u : 1u) + (usehi ? 0u : 1u);
+    A.nnz += ((alo != 0u && uselo) ? 1u : 0u) + ((ahi != 0u && usehi) ? 1u : 0u);
+
+    const float ylo = __fmul_rn(xlo, s4), yhi = __fmul_rn(xhi, s4);
+    c4 = cvt_e4m3x2(yhi, ylo);
+    float dlo, dhi;
+    diff_f16x2_f32(e4m3x2_to_f16x2(c4), ylo, yhi, dlo, dhi);
+    const float aylo = fabsf(ylo), ayhi = fabsf(yhi);
+    const bool biglo = (aylo >= FLT_MIN) && uselo, bighi = (ayhi >= FLT_MIN) && usehi;
+    const float rlo = rcp_approx(aylo), rhi = rcp_approx(ayhi);
+    if (biglo) { A.a43 = fmaf(fabsf(dlo), rlo, A.a43); A.nbig++; }
+    if (bighi) { A.a43 = fmaf(fabsf(dhi), rhi, A.a43); A.nbig++; }
+
+    if (YARD) {
+        const float zlo = __fmul_rn(xlo, s5), zhi = __fmul_rn(xhi, s5);
+        c5 = cvt_e5m2x2(zhi, zlo);
+        float elo, ehi;
+        diff_f16x2_f32(e5m2x2_to_f16x2(c5), zlo, zhi, elo, ehi);
+        if (biglo) A.a52 = fmaf(fabsf(elo), rlo, A.a52);
+        if (bighi) A.a52 = fmaf(fabsf(ehi), rhi, A.a52);
+    } else {
+        c5 = 0;
+    }
+    if (!uselo) {
+        const bool nan = (alo & 0x007F0000u) != 0u;
+        const uint32_t sg = (blo >> 24) & 0x80u;
+        c4 = (c4 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Eu));
+        c5 = (c5 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Bu));
+    }
+    if (!usehi) {
+        const bool nan = (ahi & 0x007F0000u) != 0u;
+        const uint32_t sg = (bhi >> 24) & 0x80u;
+        c4 = (c4 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Eu)) << 8);
+        c5 = (c5 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Bu)) << 8);
+    }
+}
+
+// A thread's 64 elements, held as 8 chunks of 4 words; chunk j belongs at byte offset
+// (j ^ swz) * 8 of the thread's 64 code bytes.  E4M3 codes go to the staging buffer at once; with
+// three formats the E5M2 codes wait in registers for the block's decision.
+// Results: e43 = the thread's sum of E4M3 terms, complete; e52 = its sum of E5M2 terms, complete;
+// nnz; nonfinite.
+template <bool YARD, bool THREE, bool CAREFUL, bool STORE>
+__device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s4b, uint32_t s5b,
+                                              float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite, uint2 (&k5)[8])
+{
+    const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
+    float a43[4] = {0.0f, 0.0f, 0.0f, 0.0f}, a52[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    unsigned long long cnt2[2] = {0ull, 0ull};
+    CarefulAcc A;
+    A.a43 = A.a52 = 0.0f;
+    A.nnz = A.nbig = A.nonfinite = 0u;
+    const unsigned long long s4x2 = pack_f32x2(s4, s4), s5x2 = pack_f32x2(s5, s5), tiny2 = pack_f32x2(FLT_MIN, FLT_MIN);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (CAREFUL) convert_pair_careful<YARD>(w[4 * j + i], s4, s5, A, a[i], b[i]);
+            else convert_pair_fast<YARD>(w[4 * j + i], s4x2, s5x2, tiny2, a43[i], a52[i], cnt2[i & 1], a[i], b[i]);
+        }
+        if (STORE) sts64(out_addr ^ (j << 3), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
+        if (THREE) k5[j] = make_uint2(__byte_perm(b[0], b[1], 0x5410), __byte_perm(b[2], b[3], 0x5410));
+    }
+    // scale4 / scale5 = 2^(e4 - e5)
+    const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);
+    if (CAREFUL) {
+        const float tiny = (float)(A.nnz - A.nbig);
+        nnz = A.nnz;
+        nonfinite = A.nonfinite;
+        e43 = A.a43 + tiny;
+        e52 = YARD ? A.a52 * ratio + tiny : 0.0f;
+    } else {
+        float c0, c1, c2, c3;
+        unpack_f32x2(cnt2[0], c0, c1);
+        unpack_f32x2(cnt2[1], c2, c3);
+        nnz = (uint32_t)__float2int_rn((c0 + c1) + (c2 + c3));
+        nonfinite = 0u;
+        e43 = (a43[0] + a43[1]) + (a43[2] + a43[3]);
+        e52 = YARD ? ((a52[0] + a52[1]) + (a52[2] + a52[3])) * ratio : 0.0f;
+    }
+}
+
+// Algorithm 2 for one block with the per-block metrics (M_1 = Eq. 3, M_2 = Eq. 4, or
+// Eq. 1-2 on the block alone).
+__device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43, double e52, uint32_t nnz,
+                                                 uint32_t nonfinite, uint32_t amax_bits, uint32_t minm1_bits,
+                                                 uint32_t n_elems)
+{
+    if (nonfinite) return MOR_FMT_BF16;
+    if (R.criterion == MOR_CRIT_BLOCK_VS_E5M2) {
+        const bool ok = (R.flags & MOR_FLAG_STRICT_TIES) ? (e43 < e52) : (e43 <= e52);
+        if (ok) return MOR_FMT_E4M3;
+        if (R.n_formats == 3) {
+            // max|b| < (57344 * 2^14) * min|b|, exact in binary32 (11 significant bits)
+            float mnv = minnz_value(minm1_bits);
+            if ((R.flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) && nnz < n_elems) mnv = 0.0f;
+            const float amax = __uint_as_float(amax_bits << 16);
+            if (amax < 939524096.0f * mnv) return MOR_FMT_E5M2;
+        }
+        return MOR_FMT_BF16;
+    }
+    if (R.criterion == MOR_CRIT_BLOCK_MEAN_REL) {
+        const double err = nnz ? e43 / (double)nnz : 0.0;
+        return err < (double)R.threshold ? MOR_FMT_E4M3 : MOR_FMT_BF16;
+    }
+    return MOR_FMT_E4M3;   // tensor-level criterion: decided by the finalise kernel
+}
+
+// ------------------------------------------------------------------ tile bookkeeping ----
+
+struct TileId {
+    int ti;
+    uint32_t local;
+    int row0, col0, vrows, vcols;
+};
+
+__device__ __forceinline__ TileId locate_tile(const BatchParams& b, uint32_t tile)
+{
+    int ti = 0;
+    uint32_t begin = 0;
+#pragma unroll 1
+    while (ti < b.n - 1 && tile >= b.tile_end[ti]) { begin = b.tile_end[ti]; ++ti; }
+    const TensorRec& R = b.t[ti];
+    TileId t;
+    t.ti = ti;
+    t.local = tile - begin;
+    const uint32_t bi = t.local / R.nbc, bj = t.local - bi * R.nbc;
+    t.row0 = (int)(bi * kTileRows);
+    t.col0 = (int)(bj * kTileCols);
+    const long long rr = R.rows - t.row0, cc = R.cols - t.col0;
+    t.vrows = (int)(rr < kTileRows ? rr : kTileRows);
+    t.vcols = (int)(cc < kTileCols ? cc : kTileCols);
+    return t;
+}
+
+__device__ __forceinline__ void give_up(Control& C, uint32_t* device_status)
+{
+    C.abort = 1u;
+    atomicOr(device_status, 1u);
+}
+
+__device__ __forceinline__ double shfl_xor_f64(double v, int o) { return __shfl_xor_sync(0xFFFFFFFFu, v, o); }
+
+// ------------------------------------------------------------------ load warp ----
+
+__device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in)
+{
+    uint32_t issued = 0;
+    bool ok = true;
+#pragma unroll 1
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        if (tile >= p.total_tiles) break;
+        const uint32_t s = it % kStages, n = it / kStages;
+        if (n > 0 && !mbar_wait(&C.empty[s], (n - 1) & 1u, &C.abort)) { ok = false; break; }
+        const TileId t = locate_tile(p.b, tile);
+        TileMeta m;
+        m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
+        m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
+        m.pad = 0;
+        C.meta[s] = m;
+        mbar_arrive_expect_tx(&C.full[s], kInBytes);
+        tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
+        issued = it + 1;
+    }
+    if (!ok || C.abort) {
+        // the compute warps may have left: the copies still in flight must land before the CTA goes
+        if (!ok) give_up(C, p.device_status);
+        for (uint32_t k = 0; k < (uint32_t)kStages && k < issued; ++k) {
+            const uint32_t it = issued - 1 - k;
+            mbar_wait(&C.full[it % kStages], (it / kStages) & 1u, nullptr);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ store warp ----
+
+template <int KIND, bool THREE, bool STORE>
+__device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsigned char* out, Partial* __restrict__ partials,
+                                           int lane)
+{
+    constexpr int kEntries = (KIND == KIND_ROW128) ? kTileRows : kThreads;
+    bool stores_pending = false;
+#pragma unroll 1
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        if (tile >= p.total_tiles) break;
+        const uint32_t b = it & 1u, n = it >> 1;
+        const TileId t = locate_tile(p.b, tile);
+        const TensorRec& R = p.b.t[t.ti];
+        bool ok = mbar_wait(&C.out_full[b], n & 1u, &C.abort);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) { if (lane == 0) give_up(C, p.device_status); break; }
+
+        // the threads' sums in a fixed order: lane-strided, then a butterfly
+        double s43 = 0.0, s52 = 0.0;
+        uint32_t nnz = 0, nonf = 0, n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
+#pragma unroll
+        for (int k = 0; k < kEntries / 32; ++k) {
+            const Entry e = C.entry[b][lane + 32 * k];
+            s43 += (double)e.e43;
+            s52 += (double)e.e52;
+            nnz += e.nnz_nonf & 0xFFFFu;
+            nonf += e.nnz_nonf >> 16;
+            const uint32_t sel = e.sel_min & 0xFFFFu;
+            n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
+            mn = min(mn, e.sel_min >> 16);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
+        nnz = __reduce_add_sync(0xFFFFFFFFu, nnz);
+        nonf = __reduce_add_sync(0xFFFFFFFFu, nonf);
+        mn = __reduce_min_sync(0xFFFFFFFFu, mn);
+        if (KIND == KIND_ROW128) {
+            n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
+            n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
+            nb = __reduce_add_sync(0xFFFFFFFFu, nb);
+        } else {
+            n4 = n5 = nb = 0;
+        }
+
+        const bool need_dec = KIND == KIND_BLK128 && (THREE || R.fallback != nullptr);
+        if (lane == 0) {
+            if (KIND == KIND_BLK128) {
+                const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
+                const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
+                const uint32_t bsel = decide_block(R, s43, s52, nnz, nonf, amax_bits, minm1, (uint32_t)(t.vrows * t.vcols));
+                const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
+                if (R.sel) R.sel[t.local] = (uint8_t)bsel;
+                if (R.scale_e8m0) R.scale_e8m0[t.local] = (uint8_t)(sb >> 23);
+                if (R.scale_f32) R.scale_f32[t.local] = __uint_as_float(sb);
+                if (R.block_stats) {
+                    mor_block_stats_t bs;
+                    bs.amax = __uint_as_float(amax_bits << 16);
+                    bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                    bs.nnz = nnz; bs.n_nonfinite = nonf;
+                    bs.sum_rel_e4m3 = (float)s43; bs.sum_rel_e5m2 = (float)s52;
+                    R.block_stats[t.local] = bs;
+                }
+                n4 = bsel == MOR_FMT_E4M3; n5 = bsel == MOR_FMT_E5M2; nb = bsel == MOR_FMT_BF16;
+                if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }
+            }
+            Partial P;
+            P.sum43 = s43; P.sum52 = s52; P.nnz = nnz; P.nonfinite = nonf;
+            P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
+            partials[R.tile_begin + t.local] = P;
+        }
+        if (STORE) {
+            if (KIND == KIND_BLK128 && THREE) {
+                // the compute threads put the chosen format's codes in place after the decision
+                ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) { if (lane == 0) give_up(C, p.device_status); break; }
+            }
+            if (lane == 0) {
+                tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
+                bulk_commit();
+                stores_pending = true;
+                bulk_wait_read<0>();      // the staging buffer may be overwritten from here on
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&C.out_empty[b]);
+    }
+    if (lane == 0 && stores_pending) bulk_wait_all();
+}
+
+// ------------------------------------------------------------------ compute warps ----
+
+// copy of every block that stays in BF16, straight from the registers
+__device__ __forceinline__ void write_fallback(const TensorRec& R, const uint32_t (&w)[32], const TileMeta& m, int row, int h, int swz)
+{
+    if (row >= m.vrows) return;
+    uint16_t* dst_row = R.fallback + (long long)(m.row0 + row) * R.ld + m.col0 + h * 64;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = (j ^ swz) * 8;                      // first of the chunk's 8 elements within the thread's 64
+        const int left = m.vcols - (h * 64 + c);
+        if (left >= 8) {
+            *reinterpret_cast<uint4*>(dst_row + c) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i < left) dst_row[c + i] = (uint16_t)(w[4 * j + (i >> 1)] >> (16 * (i & 1)));
+        }
+    }
+}
+
+template <int KIND, bool YARD, bool THREE, bool STORE>
+__device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
+{
+    const int lane = tid & 31, warp = tid >> 5;
+    const int row = tid >> 1, h = tid & 1;
+    // Chunk order: thread (row, h) holds the 16-byte chunk c of its 128 bytes as chunk c ^ swz.  With
+    // this choice the 8 threads of a 128-bit load phase and the 16 threads of a 64-bit store phase
+    // touch distinct banks.
+    const int swz = (row & 7) ^ (h << 2);
+    const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
+    const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
+    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out);
+
+    int cur_ti = -1;
+    uint32_t m_g = 0;
+#pragma unroll 1
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        if (tile >= p.total_tiles) break;
+        const uint32_t s = it % kStages, b = it & 1u, n2 = it >> 1;
+
+        bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
+        const TileMeta m = C.meta[s];
+        uint32_t w[32];
+        {
+            const uint32_t a = in_base + s * kInBytes + in_off;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint4 v = lds128(a ^ (j << 4));
+                w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+            }
+        }
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (lane == 0) {
+            if (ok) mbar_arrive(&C.empty[s]);          // every lane's loads have returned: the stage is free
+            else give_up(C, p.device_status);
+        }
+        if (KIND != KIND_BLK128 && !ok) break;
+
+        const TensorRec& R = p.b.t[ok ? m.ti : 0];
+        if (m.ti != cur_ti && ok) {
+            cur_ti = m.ti;
+            m_g = group_mantissa(*R.amax, R.scale_mode);   // Algorithm 1, group part, once per tensor
+        }
+
+        // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
+        uint32_t key = scan_words(w);
+        bool nonfin;
+        if (KIND == KIND_ROW128) {
+            key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
+            nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
+            if (nonfin) {
+                key = scan_words_finite(w);
+                key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
+            }
+        } else if (KIND == KIND_BLK128) {
+#pragma unroll 1
+            for (int pass = 0; pass < 2; ++pass) {
+                const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, key >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, key & 0xFFFFu);
+                if (lane == 0) C.wmax[b][pass][warp] = (hi << 16) | lo;
+                if (compute_bar_or(!ok)) return;                                   // all compute threads leave together
+                const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]);
+                const uint4 k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
+                key = key_max(key_max(__vimax3_u16x2(k0.x, k0.y, k0.z), k0.w), key_max(__vimax3_u16x2(k1.x, k1.y, k1.z), k1.w));
+                nonfin = pass == 1 || (key >> 16) >= kBf16Inf;                     // CTA-uniform
+                if (pass == 1 || !nonfin) break;
+                key = scan_words_finite(w);
+            }
+        } else {
+            nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
+            if (nonfin) key = scan_words_finite(w);
+        }
+        uint32_t amax_bits = key >> 16;
+        const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
+        // per-tensor partition: the block is the tensor, its amax was reduced by the pre-pass
+        if (KIND == KIND_TENSOR) amax_bits = __float_as_uint(*R.amax_slot) >> 16;
+
+        uint32_t s4b, s5b;
+        block_scale(amax_bits, m_g, R.scale_mode, C.rtab, s4b, s5b);
+
+        // The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_pair_fast).
+        // minm1 covers this thread's block (ROW128), this tile (BLK128), this thread (TENSOR).
+        bool careful = nonfin;
+        if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
+        if (KIND != KIND_BLK128) careful = __any_sync(0xFFFFFFFFu, careful);
+
+        // ---- staging buffer and entries of tile it - 2 must have been consumed ----
+        if (n2 > 0) {
+            bool ok2 = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
+            ok2 = __all_sync(0xFFFFFFFFu, ok2);
+            if (!ok2) {
+                if (lane == 0) give_up(C, p.device_status);
+                if (KIND != KIND_BLK128) break;
+                ok = false;
+            }
+        }
+
+        // ---- cast and error terms ----
+        float e43, e52;
+        uint32_t nnz, nonf;
+        uint2 k5[8];
+        const uint32_t oa = out_base + b * kOutBytes + out_off;
+        if (careful) convert_words<YARD, THREE, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
+        else         convert_words<YARD, THREE, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
+
+        if (KIND == KIND_ROW128) {
+            // ---- block sums, decision, metadata ----
+            e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
+            e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
+            uint32_t nz = nnz | (nonf << 16);
+            nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
+            const bool valid = row < m.vrows;
+            const uint32_t sel = decide_block(R, (double)e43, (double)e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
+            if (THREE && STORE && sel == MOR_FMT_E5M2) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
+            }
+            if (h == 0) {
+                Entry e;
+                e.e43 = e43; e.e52 = e52; e.nnz_nonf = nz;
+                e.sel_min = (valid ? sel : kSelNone) | (minm1 << 16);
+                C.entry[b][row] = e;
+                if (valid) {
+                    const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
+                    const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
+                    if (R.sel) R.sel[blk] = (uint8_t)sel;
+                    if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
+                    if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
+                    if (R.block_stats) {
+                        mor_block_stats_t bs;
+                        bs.amax = __uint_as_float(amax_bits << 16);
+                        bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                        bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
+                        R.block_stats[blk] = bs;
+                    }
+                }
+            }
+            if (STORE && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+        } else {
+            Entry e;
+            e.e43 = e43; e.e52 = e52; e.nnz_nonf = nnz | (nonf << 16);
+            e.sel_min = kSelNone | (minm1 << 16);
+            C.entry[b][tid] = e;
+            if (KIND == KIND_BLK128 && tid == 0) {
+                C.tile_scale[b][0] = s4b; C.tile_scale[b][1] = s5b; C.tile_key[b] = key;
+            }
+        }
+        if (STORE) fence_async_smem();                  // the codes must be visible to the TMA store
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&C.out_full[b]);
+
+        if (KIND == KIND_BLK128) {
+            const bool need_dec = THREE || R.fallback != nullptr;
+            if (need_dec) {
+                bool ok3 = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
+                ok3 = __all_sync(0xFFFFFFFFu, ok3);
+                if (!ok3) { if (lane == 0) give_up(C, p.device_status); ok = false; }
+                const uint32_t sel = C.dec_sel[b];
+                if (THREE && STORE) {
+                    if (ok3 && sel == MOR_FMT_E5M2) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&C.codes_full[b]);
+                }
+                if (STORE && ok3 && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ kernel ----
+
+template <int KIND, bool YARD, bool THREE, bool STORE>
+__global__ void __launch_bounds__(kMainThreads, 2)
+mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ partials)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* base = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    unsigned char* in = base;
+    unsigned char* out = base + kStages * kInBytes;
+    Control& C = *reinterpret_cast<Control*>(out + 2 * kOutBytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], kComputeWarps); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&C.out_full[b], kComputeWarps); mbar_init(&C.out_empty[b], 1);
+            mbar_init(&C.dec_full[b], 1); mbar_init(&C.codes_full[b], kComputeWarps);
+        }
+        C.abort = 0u;
+        fence_mbar_init();
+    }
+    // fl32(448 / (1 + m/128)) for the 128 mantissas of a BF16 amax: the division of Algorithm 1,
+    // done here once per CTA with the IEEE divide and looked up per block afterwards
+    if (tid < 128) C.rtab[tid] = __float_as_uint(__fdiv_rn(448.0f, 1.0f + (float)tid * 0.0078125f));
+    __syncthreads();
+
+    if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE>(p, C, in, out, tid);
+    else if (warp == kLoadWarp) { if (lane == 0) load_warp(p, C, in); }
+    else store_warp<KIND, THREE, STORE>(p, C, out, partials, lane);
+}
+
+template <int KIND, bool YARD, bool THREE, bool STORE>
+cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
+{
+    auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE>;
+    static bool configured = false;   // per instantiation; the attribute is per function, setting it twice is harmless
+    static int sm_count = 0;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e != cudaSuccess) return e;
+        int dev = 0;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const uint32_t resident = 2u * (uint32_t)sm_count;
+    const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
+    kfn<<<grid, kMainThreads, kSmemBytes, s>>>(p, partials);
+    return cudaGetLastError();
+}
+
+template <int KIND>
+cudaError_t launch_main_k(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
+{
+    if (v.three) {
+        return v.store ? launch_main_t<KIND, true, true, true>(p, partials, s)
+                       : launch_main_t<KIND, true, true, false>(p, partials, s);
+    }
+    if (v.yard) {
+        return v.store ? launch_main_t<KIND, true, false, true>(p, partials, s)
+                       : launch_main_t<KIND, true, false, false>(p, partials, s);
+    }
+    return v.store ? launch_main_t<KIND, false, false, true>(p, partials, s)
+                   : launch_main_t<KIND, false, false, false>(p, partials, s);
+}
+
+}  // namespace
+
+cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
+{
+    if (p.total_tiles == 0) return cudaSuccess;
+    switch (v.kind) {
+        case KIND_TENSOR: return launch_main_k<KIND_TENSOR>(v, p, partials, s);
+        case KIND_ROW128: return launch_main_k<KIND_ROW128>(v, p, partials, s);
+        case KIND_BLK128: return launch_main_k<KIND_BLK128>(v, p, partials, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace mor
