@@ -5,20 +5,21 @@
 // codes, scale bytes, selection bytes and a per-tile partial for the tensor-wide aggregate.
 //
 // Structure: persistent CTAs (two per SM), ten warps each.
-//   load warp      one thread walks the CTA's tiles and brings each one in with a TMA tile load
-//                  (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) into a two-stage
-//                  ring of 32 KiB buffers, signalling an mbarrier per stage;
+//   load warp      sleeps on a hardware barrier until the compute warps have copied a stage of the
+//                  two-stage ring of 32 KiB buffers to registers, then one thread starts the TMA
+//                  tile load (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) of the
+//                  tile that uses the stage next; an mbarrier per stage tells when it has landed;
 //   compute warps  8 warps, two threads per tile row.  A thread copies its 64 elements from the
-//                  stage to registers (the stage is handed back to the load warp at once), scans
-//                  them for amax / smallest non-zero, derives the scale, converts and accumulates
-//                  the error terms from the registers, and writes its codes to a 16 KiB staging
-//                  buffer;
-//   store warp     waits for the staging buffer, issues the TMA tile store of the codes (clipped
-//                  at the tensor's edge by the hardware), adds up the threads' sums in a fixed
-//                  order, and writes the tile's partial and, for 128x128 blocks, the block's
-//                  decision and metadata.
+//                  stage to registers, scans them for amax / smallest non-zero, derives the scale,
+//                  converts and accumulates the error terms from the registers, and writes its
+//                  codes to a 16 KiB staging buffer;
+//   store warp     sleeps on a hardware barrier until the staging buffer is complete, issues the
+//                  TMA tile store of the codes (clipped at the tensor's edge by the hardware),
+//                  adds up the threads' sums in a fixed order, and writes the tile's partial and,
+//                  for 128x128 blocks, the block's decision and metadata.
 // Every wait on an mbarrier is bounded; a wait that runs out sets a status word that the
-// finalise kernel copies into mor_tensor_stats_t.status, and the CTA winds down.
+// finalise kernel copies into mor_tensor_stats_t.status.  From then on the CTA's threads skip
+// the work and the waits but keep every barrier arrival, so that nobody is left waiting.
 //
 // Arithmetic that must be exact: amax (integer compare of BF16 bit patterns), the scale (IEEE
 // binary32 division, looked up by the 7 mantissa bits of the BF16 amax from a table that each
@@ -38,10 +39,12 @@ constexpr int kStages = 2;
 constexpr int kInBytes = kTileRows * kTileCols * 2;      // 32768
 constexpr int kOutBytes = kTileRows * kTileCols;         // 16384
 constexpr int kComputeWarps = kThreads / 32;             // 8
-constexpr int kLoadWarp = kComputeWarps;                 // warp 8
-constexpr int kStoreWarp = kComputeWarps + 1;            // warp 9
+constexpr int kLoadWarp = kComputeWarps;                 // warp 8; warp 9 is the store warp
+constexpr int kBarCompute = 1;                           // hardware barrier of the compute threads
+constexpr int kBarOutFull = 2;                           // + staging buffer index: compute threads arrive, store warp waits
+constexpr int kBarStageFree = 4;                         // + stage index: compute threads arrive, load warp waits
 constexpr uint32_t kBf16Inf = 0x7F80u;
-constexpr uint32_t kSpinLimit = 1u << 17;                // x 20 us suspend hint: a few seconds at most
+constexpr long long kWaitCycles = 4000000000ll;          // a wait on an mbarrier gives up after about two seconds
 constexpr uint32_t kSelNone = 3u;                        // entry of a tile row outside the tensor
 
 // What the load warp tells the other warps about the tile in a stage.
@@ -62,8 +65,8 @@ struct __align__(16) Entry {
 };
 
 struct Control {
-    unsigned long long full[kStages], empty[kStages];   // input ring
-    unsigned long long out_full[2], out_empty[2];       // code staging + entries
+    unsigned long long full[kStages];                   // input ring: the tile has landed
+    unsigned long long out_empty[2];                    // code staging + entries have been consumed
     unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
     unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
     TileMeta meta[kStages];
@@ -73,6 +76,7 @@ struct Control {
     uint32_t tile_key[2];                                // BLK128: amax bits << 16 | 0xFFFF - (min - 1)
     uint32_t dec_sel[2];
     uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
+    uint32_t issued;                                     // tile loads issued so far by this CTA
     volatile uint32_t abort;
 };
 
@@ -94,19 +98,35 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Poll with a pause between tries (the pause keeps a waiting warp from taking issue slots away
+// from the warps that compute); gives up after kWaitCycles.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const volatile uint32_t* abort_flag)
+{
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            __nanosleep(64);
+            if (mbar_test(bar, parity)) return true;
+        }
+        if (abort_flag != nullptr && *abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+}
 // Bounded wait for the phase with the given parity; false when the limit ran out or (with a flag
 // given) another thread of the CTA has given up already.
 __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, const volatile uint32_t* abort_flag)
 {
     const uint32_t a = smem_addr(bar);
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        uint32_t done;
-        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
-                     : "=r"(done) : "r"(a), "r"(parity), "r"(20000u) : "memory");
-        if (done) return true;
-        if (abort_flag != nullptr && *abort_flag) return false;
-    }
-    return false;
+    if (mbar_test(a, parity)) return true;
+    return mbar_wait_slow(a, parity, abort_flag);
 }
 __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, void* bar)
 {
@@ -127,9 +147,28 @@ __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier
 __device__ __forceinline__ bool compute_bar_or(bool v)
 {
     uint32_t r;
-    asm volatile("{ .reg .pred p, q; setp.ne.u32 p, %1, 0; barrier.cta.red.or.pred q, 1, %2, p; selp.u32 %0, 1, 0, q; }"
-                 : "=r"(r) : "r"((uint32_t)v), "n"(kThreads) : "memory");
+    asm volatile("{ .reg .pred p, q; setp.ne.u32 p, %1, 0; barrier.cta.red.or.pred q, %2, %3, p; selp.u32 %0, 1, 0, q; }"
+                 : "=r"(r) : "r"((uint32_t)v), "n"(kBarCompute), "n"(kThreads) : "memory");
     return r != 0;
+}
+// Producer / consumer hand-off on hardware barriers: the 256 compute threads announce, the 32
+// threads of the load warp (a stage is free) or of the store warp (a staging buffer is complete)
+// sleep until all have.  A thread asleep on a hardware barrier takes no issue slots.
+__device__ __forceinline__ void stage_free_arrive(uint32_t s)
+{
+    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(kBarStageFree + s), "n"(kThreads + 32) : "memory");
+}
+__device__ __forceinline__ void stage_free_sync(uint32_t s)
+{
+    asm volatile("barrier.cta.sync %0, %1;" ::"r"(kBarStageFree + s), "n"(kThreads + 32) : "memory");
+}
+__device__ __forceinline__ void out_full_arrive(uint32_t b)
+{
+    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(kBarOutFull + b), "n"(kThreads + 32) : "memory");
+}
+__device__ __forceinline__ void out_full_sync(uint32_t b)
+{
+    asm volatile("barrier.cta.sync %0, %1;" ::"r"(kBarOutFull + b), "n"(kThreads + 32) : "memory");
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t a)
@@ -175,6 +214,12 @@ __device__ __forceinline__ void diff_f16x2_f32(uint32_t q, float ylo, float yhi,
 {
     asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; sub.f32.f16 %0, l, %3; sub.f32.f16 %1, h, %4; }"
         : "=f"(dlo), "=f"(dhi) : "r"(q), "f"(ylo), "f"(yhi));
+}
+// the two BF16 halves of a word as binary32, by the mixed-precision subtract x - 0 (keeps -0)
+__device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi)
+{
+    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; sub.f32.bf16 %0, l, %3; sub.f32.bf16 %1, h, %3; }"
+        : "=f"(lo), "=f"(hi) : "r"(w), "f"(0.0f));
 }
 __device__ __forceinline__ float rcp_ftz(float a)
 {
@@ -275,29 +320,48 @@ __device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
 //   min   per-halfword min of (|x| bits - 1) mod 2^16: zeros wrap to 0xFFFF and drop out.
 __device__ __forceinline__ uint32_t scan_words(const uint32_t (&w)[32])
 {
-    uint32_t mx = 0u, mn = 0xFFFFFFFFu;
+    uint32_t mx[2] = {0u, 0u}, mn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-        const uint32_t a0 = w[i] & 0x7FFF7FFFu, a1 = w[i + 1] & 0x7FFF7FFFu;
-        mx = __vimax3_u16x2(mx, a0, a1);
-        mn = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn);
-        mn = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn);
+    for (int i = 0; i < 32; i += 4) {
+        const uint32_t a0 = w[i] & 0x7FFF7FFFu, a1 = w[i + 1] & 0x7FFF7FFFu, a2 = w[i + 2] & 0x7FFF7FFFu, a3 = w[i + 3] & 0x7FFF7FFFu;
+        mx[0] = __vimax3_u16x2(mx[0], a0, a1);
+        mx[1] = __vimax3_u16x2(mx[1], a2, a3);
+        mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
+        mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
+        mn[2] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn[2]);
+        mn[3] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn[3]);
     }
-    const uint32_t amax = max(mx & 0xFFFFu, mx >> 16), minm1 = min(mn & 0xFFFFu, mn >> 16);
+    const uint32_t mxx = __vimax3_u16x2(mx[0], mx[1], mx[1]);
+    const uint32_t mnn = __vimin3_u16x2(__vimin3_u16x2(mn[0], mn[1], mn[2]), mn[3], mn[3]);
+    const uint32_t amax = max(mxx & 0xFFFFu, mxx >> 16), minm1 = min(mnn & 0xFFFFu, mnn >> 16);
     return (amax << 16) | (0xFFFFu - minm1);
 }
 
-// the same over finite elements only (used once a non-finite element has been seen)
-__device__ __noinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
+// the same over finite elements only (used once a non-finite element has been seen).  A real
+// call, with the words passed by value in registers: inlined, the compiler turns this rare path
+// into predicated instructions that every tile would pay for.
+__device__ __forceinline__ void scan_finite4(uint4 v, uint32_t& m, uint32_t& n)
 {
-    uint32_t m = 0u, n = 0xFFFFu;
-#pragma unroll 1
-    for (int i = 0; i < 32; ++i) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
         const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
         if (lo < kBf16Inf) { m = max(m, lo); n = min(n, (lo - 1u) & 0xFFFFu); }
         if (hi < kBf16Inf) { m = max(m, hi); n = min(n, (hi - 1u) & 0xFFFFu); }
     }
+}
+__device__ __noinline__ uint32_t scan_finite_call(uint4 a, uint4 b, uint4 c, uint4 d, uint4 e, uint4 f, uint4 g, uint4 h)
+{
+    uint32_t m = 0u, n = 0xFFFFu;
+    scan_finite4(a, m, n); scan_finite4(b, m, n); scan_finite4(c, m, n); scan_finite4(d, m, n);
+    scan_finite4(e, m, n); scan_finite4(f, m, n); scan_finite4(g, m, n); scan_finite4(h, m, n);
     return (m << 16) | (0xFFFFu - n);
+}
+__device__ __forceinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
+{
+#define MOR_W4(j) make_uint4(w[4 * (j)], w[4 * (j) + 1], w[4 * (j) + 2], w[4 * (j) + 3])
+    return scan_finite_call(MOR_W4(0), MOR_W4(1), MOR_W4(2), MOR_W4(3), MOR_W4(4), MOR_W4(5), MOR_W4(6), MOR_W4(7));
+#undef MOR_W4
 }
 
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
@@ -316,7 +380,9 @@ __device__ __forceinline__ void convert_pair_fast(uint32_t w, unsigned long long
                                                   unsigned long long tiny2, float& a43, float& a52,
                                                   unsigned long long& cnt2, uint32_t& c4, uint32_t& c5)
 {
-    const unsigned long long x2 = pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    float xlo, xhi;
+    unpack_bf16x2(w, xlo, xhi);
+    const unsigned long long x2 = pack_f32x2(xlo, xhi);
     const unsigned long long y2 = mul_f32x2(x2, s4x2);
     float ylo, yhi, ulo, uhi;
     unpack_f32x2(y2, ylo, yhi);
@@ -466,6 +532,7 @@ __device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43,
     return MOR_FMT_E4M3;   // tensor-level criterion: decided by the finalise kernel
 }
 
+
 // ------------------------------------------------------------------ tile bookkeeping ----
 
 struct TileId {
@@ -503,29 +570,39 @@ __device__ __forceinline__ double shfl_xor_f64(double v, int o) { return __shfl_
 
 // ------------------------------------------------------------------ load warp ----
 
-__device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in)
+// One thread: start the TMA load of the CTA's tile number `it` into its stage (nothing when the CTA
+// has no such tile).  The stage must be free.
+__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it)
 {
-    uint32_t issued = 0;
-    bool ok = true;
+    const uint32_t tile = blockIdx.x + it * gridDim.x;
+    if (tile >= p.total_tiles) return;
+    const uint32_t s = it % kStages;
+    const TileId t = locate_tile(p.b, tile);
+    TileMeta m;
+    m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
+    m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
+    m.pad = 0;
+    C.meta[s] = m;
+    mbar_arrive_expect_tx(&C.full[s], kInBytes);
+    tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
+    C.issued = it + 1;
+}
+
+__device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in, int lane)
+{
+    if (lane == 0) {
+        for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load(p, C, in, it);
+    }
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
         const uint32_t tile = blockIdx.x + it * gridDim.x;
         if (tile >= p.total_tiles) break;
-        const uint32_t s = it % kStages, n = it / kStages;
-        if (n > 0 && !mbar_wait(&C.empty[s], (n - 1) & 1u, &C.abort)) { ok = false; break; }
-        const TileId t = locate_tile(p.b, tile);
-        TileMeta m;
-        m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
-        m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
-        m.pad = 0;
-        C.meta[s] = m;
-        mbar_arrive_expect_tx(&C.full[s], kInBytes);
-        tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
-        issued = it + 1;
+        stage_free_sync(it % kStages);                  // sleeps until every compute thread has its copy
+        if (lane == 0 && !C.abort) issue_tile_load(p, C, in, it + kStages);
     }
-    if (!ok || C.abort) {
-        // the compute warps may have left: the copies still in flight must land before the CTA goes
-        if (!ok) give_up(C, p.device_status);
+    if (lane == 0 && C.abort) {
+        // copies that may still be in flight must land (or be given up on) before the CTA goes
+        const uint32_t issued = C.issued;
         for (uint32_t k = 0; k < (uint32_t)kStages && k < issued; ++k) {
             const uint32_t it = issued - 1 - k;
             mbar_wait(&C.full[it % kStages], (it / kStages) & 1u, nullptr);
@@ -546,77 +623,78 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const uint32_t tile = blockIdx.x + it * gridDim.x;
         if (tile >= p.total_tiles) break;
         const uint32_t b = it & 1u, n = it >> 1;
-        const TileId t = locate_tile(p.b, tile);
-        const TensorRec& R = p.b.t[t.ti];
-        bool ok = mbar_wait(&C.out_full[b], n & 1u, &C.abort);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (!ok) { if (lane == 0) give_up(C, p.device_status); break; }
+        out_full_sync(b);                                // sleeps until every compute thread has arrived
+        if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
+            const TileId t = locate_tile(p.b, tile);
+            const TensorRec& R = p.b.t[t.ti];
 
-        // the threads' sums in a fixed order: lane-strided, then a butterfly
-        double s43 = 0.0, s52 = 0.0;
-        uint32_t nnz = 0, nonf = 0, n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
+            // the threads' sums in a fixed order: lane-strided, then a butterfly
+            double s43 = 0.0, s52 = 0.0;
+            uint32_t nnz = 0, nonf = 0, n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
 #pragma unroll
-        for (int k = 0; k < kEntries / 32; ++k) {
-            const Entry e = C.entry[b][lane + 32 * k];
-            s43 += (double)e.e43;
-            s52 += (double)e.e52;
-            nnz += e.nnz_nonf & 0xFFFFu;
-            nonf += e.nnz_nonf >> 16;
-            const uint32_t sel = e.sel_min & 0xFFFFu;
-            n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
-            mn = min(mn, e.sel_min >> 16);
-        }
+            for (int k = 0; k < kEntries / 32; ++k) {
+                const Entry e = C.entry[b][lane + 32 * k];
+                s43 += (double)e.e43;
+                s52 += (double)e.e52;
+                nnz += e.nnz_nonf & 0xFFFFu;
+                nonf += e.nnz_nonf >> 16;
+                const uint32_t sel = e.sel_min & 0xFFFFu;
+                n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
+                mn = min(mn, e.sel_min >> 16);
+            }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
-        nnz = __reduce_add_sync(0xFFFFFFFFu, nnz);
-        nonf = __reduce_add_sync(0xFFFFFFFFu, nonf);
-        mn = __reduce_min_sync(0xFFFFFFFFu, mn);
-        if (KIND == KIND_ROW128) {
-            n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
-            n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
-            nb = __reduce_add_sync(0xFFFFFFFFu, nb);
-        } else {
-            n4 = n5 = nb = 0;
-        }
+            for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
+            nnz = __reduce_add_sync(0xFFFFFFFFu, nnz);
+            nonf = __reduce_add_sync(0xFFFFFFFFu, nonf);
+            mn = __reduce_min_sync(0xFFFFFFFFu, mn);
+            if (KIND == KIND_ROW128) {
+                n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
+                n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
+                nb = __reduce_add_sync(0xFFFFFFFFu, nb);
+            } else {
+                n4 = n5 = nb = 0;
+            }
 
-        const bool need_dec = KIND == KIND_BLK128 && (THREE || R.fallback != nullptr);
-        if (lane == 0) {
-            if (KIND == KIND_BLK128) {
-                const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
-                const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
-                const uint32_t bsel = decide_block(R, s43, s52, nnz, nonf, amax_bits, minm1, (uint32_t)(t.vrows * t.vcols));
-                const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
-                if (R.sel) R.sel[t.local] = (uint8_t)bsel;
-                if (R.scale_e8m0) R.scale_e8m0[t.local] = (uint8_t)(sb >> 23);
-                if (R.scale_f32) R.scale_f32[t.local] = __uint_as_float(sb);
-                if (R.block_stats) {
-                    mor_block_stats_t bs;
-                    bs.amax = __uint_as_float(amax_bits << 16);
-                    bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                    bs.nnz = nnz; bs.n_nonfinite = nonf;
-                    bs.sum_rel_e4m3 = (float)s43; bs.sum_rel_e5m2 = (float)s52;
-                    R.block_stats[t.local] = bs;
-                }
-                n4 = bsel == MOR_FMT_E4M3; n5 = bsel == MOR_FMT_E5M2; nb = bsel == MOR_FMT_BF16;
-                if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }
-            }
-            Partial P;
-            P.sum43 = s43; P.sum52 = s52; P.nnz = nnz; P.nonfinite = nonf;
-            P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
-            partials[R.tile_begin + t.local] = P;
-        }
-        if (STORE) {
-            if (KIND == KIND_BLK128 && THREE) {
-                // the compute threads put the chosen format's codes in place after the decision
-                ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) { if (lane == 0) give_up(C, p.device_status); break; }
-            }
+            const bool need_dec = KIND == KIND_BLK128 && (THREE || R.fallback != nullptr);
             if (lane == 0) {
-                tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
-                bulk_commit();
-                stores_pending = true;
-                bulk_wait_read<0>();      // the staging buffer may be overwritten from here on
+                if (KIND == KIND_BLK128) {
+                    const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
+                    const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
+                    const uint32_t bsel = decide_block(R, s43, s52, nnz, nonf, amax_bits, minm1, (uint32_t)(t.vrows * t.vcols));
+                    const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
+                    if (R.sel) R.sel[t.local] = (uint8_t)bsel;
+                    if (R.scale_e8m0) R.scale_e8m0[t.local] = (uint8_t)(sb >> 23);
+                    if (R.scale_f32) R.scale_f32[t.local] = __uint_as_float(sb);
+                    if (R.block_stats) {
+                        mor_block_stats_t bs;
+                        bs.amax = __uint_as_float(amax_bits << 16);
+                        bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                        bs.nnz = nnz; bs.n_nonfinite = nonf;
+                        bs.sum_rel_e4m3 = (float)s43; bs.sum_rel_e5m2 = (float)s52;
+                        R.block_stats[t.local] = bs;
+                    }
+                    n4 = bsel == MOR_FMT_E4M3; n5 = bsel == MOR_FMT_E5M2; nb = bsel == MOR_FMT_BF16;
+                    if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }
+                }
+                Partial P;
+                P.sum43 = s43; P.sum52 = s52; P.nnz = nnz; P.nonfinite = nonf;
+                P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
+                partials[R.tile_begin + t.local] = P;
+            }
+            if (STORE) {
+                bool ok = true;
+                if (KIND == KIND_BLK128 && THREE) {
+                    // the compute threads put the chosen format's codes in place after the decision
+                    ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok && lane == 0) give_up(C, p.device_status);
+                }
+                if (ok && lane == 0) {
+                    tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
+                    bulk_commit();
+                    stores_pending = true;
+                    bulk_wait_read<0>();      // the staging buffer may be overwritten from here on
+                }
             }
         }
         __syncwarp();
@@ -661,14 +739,19 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
 
     int cur_ti = -1;
     uint32_t m_g = 0;
+    bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
         const uint32_t tile = blockIdx.x + it * gridDim.x;
         if (tile >= p.total_tiles) break;
         const uint32_t s = it % kStages, b = it & 1u, n2 = it >> 1;
 
-        bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
-        const TileMeta m = C.meta[s];
+        if (!dead) {
+            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+        }
+        TileMeta m = C.meta[s];
         uint32_t w[32];
         {
             const uint32_t a = in_base + s * kInBytes + in_off;
@@ -678,22 +761,17 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
             }
         }
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (lane == 0) {
-            if (ok) mbar_arrive(&C.empty[s]);          // every lane's loads have returned: the stage is free
-            else give_up(C, p.device_status);
-        }
-        if (KIND != KIND_BLK128 && !ok) break;
-
-        const TensorRec& R = p.b.t[ok ? m.ti : 0];
-        if (m.ti != cur_ti && ok) {
+        stage_free_arrive(s);                           // this thread's copy of the stage is in registers
+        if (dead) m.ti = 0;
+        const TensorRec& R = p.b.t[m.ti];
+        if (m.ti != cur_ti && !dead) {
             cur_ti = m.ti;
             m_g = group_mantissa(*R.amax, R.scale_mode);   // Algorithm 1, group part, once per tensor
         }
 
         // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
         uint32_t key = scan_words(w);
-        bool nonfin;
+        bool nonfin = false;
         if (KIND == KIND_ROW128) {
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
@@ -706,11 +784,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             for (int pass = 0; pass < 2; ++pass) {
                 const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, key >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, key & 0xFFFFu);
                 if (lane == 0) C.wmax[b][pass][warp] = (hi << 16) | lo;
-                if (compute_bar_or(!ok)) return;                                   // all compute threads leave together
+                dead = compute_bar_or(dead);                                       // also spreads the word that a wait ran out
                 const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]);
                 const uint4 k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
                 key = key_max(key_max(__vimax3_u16x2(k0.x, k0.y, k0.z), k0.w), key_max(__vimax3_u16x2(k1.x, k1.y, k1.z), k1.w));
                 nonfin = pass == 1 || (key >> 16) >= kBf16Inf;                     // CTA-uniform
+                if (dead) { key = 0u; nonfin = false; }
                 if (pass == 1 || !nonfin) break;
                 key = scan_words_finite(w);
             }
@@ -733,79 +812,79 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         if (KIND != KIND_BLK128) careful = __any_sync(0xFFFFFFFFu, careful);
 
         // ---- staging buffer and entries of tile it - 2 must have been consumed ----
-        if (n2 > 0) {
-            bool ok2 = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
-            ok2 = __all_sync(0xFFFFFFFFu, ok2);
-            if (!ok2) {
-                if (lane == 0) give_up(C, p.device_status);
-                if (KIND != KIND_BLK128) break;
-                ok = false;
-            }
+        if (n2 > 0 && !dead) {
+            bool ok = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
         }
 
-        // ---- cast and error terms ----
-        float e43, e52;
-        uint32_t nnz, nonf;
-        uint2 k5[8];
         const uint32_t oa = out_base + b * kOutBytes + out_off;
-        if (careful) convert_words<YARD, THREE, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
-        else         convert_words<YARD, THREE, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
+        uint2 k5[8];
+        uint32_t sel = MOR_FMT_E4M3;
+        if (!dead) {
+            // ---- cast and error terms ----
+            float e43, e52;
+            uint32_t nnz, nonf;
+            if (careful) convert_words<YARD, THREE, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
+            else         convert_words<YARD, THREE, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
 
-        if (KIND == KIND_ROW128) {
-            // ---- block sums, decision, metadata ----
-            e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
-            e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
-            uint32_t nz = nnz | (nonf << 16);
-            nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
-            const bool valid = row < m.vrows;
-            const uint32_t sel = decide_block(R, (double)e43, (double)e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
-            if (THREE && STORE && sel == MOR_FMT_E5M2) {
+            if (KIND == KIND_ROW128) {
+                // ---- block sums, decision, metadata ----
+                e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
+                e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
+                uint32_t nz = nnz | (nonf << 16);
+                nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
+                const bool valid = row < m.vrows;
+                sel = decide_block(R, (double)e43, (double)e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
+                if (THREE && STORE && sel == MOR_FMT_E5M2) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
-            }
-            if (h == 0) {
-                Entry e;
-                e.e43 = e43; e.e52 = e52; e.nnz_nonf = nz;
-                e.sel_min = (valid ? sel : kSelNone) | (minm1 << 16);
-                C.entry[b][row] = e;
-                if (valid) {
-                    const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
-                    const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
-                    if (R.sel) R.sel[blk] = (uint8_t)sel;
-                    if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
-                    if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
-                    if (R.block_stats) {
-                        mor_block_stats_t bs;
-                        bs.amax = __uint_as_float(amax_bits << 16);
-                        bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                        bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
-                        R.block_stats[blk] = bs;
+                    for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
+                }
+                if (h == 0) {
+                    Entry e;
+                    e.e43 = e43; e.e52 = e52; e.nnz_nonf = nz;
+                    e.sel_min = (valid ? sel : kSelNone) | (minm1 << 16);
+                    C.entry[b][row] = e;
+                    if (valid) {
+                        const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
+                        const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
+                        if (R.sel) R.sel[blk] = (uint8_t)sel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
+                        if (R.block_stats) {
+                            mor_block_stats_t bs;
+                            bs.amax = __uint_as_float(amax_bits << 16);
+                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                            bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
+                            R.block_stats[blk] = bs;
+                        }
                     }
                 }
+                if (STORE && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+            } else {
+                Entry e;
+                e.e43 = e43; e.e52 = e52; e.nnz_nonf = nnz | (nonf << 16);
+                e.sel_min = kSelNone | (minm1 << 16);
+                C.entry[b][tid] = e;
+                if (KIND == KIND_BLK128 && tid == 0) {
+                    C.tile_scale[b][0] = s4b; C.tile_scale[b][1] = s5b; C.tile_key[b] = key;
+                }
             }
-            if (STORE && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
-        } else {
-            Entry e;
-            e.e43 = e43; e.e52 = e52; e.nnz_nonf = nnz | (nonf << 16);
-            e.sel_min = kSelNone | (minm1 << 16);
-            C.entry[b][tid] = e;
-            if (KIND == KIND_BLK128 && tid == 0) {
-                C.tile_scale[b][0] = s4b; C.tile_scale[b][1] = s5b; C.tile_key[b] = key;
-            }
+            if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
         }
-        if (STORE) fence_async_smem();                  // the codes must be visible to the TMA store
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&C.out_full[b]);
+        out_full_arrive(b);
 
         if (KIND == KIND_BLK128) {
             const bool need_dec = THREE || R.fallback != nullptr;
             if (need_dec) {
-                bool ok3 = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
-                ok3 = __all_sync(0xFFFFFFFFu, ok3);
-                if (!ok3) { if (lane == 0) give_up(C, p.device_status); ok = false; }
-                const uint32_t sel = C.dec_sel[b];
+                if (!dead) {
+                    bool ok = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+                }
+                if (!dead) sel = C.dec_sel[b];
                 if (THREE && STORE) {
-                    if (ok3 && sel == MOR_FMT_E5M2) {
+                    if (!dead && sel == MOR_FMT_E5M2) {
 #pragma unroll
                         for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
                     }
@@ -813,7 +892,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&C.codes_full[b]);
                 }
-                if (STORE && ok3 && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                if (STORE && !dead && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
             }
         }
     }
@@ -833,12 +912,14 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], kComputeWarps); }
+        for (int s = 0; s < kStages; ++s) mbar_init(&C.full[s], 1);
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&C.out_full[b], kComputeWarps); mbar_init(&C.out_empty[b], 1);
-            mbar_init(&C.dec_full[b], 1); mbar_init(&C.codes_full[b], kComputeWarps);
+            mbar_init(&C.out_empty[b], 1);
+            mbar_init(&C.dec_full[b], 1);
+            mbar_init(&C.codes_full[b], kComputeWarps);
         }
         C.abort = 0u;
+        C.issued = 0u;
         fence_mbar_init();
     }
     // fl32(448 / (1 + m/128)) for the 128 mantissas of a BF16 amax: the division of Algorithm 1,
@@ -847,7 +928,7 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     __syncthreads();
 
     if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE>(p, C, in, out, tid);
-    else if (warp == kLoadWarp) { if (lane == 0) load_warp(p, C, in); }
+    else if (warp == kLoadWarp) load_warp(p, C, in, lane);
     else store_warp<KIND, THREE, STORE>(p, C, out, partials, lane);
 }
 
@@ -855,19 +936,20 @@ template <int KIND, bool YARD, bool THREE, bool STORE>
 cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
 {
     auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE>;
-    static bool configured = false;   // per instantiation; the attribute is per function, setting it twice is harmless
-    static int sm_count = 0;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    static bool configured[64] = {};   // per instantiation and device
+    static int sm_count[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+        e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        int dev = 0;
-        e = cudaGetDevice(&dev);
+        e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
-    const uint32_t resident = 2u * (uint32_t)sm_count;
+    const uint32_t resident = 2u * (uint32_t)sm_count[dev];
     const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
     kfn<<<grid, kMainThreads, kSmemBytes, s>>>(p, partials);
     return cudaGetLastError();
