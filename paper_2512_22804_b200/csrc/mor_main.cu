@@ -44,16 +44,16 @@ constexpr int kBarCompute = 1;                           // hardware barrier of 
 constexpr int kBarOutFull = 2;                           // + staging buffer index: compute threads arrive, store warp waits
 constexpr int kBarStageFree = 4;                         // + stage index: compute threads arrive, load warp waits
 constexpr uint32_t kBf16Inf = 0x7F80u;
-constexpr long long kWaitCycles = 4000000000ll;          // a wait on an mbarrier gives up after about two seconds
+constexpr long long kWaitCycles = 400000000ll;           // a wait on an mbarrier gives up after about 0.2 s
 constexpr uint32_t kSelNone = 3u;                        // entry of a tile row outside the tensor
 
 // What the load warp tells the other warps about the tile in a stage.
-struct TileMeta {
-    int32_t ti;            // tensor index within the launch, -1 = no more tiles
-    uint32_t local;        // tile index within the tensor
-    int32_t row0, col0;    // first row / column of the tile
+struct __align__(16) TileMeta {
+    int32_t ti;            // tensor index within the launch
     int32_t vrows, vcols;  // rows / columns of the tile inside the tensor (1..128)
     uint32_t blk_base;     // ROW128: index of the block of the tile's first row
+    uint32_t local;        // tile index within the tensor
+    int32_t row0, col0;    // first row / column of the tile
     uint32_t pad;
 };
 
@@ -176,6 +176,10 @@ __device__ __forceinline__ uint4 lds128(uint32_t a)
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void sts64(uint32_t a, uint2 v)
 {
@@ -508,7 +512,8 @@ __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t 
 
 // Algorithm 2 for one block with the per-block metrics (M_1 = Eq. 3, M_2 = Eq. 4, or
 // Eq. 1-2 on the block alone).
-__device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43, double e52, uint32_t nnz,
+template <typename T>
+__device__ __forceinline__ uint32_t decide_block(const TensorRec& R, T e43, T e52, uint32_t nnz,
                                                  uint32_t nonfinite, uint32_t amax_bits, uint32_t minm1_bits,
                                                  uint32_t n_elems)
 {
@@ -526,7 +531,7 @@ __device__ __forceinline__ uint32_t decide_block(const TensorRec& R, double e43,
         return MOR_FMT_BF16;
     }
     if (R.criterion == MOR_CRIT_BLOCK_MEAN_REL) {
-        const double err = nnz ? e43 / (double)nnz : 0.0;
+        const double err = nnz ? (double)e43 / (double)nnz : 0.0;
         return err < (double)R.threshold ? MOR_FMT_E4M3 : MOR_FMT_BF16;
     }
     return MOR_FMT_E4M3;   // tensor-level criterion: decided by the finalise kernel
@@ -655,7 +660,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 n4 = n5 = nb = 0;
             }
 
-            const bool need_dec = KIND == KIND_BLK128 && (THREE || R.fallback != nullptr);
+            const bool need_dec = KIND == KIND_BLK128 && (THREE || (STORE && R.fallback != nullptr));
             if (lane == 0) {
                 if (KIND == KIND_BLK128) {
                     const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
@@ -735,10 +740,15 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     const int swz = (row & 7) ^ (h << 2);
     const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
     const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
-    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out);
+    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
 
+    // what changes only with the tensor, kept in registers
     int cur_ti = -1;
-    uint32_t m_g = 0;
+    uint32_t m_g = 0;            // Algorithm 1, group part
+    int scale_mode = 0;
+    bool has_fallback = false;
+    uint32_t tensor_amax_bits = 0;
+    const uint32_t meta_base = smem_addr(&C.meta[0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
@@ -751,7 +761,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
         }
-        TileMeta m = C.meta[s];
+        TileMeta m;
+        {
+            const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
+            m.ti = dead ? 0 : (int32_t)q.x; m.vrows = (int32_t)q.y; m.vcols = (int32_t)q.z; m.blk_base = q.w;
+            m.local = 0; m.row0 = 0; m.col0 = 0; m.pad = 0;
+        }
         uint32_t w[32];
         {
             const uint32_t a = in_base + s * kInBytes + in_off;
@@ -761,13 +776,21 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
             }
         }
-        stage_free_arrive(s);                           // this thread's copy of the stage is in registers
-        if (dead) m.ti = 0;
         const TensorRec& R = p.b.t[m.ti];
-        if (m.ti != cur_ti && !dead) {
+        if (m.ti != cur_ti) {
             cur_ti = m.ti;
-            m_g = group_mantissa(*R.amax, R.scale_mode);   // Algorithm 1, group part, once per tensor
+            scale_mode = R.scale_mode;
+            has_fallback = STORE && R.fallback != nullptr;
+            if (!dead) {
+                m_g = group_mantissa(*R.amax, scale_mode);
+                if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
+            }
         }
+        if (has_fallback) {      // the copy of BF16 blocks needs the tile's position too
+            const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
+            m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z;
+        }
+        stage_free_arrive(s);                           // this thread's copy of the stage is in registers
 
         // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
         uint32_t key = scan_words(w);
@@ -800,10 +823,10 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         uint32_t amax_bits = key >> 16;
         const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
         // per-tensor partition: the block is the tensor, its amax was reduced by the pre-pass
-        if (KIND == KIND_TENSOR) amax_bits = __float_as_uint(*R.amax_slot) >> 16;
+        if (KIND == KIND_TENSOR) amax_bits = tensor_amax_bits;
 
         uint32_t s4b, s5b;
-        block_scale(amax_bits, m_g, R.scale_mode, C.rtab, s4b, s5b);
+        block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
 
         // The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_pair_fast).
         // minm1 covers this thread's block (ROW128), this tile (BLK128), this thread (TENSOR).
@@ -835,16 +858,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 uint32_t nz = nnz | (nonf << 16);
                 nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
                 const bool valid = row < m.vrows;
-                sel = decide_block(R, (double)e43, (double)e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
+                sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
                 if (THREE && STORE && sel == MOR_FMT_E5M2) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
                 }
                 if (h == 0) {
-                    Entry e;
-                    e.e43 = e43; e.e52 = e52; e.nnz_nonf = nz;
-                    e.sel_min = (valid ? sel : kSelNone) | (minm1 << 16);
-                    C.entry[b][row] = e;
+                    sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
+                           make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
                     if (valid) {
                         const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
                         const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
@@ -860,12 +881,10 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                         }
                     }
                 }
-                if (STORE && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                if (has_fallback && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
             } else {
-                Entry e;
-                e.e43 = e43; e.e52 = e52; e.nnz_nonf = nnz | (nonf << 16);
-                e.sel_min = kSelNone | (minm1 << 16);
-                C.entry[b][tid] = e;
+                sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
+                       make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
                 if (KIND == KIND_BLK128 && tid == 0) {
                     C.tile_scale[b][0] = s4b; C.tile_scale[b][1] = s5b; C.tile_key[b] = key;
                 }
@@ -875,7 +894,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         out_full_arrive(b);
 
         if (KIND == KIND_BLK128) {
-            const bool need_dec = THREE || R.fallback != nullptr;
+            const bool need_dec = THREE || has_fallback;
             if (need_dec) {
                 if (!dead) {
                     bool ok = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
@@ -892,7 +911,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&C.codes_full[b]);
                 }
-                if (STORE && !dead && R.fallback != nullptr && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                if (has_fallback && !dead && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
             }
         }
     }
