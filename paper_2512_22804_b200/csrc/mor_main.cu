@@ -465,13 +465,13 @@ __device__ __forceinline__ void convert_pair_careful(uint32_t w, float s4, float
 }
 
 // A thread's 64 elements, held as 8 chunks of 4 words; chunk j belongs at byte offset
-// (j ^ swz) * 8 of the thread's 64 code bytes.  E4M3 codes go to the staging buffer at once; with
-// three formats the E5M2 codes wait in registers for the block's decision.
+// (j ^ swz) * 8 of the thread's 64 code bytes.  The E4M3 codes go to the staging buffer; a block
+// that ends up in E5M2 has them replaced afterwards (emit_e5m2_codes).
 // Results: e43 = the thread's sum of E4M3 terms, complete; e52 = its sum of E5M2 terms, complete;
 // nnz; nonfinite.
-template <bool YARD, bool THREE, bool CAREFUL, bool STORE>
+template <bool YARD, bool CAREFUL, bool STORE>
 __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s4b, uint32_t s5b,
-                                              float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite, uint2 (&k5)[8])
+                                              float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite)
 {
     const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
     float a43[4] = {0.0f, 0.0f, 0.0f, 0.0f}, a52[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -489,7 +489,6 @@ __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t 
             else convert_pair_fast<YARD>(w[4 * j + i], s4x2, s5x2, tiny2, a43[i], a52[i], cnt2[i & 1], a[i], b[i]);
         }
         if (STORE) sts64(out_addr ^ (j << 3), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
-        if (THREE) k5[j] = make_uint2(__byte_perm(b[0], b[1], 0x5410), __byte_perm(b[2], b[3], 0x5410));
     }
     // scale4 / scale5 = 2^(e4 - e5)
     const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);
@@ -507,6 +506,26 @@ __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t 
         nonfinite = 0u;
         e43 = (a43[0] + a43[1]) + (a43[2] + a43[3]);
         e52 = YARD ? ((a52[0] + a52[1]) + (a52[2] + a52[3])) * ratio : 0.0f;
+    }
+}
+
+// The E5M2 codes of a thread's 64 elements, for a block that selected E5M2 (such a block holds no
+// NaN or inf): z = fl32(x * scale5), RNE-saturating cast, over the E4M3 codes in the staging buffer.
+__device__ __forceinline__ void emit_e5m2_codes(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s5b)
+{
+    const float s5 = __uint_as_float(s5b);
+    const unsigned long long s5x2 = pack_f32x2(s5, s5);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t ww = w[4 * j + i];
+            float zlo, zhi;
+            unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(ww << 16), __uint_as_float(ww & 0xFFFF0000u)), s5x2), zlo, zhi);
+            c[i] = cvt_e5m2x2(zhi, zlo);
+        }
+        sts64(out_addr ^ (j << 3), make_uint2(__byte_perm(c[0], c[1], 0x5410), __byte_perm(c[2], c[3], 0x5410)));
     }
 }
 
@@ -842,14 +861,13 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         }
 
         const uint32_t oa = out_base + b * kOutBytes + out_off;
-        uint2 k5[8];
         uint32_t sel = MOR_FMT_E4M3;
         if (!dead) {
             // ---- cast and error terms ----
             float e43, e52;
             uint32_t nnz, nonf;
-            if (careful) convert_words<YARD, THREE, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
-            else         convert_words<YARD, THREE, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf, k5);
+            if (careful) convert_words<YARD, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
+            else         convert_words<YARD, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
 
             if (KIND == KIND_ROW128) {
                 // ---- block sums, decision, metadata ----
@@ -859,10 +877,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
                 const bool valid = row < m.vrows;
                 sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
-                if (THREE && STORE && sel == MOR_FMT_E5M2) {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
-                }
+                if (THREE && STORE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
                 if (h == 0) {
                     sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
                            make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
@@ -903,10 +918,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 }
                 if (!dead) sel = C.dec_sel[b];
                 if (THREE && STORE) {
-                    if (!dead && sel == MOR_FMT_E5M2) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) sts64(oa ^ (j << 3), k5[j]);
-                    }
+                    if (!dead && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&C.codes_full[b]);
