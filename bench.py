@@ -44,9 +44,11 @@ BLOCK = (128, 128)
 ALG_BYTES_MAIN = 2.0 + 1.0 + 2.0 / (BLOCK[0] * BLOCK[1])      # BF16 read + code write + scale and selection bytes
 ALG_BYTES_STEP = ALG_BYTES_MAIN + 2.0                           # + the tensor-amax read
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one main-kernel launch over this workload's
-# batch, from the ncu capture summarised under profiles/ (None until captured)
-MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one main-kernel launch: captured on 6 tensors
+# (266.4 MB for 100.66 M elements; traffic grows in proportion to the elements) and scaled to the
+# 16 tensors of the default batch.  The write part is an undercount: codes still in L2 when the
+# kernel ends have not reached DRAM yet.  Must be set back to None when the kernel changes.
+MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH = 710.5e6
 
 
 def measured_peak():
@@ -233,7 +235,7 @@ def main():
                 "peak": peak, "peak_source": f"{peak_kind} copy bandwidth", "unit": "GB/s", "frac": achieved / peak,
                 "frac_of_8TBs": achieved / 8000.0, "ms_per_launch": ms_main,
                 "algorithmic_bytes_per_launch": elements * ALG_BYTES_MAIN,
-                "traffic": MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH}
+                "traffic": MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH * (B / 16.0) if MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH else None}
 
     # ---- end to end through the host-memory entry point: pinned inputs in, codes/scales/selection/stats out
     e2e = None
@@ -284,7 +286,7 @@ def main():
     # ---- the oracle on this machine's host cores (rank 0, single GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        reps = 5
+        reps = 9
         ts_ = []
         for _ in range(reps):
             t0 = time.perf_counter()
