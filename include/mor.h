@@ -35,7 +35,8 @@ typedef enum {
     MOR_ERR_ALIGNMENT = 3,     /* base pointer or leading dimension not aligned as stated     */
     MOR_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than mor_workspace_bytes()        */
     MOR_ERR_CUDA = 5,          /* a CUDA runtime call failed (launch, copy)                   */
-    MOR_ERR_TIMEOUT = 6,       /* reserved: a bounded device-side wait expired                */
+    MOR_ERR_TIMEOUT = 6,       /* a bounded device-side wait expired (reported in
+                                  mor_tensor_stats_t.status; the outputs are then incomplete)  */
     MOR_ERR_STATIC_SCRATCH = 7 /* mor_analyze_quantize_static: the tensor needs more scratch than
                                   the built-in array holds                                    */
 } mor_status_t;
@@ -136,7 +137,7 @@ typedef struct mor_outputs {
     uint8_t* codes;         /* [rows, codes_ld] FP8 codes, 16-byte aligned.  E4M3 codes
                                everywhere except in blocks that selected E5M2; blocks that
                                selected BF16 still hold their E4M3 codes.  Bytes in columns
-                               cols..roundup(cols,16)-1 of each row are overwritten with 0   */
+                               cols..codes_ld-1 of each row are left untouched               */
     int64_t  codes_ld;      /* bytes between row starts; >= roundup(cols,16); multiple of 16 */
     uint8_t* scale_e8m0;    /* [n_blocks] biased binary32 exponent of the selected format's
                                scale.  The scale is bits((e << 23) | group_mantissa); the
@@ -152,8 +153,8 @@ typedef struct mor_outputs {
     mor_tensor_stats_t* tensor_stats; /* required                                            */
 } mor_outputs_t;
 
-/* Bytes of DEVICE scratch the calls below need for these `n` descriptors (partial sums per
- * tile and one amax slot per tensor).  Only shapes and block shapes are read.  Returns 0 on
+/* Bytes of DEVICE scratch the calls below need for these `n` descriptors (one partial result per
+ * 128 x 128 tile, one amax slot and one counter per tensor, one status word).  Only shapes and block shapes are read.  Returns 0 on
  * a NULL or negative argument.  The scratch needs no initialisation and 256-byte alignment. */
 size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n);
 
