@@ -48,7 +48,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (266.4 MB for 100.66 M elements; traffic grows in proportion to the elements) and scaled to the
 # 16 tensors of the default batch.  The write part is an undercount: codes still in L2 when the
 # kernel ends have not reached DRAM yet.  Must be set back to None when the kernel changes.
-MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH = 710.5e6
+MAIN_KERNEL_DRAM_BYTES_PER_LAUNCH = None
 
 
 def measured_peak():

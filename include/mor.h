@@ -154,7 +154,8 @@ typedef struct mor_outputs {
 } mor_outputs_t;
 
 /* Bytes of DEVICE scratch the calls below need for these `n` descriptors (one partial result per
- * 128 x 128 tile, one amax slot and one counter per tensor, one status word).  Only shapes and block shapes are read.  Returns 0 on
+ * 128 x 128 tile, block keys handed from the amax pre-pass to the main kernel, one amax slot and
+ * one counter per tensor, one status word).  Only shapes and block shapes are read.  Returns 0 on
  * a NULL or negative argument.  The scratch needs no initialisation and 256-byte alignment. */
 size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n);
 
@@ -215,15 +216,16 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
  * comes from an array of MOR_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU
  * that loads the library holds that much memory until the process exits.  The call makes no
  * cudaMalloc / cudaFree and uses no allocating library routine.
- *   - Limit: mor_workspace_bytes(host_desc, 1) must not exceed MOR_STATIC_SCRATCH_BYTES (512 KiB:
- *     about 13,000 tiles of 128 x 128 elements, i.e. tensors up to roughly 214 M elements);
- *     larger tensors are refused with MOR_ERR_STATIC_SCRATCH and nothing is launched.
+ *   - Limit: mor_workspace_bytes(host_desc, 1) must not exceed MOR_STATIC_SCRATCH_BYTES (2 MiB).
+ *     The scratch holds 56 bytes per 128 x 128 tile, and 552 with the (1,128) partition (one key
+ *     per block), so the limit is roughly 600 M elements, or 62 M elements for (1,128); larger
+ *     tensors are refused with MOR_ERR_STATIC_SCRATCH and nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.
  *   - All calls share the one array, and it keeps what the previous call left in it; the call
  *     clears the part that has to start at zero.  Two calls whose kernels overlap on the GPU
  *     (different streams, no ordering between them) race on it: order them.  */
-#define MOR_STATIC_SCRATCH_BYTES (512 * 1024)
+#define MOR_STATIC_SCRATCH_BYTES (2 * 1024 * 1024)
 mor_status_t mor_analyze_quantize_static(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                          void* cuda_stream);
 

@@ -27,7 +27,7 @@ LIB_PATH = os.path.join(_HERE, "libmor_b200.so")
 MOR_OK = 0
 (MOR_ERR_INVALID_ARG, MOR_ERR_UNSUPPORTED, MOR_ERR_ALIGNMENT, MOR_ERR_WORKSPACE, MOR_ERR_CUDA,
  MOR_ERR_TIMEOUT, MOR_ERR_STATIC_SCRATCH) = range(1, 8)
-MOR_STATIC_SCRATCH_BYTES = 512 * 1024
+MOR_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 MOR_FMT_E4M3, MOR_FMT_E5M2, MOR_FMT_BF16 = 0, 1, 2
 MOR_SCALE_GAM, MOR_SCALE_E8M0, MOR_SCALE_FP32_AMAX = 0, 1, 2
 MOR_CRIT_TENSOR_MEAN_REL, MOR_CRIT_BLOCK_VS_E5M2, MOR_CRIT_BLOCK_MEAN_REL = 0, 1, 2

@@ -15,7 +15,8 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 struct Shape {
     int kind;
-    uint32_t nbc, nbr, n_units, n_tiles, amax_tiles;
+    uint32_t nbc, nbr, n_units, n_tiles;
+    uint64_t key_words;      // words of block keys the pre-pass writes for the main kernel
     uint64_t n_blocks;
 };
 
@@ -34,7 +35,6 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     if (segs >= (1ull << 31) || nbc >= (1ull << 24)) return MOR_ERR_UNSUPPORTED;
     s.nbc = (uint32_t)nbc;
     s.nbr = (uint32_t)nbr;
-    s.amax_tiles = (uint32_t)((segs + kSegsPerTile - 1) / kSegsPerTile);
     s.n_tiles = (uint32_t)(nbr * nbc);       // the main kernel works on 128 x 128 tiles whatever the partition
     if (s.kind == KIND_BLK128) {
         s.n_units = s.n_tiles;
@@ -43,6 +43,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
+    s.key_words = (uint64_t)s.n_tiles * (s.kind == KIND_ROW128 ? (uint64_t)kTileRows : 4u);
     return MOR_OK;
 }
 
@@ -138,17 +139,18 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
 }
 
 struct Layout {
-    size_t amax_off, nonf_off, status_off, partial_off, total;
+    size_t amax_off, nonf_off, status_off, partial_off, keys_off, total;
 };
 
-Layout layout_of(int n, uint64_t tiles)
+Layout layout_of(int n, uint64_t tiles, uint64_t key_words)
 {
     Layout l;
     l.amax_off = 0;
     l.nonf_off = (size_t)n * sizeof(float);
     l.status_off = 2 * (size_t)n * sizeof(float);
     l.partial_off = round_up(l.status_off + sizeof(uint32_t), kAlign);
-    l.total = l.partial_off + round_up((size_t)tiles * sizeof(Partial), kAlign);
+    l.keys_off = l.partial_off + round_up((size_t)tiles * sizeof(Partial), kAlign);
+    l.total = l.keys_off + round_up((size_t)key_words * sizeof(uint32_t), kAlign);
     return l;
 }
 
@@ -158,6 +160,8 @@ struct Item {
     Shape s;
     MainVariant v;
     uint32_t tile_begin;
+    uint64_t key_begin;      // first word of the tensor's keys
+    bool prepass;            // the amax pre-pass runs for this tensor (and leaves keys)
     int index;
 };
 
@@ -176,6 +180,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
+    r.keys = it.prepass ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
+    r.key_stride = it.s.kind == KIND_ROW128 ? (uint32_t)kTileRows : 4u;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.tile_begin = it.tile_begin;
@@ -185,7 +191,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
 
 inline bool same_variant(const MainVariant& a, const MainVariant& b)
 {
-    return a.kind == b.kind && a.yard == b.yard && a.three == b.three && a.store == b.store;
+    return a.kind == b.kind && a.yard == b.yard && a.three == b.three && a.store == b.store && a.scan == b.scan;
 }
 
 // The launch sequence shared by every entry point.
@@ -197,9 +203,13 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     };
     const int n = (int)items.size();
     uint64_t tiles = 0;
-    for (Item& it : items) { it.tile_begin = (uint32_t)tiles; tiles += it.s.n_tiles; }
+    uint64_t key_words = 0;
+    for (Item& it : items) {
+        it.tile_begin = (uint32_t)tiles; tiles += it.s.n_tiles;
+        it.key_begin = key_words; key_words += it.s.key_words;
+    }
     if (tiles >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
-    const Layout l = layout_of(n, tiles);
+    const Layout l = layout_of(n, tiles, key_words);
     if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign)) return MOR_ERR_ALIGNMENT;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -221,11 +231,9 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         for (const Item& it : items) {
             // a supplied group amax only fixes the shared mantissa; the per-tensor partition still
             // needs its block amax, which is the tensor amax, from the data (Algorithm 1)
-            if ((it.d->group_amax && it.s.kind != KIND_TENSOR) || it.s.amax_tiles == 0) continue;
+            if (!it.prepass) continue;
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);
-            r.n_units = (uint32_t)((uint64_t)it.d->rows * it.s.nbc);   // row pieces, whatever the partition
-            r.n_tiles = it.s.amax_tiles;
             t_end += r.n_tiles;
             bp.tile_end[bp.n++] = t_end;
             if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
@@ -292,6 +300,10 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.three = d->n_formats == 3;
     it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
     it.v.store = store;
+    // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
+    // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
+    it.prepass = it.s.n_tiles != 0 && !(d->group_amax != nullptr && it.s.kind != KIND_TENSOR);
+    it.v.scan = !it.prepass;
     return MOR_OK;
 }
 
@@ -305,13 +317,14 @@ extern "C" {
 size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n)
 {
     if (host_descs == nullptr || n <= 0) return 0;
-    uint64_t tiles = 0;
+    uint64_t tiles = 0, key_words = 0;
     for (int i = 0; i < n; ++i) {
         Shape s;
         if (shape_of(host_descs[i], s) != MOR_OK) return 0;
         tiles += s.n_tiles;
+        key_words += s.key_words;
     }
-    return layout_of(n, tiles).total;
+    return layout_of(n, tiles, key_words).total;
 }
 
 mor_status_t mor_analyze_quantize_batched_ex(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
@@ -362,7 +375,7 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
     if (host_descs == nullptr || n < 0 || (n > 0 && amax_out == nullptr)) return MOR_ERR_INVALID_ARG;
     if (n == 0) return MOR_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const Layout l = layout_of(n, 0);
+    const Layout l = layout_of(n, 0, 0);
     if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign) || !aligned(amax_out, 4)) return MOR_ERR_ALIGNMENT;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
@@ -377,12 +390,10 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         mor_status_t st = check_desc(d, it.s);
         if (st != MOR_OK) return st;
         std::memset(&it.o, 0, sizeof(it.o));
-        it.d = &d; it.index = i; it.tile_begin = 0;
-        if (it.s.amax_tiles) {
+        it.d = &d; it.index = i; it.tile_begin = 0; it.key_begin = 0; it.prepass = false;   // no keys wanted
+        if (it.s.n_tiles) {
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);
-            r.n_units = (uint32_t)((uint64_t)d.rows * it.s.nbc);
-            r.n_tiles = it.s.amax_tiles;
             t_end += r.n_tiles;
             bp.tile_end[bp.n++] = t_end;
         }
@@ -415,7 +426,7 @@ bool staging_of(const mor_tensor_desc_t& d, int64_t codes_ld, Staging& g)
     g.sf32 = take((size_t)s.n_blocks * 4);
     g.bstats = take((size_t)s.n_blocks * sizeof(mor_block_stats_t));
     g.tstats = take(sizeof(mor_tensor_stats_t));
-    g.ws_bytes = layout_of(1, s.n_tiles).total;
+    g.ws_bytes = layout_of(1, s.n_tiles, s.key_words).total;
     g.ws = take(g.ws_bytes);
     g.total = off;
     return true;

@@ -14,8 +14,7 @@ namespace mor {
 // The main kernel works on tiles of 128 rows x 128 columns (32 KiB of BF16), whatever the
 // partition: a tile is one 128x128 block, or 128 one-row blocks of 128 elements, or a piece of
 // the single block of the per-tensor partition.  Tiles are numbered row-major over the tile
-// grid [ceil(rows/128), ceil(cols/128)].  The amax pre-pass has its own tiling: 128
-// consecutive 128-element row pieces per CTA.
+// grid [ceil(rows/128), ceil(cols/128)].  The amax pre-pass uses the same tiles.
 constexpr int kTileRows = 128;
 constexpr int kTileCols = 128;
 constexpr int kSegsPerTile = 128;
@@ -48,6 +47,8 @@ struct TensorRec {
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
+    uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
+    uint32_t key_stride;          // words per tile in `keys`: 128 (one key per row piece) or 4 (one per tile)
     int64_t rows, cols, ld, codes_ld;
     uint32_t nbc;                 // tile columns = ceil(cols / 128)
     uint32_t nbr;                 // tile rows = ceil(rows / 128)
@@ -80,6 +81,7 @@ struct MainVariant {
     bool yard;       // evaluate E5M2 as well (Eq. 3, or statistics asked for)
     bool three;      // three-way recipe: keep E5M2 codes and the non-zero minimum (Eq. 4)
     bool store;      // write codes (false for mor_select_stats)
+    bool scan;       // the kernel scans the data for amax / smallest non-zero itself (no keys from the pre-pass)
 };
 
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);

@@ -61,19 +61,6 @@ __device__ __forceinline__ int find_tensor(const BatchParams& p, uint32_t tile, 
     return ti;
 }
 
-// Where row piece `s` of pre-pass tile `local` lives: the pieces are the 128-element pieces of
-// the rows in row-major order.
-__device__ __forceinline__ void piece_geometry(const TensorRec& R, uint32_t local, int s, long long& off, int& n)
-{
-    const uint32_t u = local * (uint32_t)kSegsPerTile + (uint32_t)s;
-    const uint32_t r = u / R.nbc;
-    const long long c0 = (long long)(u - r * R.nbc) * kSegElems;
-    const bool valid = u < R.n_units;
-    const long long left = R.cols - c0;
-    n = valid ? (int)(left < kSegElems ? left : kSegElems) : 0;
-    off = valid ? (long long)r * R.ld + c0 : 0;
-}
-
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll
@@ -88,68 +75,137 @@ __device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
 
 // ------------------------------------------------------------------ amax pre-pass ----
 
-// One tile of 128 row pieces per CTA; 16-byte loads straight to registers.  The packed BF16
-// maximum lets NaN and inf through; a thread that meets one rescans its registers with a
-// filter and counts them.
-__global__ void __launch_bounds__(kThreads)
-mor_amax_kernel(const __grid_constant__ BatchParams p, float* __restrict__ amax_slots_unused)
+// Key of 8 elements (four packed BF16 pairs): amax bits << 16 | 0xFFFF - (smallest non-zero bits - 1),
+// so that keys combine with a packed 16-bit maximum.  NaN and inf compare above every finite pattern.
+__device__ __forceinline__ uint32_t key_of_chunk(uint4 v)
 {
-    (void)amax_slots_unused;
-    __shared__ long long s_off[kSegsPerTile];
-    __shared__ int s_n[kSegsPerTile];
-    __shared__ uint32_t s_wmax[kThreads / 32], s_wnf[kThreads / 32];
+    const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+    const uint32_t mx = __vimax3_u16x2(__vimax3_u16x2(a0, a1, a2), a3, a3);
+    uint32_t mn = __viaddmin_u16x2(a0, 0xFFFFFFFFu, 0xFFFFFFFFu);
+    mn = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn);
+    mn = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn);
+    mn = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn);
+    return (max(mx & 0xFFFFu, mx >> 16) << 16) | (0xFFFFu - min(mn & 0xFFFFu, mn >> 16));
+}
+// the same over finite elements only, with the count of the others (a real call: rare path)
+__device__ __noinline__ uint2 key_of_chunk_finite(uint4 v)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t m = 0u, n = 0xFFFFu, nf = 0u;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
+        if (lo < kBf16Inf) { m = max(m, lo); n = min(n, (lo - 1u) & 0xFFFFu); } else nf++;
+        if (hi < kBf16Inf) { m = max(m, hi); n = min(n, (hi - 1u) & 0xFFFFu); } else nf++;
+    }
+    return make_uint2((m << 16) | (0xFFFFu - n), nf);
+}
+__device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
+
+// One 128 x 128 tile per CTA (the tiling of the main kernel); 16-byte loads straight to registers,
+// 16 lanes per 256-byte row piece.  Results: the tensor's amax (Algorithm 1, "g_amax <- max(abs(g))"
+// with the tensor as one group) by atomicMax, the count of NaN/inf elements, and, when the tensor
+// record has a key array, the key of every row piece of the tile (1x128 partition: that is the
+// block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main
+// kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its elements (the key itself
+// covers the finite ones only).
+__global__ void __launch_bounds__(kThreads)
+mor_amax_kernel(const __grid_constant__ BatchParams p)
+{
+    __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32];
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     uint32_t local;
     const TensorRec& R = p.t[find_tensor(p, blockIdx.x, local)];
-    if (t < kSegsPerTile) piece_geometry(R, local, t, s_off[t], s_n[t]);
-    __syncthreads();
+    const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
+    const long long row0 = (long long)bi * kTileRows, col0 = (long long)bj * kTileCols;
 
     uint4 v[8];
     const int k = t & 15;
+    const long long first = row0 + (t >> 4);
+    const uint16_t* src = R.x + first * R.ld + col0 + 8 * k;
+    const long long step = 16 * R.ld;
+    if (row0 + kTileRows <= R.rows && col0 + kTileCols <= R.cols) {
+        // a tile inside the tensor: eight 16-byte loads, 16 rows apart
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int seg = (t >> 4) + 16 * j;
-        const int left = s_n[seg] - 8 * k;
-        v[j] = make_uint4(0u, 0u, 0u, 0u);
-        if (left >= 8) {
-            v[j] = *reinterpret_cast<const uint4*>(R.x + s_off[seg] + 8 * k);
-        } else if (left > 0) {
-            const uint16_t* src = R.x + s_off[seg] + 8 * k;
-            uint16_t e[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            for (int i = 0; i < left; ++i) e[i] = src[i];
-            v[j] = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
-                              e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
-        }
-    }
-    __nv_bfloat162 m = __float2bfloat162_rn(0.0f);
+        for (int j = 0; j < 8; ++j, src += step) v[j] = *reinterpret_cast<const uint4*>(src);
+    } else {
+        const long long left = R.cols - col0 - 8 * k;       // elements of this thread's 16-byte chunk inside the tensor
+        const int nrows = (int)((R.rows - first + 15) >> 4); // this thread's rows (first, first + 16, ...) inside the tensor
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m = __hmax2_nan(m, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
-    }
-    const uint32_t mb = *reinterpret_cast<const uint32_t*>(&m);
-    uint32_t amax = max(mb & 0xFFFFu, mb >> 16), nf = 0;
-    if (amax >= kBf16Inf) {
-        amax = 0;
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
-            for (int i = 0; i < 4; ++i) {
-                const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
-                if (lo < kBf16Inf) amax = max(amax, lo); else nf++;
-                if (hi < kBf16Inf) amax = max(amax, hi); else nf++;
+        for (int j = 0; j < 8; ++j, src += step) {
+            v[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (j < nrows) {
+                if (left >= 8) {
+                    v[j] = *reinterpret_cast<const uint4*>(src);
+                } else if (left > 0) {
+                    uint16_t e[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    for (int i = 0; i < (int)left; ++i) e[i] = src[i];
+                    v[j] = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
+                                      e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
+                }
             }
         }
     }
-    amax = __reduce_max_sync(0xFFFFFFFFu, amax);
+    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kTileRows;
+    uint32_t key[8], all = 0u, nf = 0u;
+    if (per_piece) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { key[j] = key_of_chunk(v[j]); all = key_max(all, key[j]); }
+    } else {
+        // one key for the thread's 64 elements: packed halves are folded once at the end
+        uint32_t mx = 0u, mn[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
+            mx = __vimax3_u16x2(__vimax3_u16x2(mx, a0, a1), a2, a3);
+            mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
+            mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
+            mn[0] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn[0]);
+            mn[1] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn[1]);
+            key[j] = 0u;
+        }
+        const uint32_t m2 = __vimin3_u16x2(mn[0], mn[1], mn[1]);
+        all = (max(mx & 0xFFFFu, mx >> 16) << 16) | (0xFFFFu - min(m2 & 0xFFFFu, m2 >> 16));
+    }
+    // NaN or inf somewhere in the warp's data: redo the keys over finite elements and count the others
+    const bool warp_nf = __any_sync(0xFFFFFFFFu, (all >> 16) >= kBf16Inf);
+    uint32_t nf_piece = 0u;                                  // bit j: this thread saw NaN/inf in its chunk of piece j
+    if (warp_nf) {
+        all = 0u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint2 r = key_of_chunk_finite(v[j]);
+            key[j] = r.x;
+            all = key_max(all, r.x);
+            nf += r.y;
+            nf_piece |= (r.y ? 1u : 0u) << j;
+        }
+    }
+    if (per_piece) {
+        // one key per row piece: combine the 16 lanes that share the piece
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            uint32_t kk = key[j];
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) kk = key_max(kk, __shfl_xor_sync(0xFFFFFFFFu, kk, o));
+            if (warp_nf) {
+                const uint32_t b = __ballot_sync(0xFFFFFFFFu, (nf_piece >> j) & 1u);
+                if ((b >> (lane & 16)) & 0xFFFFu) kk |= 0x80000000u;
+            }
+            if (k == 0) R.keys[(size_t)local * kTileRows + (t >> 4) + 16 * j] = kk;
+        }
+    }
+    const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
-    if (lane == 0) { s_wmax[warp] = amax; s_wnf[warp] = nf; }
+    if (lane == 0) { s_wkey[warp] = (hi << 16) | lo; s_wnf[warp] = nf; }
     __syncthreads();
     if (t == 0) {
-        for (int i = 1; i < kThreads / 32; ++i) { amax = max(amax, s_wmax[i]); nf += s_wnf[i]; }
+        uint32_t kk = s_wkey[0];
+        for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; }
+        if (R.keys != nullptr && R.key_stride != (uint32_t)kTileRows) R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
         // non-negative binary32 patterns order like the values
-        atomicMax(reinterpret_cast<unsigned int*>(R.amax_slot), amax << 16);
+        atomicMax(reinterpret_cast<unsigned int*>(R.amax_slot), (kk >> 16) << 16);
         if (nf) atomicAdd(R.nonfinite_slot, nf);
     }
 }
@@ -261,7 +317,7 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s)
 {
     if (total_tiles == 0) return cudaSuccess;
-    mor_amax_kernel<<<total_tiles, kThreads, 0, s>>>(p, nullptr);
+    mor_amax_kernel<<<total_tiles, kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -70,6 +70,7 @@ struct Control {
     unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
     unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
     TileMeta meta[kStages];
+    uint32_t keys[kStages][kTileRows];                   // block keys of the tile from the pre-pass (arrive with the tile)
     Entry entry[2][kThreads];
     uint32_t wmax[2][2][kComputeWarps];                  // BLK128: per tile parity, per pass: warp amax | inverted min
     uint32_t tile_scale[2][2];                           // BLK128: scale bits (E4M3, E5M2) of the tile
@@ -132,6 +133,12 @@ __device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map,
 {
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                  ::"r"(smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
+}
+// plain bulk copy global -> shared (16-byte aligned, size a multiple of 16), completing on the same mbarrier
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, void* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 __device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, int x, int y, const void* src)
 {
@@ -607,8 +614,11 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
     m.pad = 0;
     C.meta[s] = m;
-    mbar_arrive_expect_tx(&C.full[s], kInBytes);
+    const TensorRec& R = p.b.t[t.ti];
+    const uint32_t key_bytes = R.keys != nullptr ? R.key_stride * 4u : 0u;
+    mbar_arrive_expect_tx(&C.full[s], kInBytes + key_bytes);
     tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
+    if (key_bytes) bulk_load(&C.keys[s][0], R.keys + (size_t)t.local * R.key_stride, key_bytes, &C.full[s]);
     C.issued = it + 1;
 }
 
@@ -748,7 +758,7 @@ __device__ __forceinline__ void write_fallback(const TensorRec& R, const uint32_
     }
 }
 
-template <int KIND, bool YARD, bool THREE, bool STORE>
+template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
 __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
 {
     const int lane = tid & 31, warp = tid >> 5;
@@ -767,7 +777,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     int scale_mode = 0;
     bool has_fallback = false;
     uint32_t tensor_amax_bits = 0;
-    const uint32_t meta_base = smem_addr(&C.meta[0]);
+    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
@@ -809,12 +819,21 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
             m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z;
         }
+        uint32_t key = 0u;
+        if (!SCAN) {
+            // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (KIND == KIND_ROW128 ? (uint32_t)row * 4u : 0u)));
+        }
         stage_free_arrive(s);                           // this thread's copy of the stage is in registers
 
         // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
-        uint32_t key = scan_words(w);
         bool nonfin = false;
-        if (KIND == KIND_ROW128) {
+        if (!SCAN) {
+            nonfin = (key >> 31) != 0u;
+            key &= 0x7FFFFFFFu;
+            if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);
+        } else if (KIND == KIND_ROW128) {
+            key = scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
             if (nonfin) {
@@ -822,6 +841,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             }
         } else if (KIND == KIND_BLK128) {
+            key = scan_words(w);
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
                 const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, key >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, key & 0xFFFFu);
@@ -836,6 +856,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = scan_words_finite(w);
             }
         } else {
+            key = scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
             if (nonfin) key = scan_words_finite(w);
         }
@@ -931,7 +952,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
 
 // ------------------------------------------------------------------ kernel ----
 
-template <int KIND, bool YARD, bool THREE, bool STORE>
+template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
 __global__ void __launch_bounds__(kMainThreads, 2)
 mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ partials)
 {
@@ -958,15 +979,15 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     if (tid < 128) C.rtab[tid] = __float_as_uint(__fdiv_rn(448.0f, 1.0f + (float)tid * 0.0078125f));
     __syncthreads();
 
-    if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE>(p, C, in, out, tid);
+    if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE, SCAN>(p, C, in, out, tid);
     else if (warp == kLoadWarp) load_warp(p, C, in, lane);
     else store_warp<KIND, THREE, STORE>(p, C, out, partials, lane);
 }
 
-template <int KIND, bool YARD, bool THREE, bool STORE>
+template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
 cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
 {
-    auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE>;
+    auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE, SCAN>;
     static bool configured[64] = {};   // per instantiation and device
     static int sm_count[64] = {};
     int dev = 0;
@@ -986,19 +1007,25 @@ cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s
     return cudaGetLastError();
 }
 
+template <int KIND, bool SCAN>
+cudaError_t launch_main_ks(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
+{
+    if (v.three) {
+        return v.store ? launch_main_t<KIND, true, true, true, SCAN>(p, partials, s)
+                       : launch_main_t<KIND, true, true, false, SCAN>(p, partials, s);
+    }
+    if (v.yard) {
+        return v.store ? launch_main_t<KIND, true, false, true, SCAN>(p, partials, s)
+                       : launch_main_t<KIND, true, false, false, SCAN>(p, partials, s);
+    }
+    return v.store ? launch_main_t<KIND, false, false, true, SCAN>(p, partials, s)
+                   : launch_main_t<KIND, false, false, false, SCAN>(p, partials, s);
+}
+
 template <int KIND>
 cudaError_t launch_main_k(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
 {
-    if (v.three) {
-        return v.store ? launch_main_t<KIND, true, true, true>(p, partials, s)
-                       : launch_main_t<KIND, true, true, false>(p, partials, s);
-    }
-    if (v.yard) {
-        return v.store ? launch_main_t<KIND, true, false, true>(p, partials, s)
-                       : launch_main_t<KIND, true, false, false>(p, partials, s);
-    }
-    return v.store ? launch_main_t<KIND, false, false, true>(p, partials, s)
-                   : launch_main_t<KIND, false, false, false>(p, partials, s);
+    return v.scan ? launch_main_ks<KIND, true>(v, p, partials, s) : launch_main_ks<KIND, false>(v, p, partials, s);
 }
 
 }  // namespace

@@ -5,8 +5,8 @@
 // inside somebody else's runtime that owns all device memory, a real-time loop in which an
 // allocation's implicit device synchronisation is not acceptable, a process whose memory
 // budget was fixed at start-up.  Such a caller still owns its inputs and outputs; only the
-// scratch (one amax slot, one counter and one 40-byte partial result per 32 KiB tile of input)
-// comes from here.
+// scratch (an amax slot and a counter, then per 32 KiB tile of input one 40-byte partial result and
+// the block keys that the amax pre-pass hands to the main kernel) comes from here.
 #include <mutex>
 
 #include "mor_internal.h"

@@ -61,7 +61,7 @@ def test_static_scratch_refuses_tensors_beyond_its_limit():
     import torch
 
     r = mb.Recipe((128, 128), TWO)
-    rows = cols = 128 * 120                                              # 14,400 tiles * 40 B > 512 KiB
+    rows = cols = 128 * 200                                              # 40,000 tiles * 56 B > 2 MiB
     d = mb.make_desc(0x10000, rows, cols, cols, r)
     assert mb.mor_workspace_bytes([d]) > mb.MOR_STATIC_SCRATCH_BYTES
     o = mb.mor_outputs_t()
