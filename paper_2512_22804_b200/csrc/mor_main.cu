@@ -657,25 +657,36 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const uint32_t tile = blockIdx.x + it * gridDim.x;
         if (tile >= p.total_tiles) break;
         const uint32_t b = it & 1u, n = it >> 1;
+        const TileId t = locate_tile(p.b, tile);        // before the wait: off the critical path
+        const TensorRec& R = p.b.t[t.ti];
+        const bool need_dec = KIND == KIND_BLK128 && (THREE || (STORE && R.fallback != nullptr));
+        const bool codes_wait = STORE && KIND == KIND_BLK128 && THREE;
         out_full_sync(b);                                // sleeps until every compute thread has arrived
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
-            const TileId t = locate_tile(p.b, tile);
-            const TensorRec& R = p.b.t[t.ti];
+            if (STORE && !codes_wait && lane == 0) {
+                // the codes are complete: start the tile store at once, it runs while the sums are formed
+                tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
+                bulk_commit();
+                stores_pending = true;
+            }
 
-            // the threads' sums in a fixed order: lane-strided, then a butterfly
-            double s43 = 0.0, s52 = 0.0;
+            // the threads' sums in a fixed order: lane-strided in binary32, then a butterfly in double
+            float f43 = 0.0f, f52 = 0.0f;
             uint32_t nnz = 0, nonf = 0, n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
 #pragma unroll
             for (int k = 0; k < kEntries / 32; ++k) {
                 const Entry e = C.entry[b][lane + 32 * k];
-                s43 += (double)e.e43;
-                s52 += (double)e.e52;
+                f43 += e.e43;
+                f52 += e.e52;
                 nnz += e.nnz_nonf & 0xFFFFu;
                 nonf += e.nnz_nonf >> 16;
-                const uint32_t sel = e.sel_min & 0xFFFFu;
-                n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
+                if (KIND == KIND_ROW128) {
+                    const uint32_t sel = e.sel_min & 0xFFFFu;
+                    n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
+                }
                 mn = min(mn, e.sel_min >> 16);
             }
+            double s43 = (double)f43, s52 = (double)f52;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
             nnz = __reduce_add_sync(0xFFFFFFFFu, nnz);
@@ -685,16 +696,14 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
                 n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
                 nb = __reduce_add_sync(0xFFFFFFFFu, nb);
-            } else {
-                n4 = n5 = nb = 0;
             }
 
-            const bool need_dec = KIND == KIND_BLK128 && (THREE || (STORE && R.fallback != nullptr));
             if (lane == 0) {
                 if (KIND == KIND_BLK128) {
                     const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
                     const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
                     const uint32_t bsel = decide_block(R, s43, s52, nnz, nonf, amax_bits, minm1, (uint32_t)(t.vrows * t.vcols));
+                    if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }   // first: compute threads may be waiting
                     const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
                     if (R.sel) R.sel[t.local] = (uint8_t)bsel;
                     if (R.scale_e8m0) R.scale_e8m0[t.local] = (uint8_t)(sb >> 23);
@@ -708,28 +717,25 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                         R.block_stats[t.local] = bs;
                     }
                     n4 = bsel == MOR_FMT_E4M3; n5 = bsel == MOR_FMT_E5M2; nb = bsel == MOR_FMT_BF16;
-                    if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }
                 }
                 Partial P;
                 P.sum43 = s43; P.sum52 = s52; P.nnz = nnz; P.nonfinite = nonf;
                 P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
                 partials[R.tile_begin + t.local] = P;
             }
-            if (STORE) {
-                bool ok = true;
-                if (KIND == KIND_BLK128 && THREE) {
-                    // the compute threads put the chosen format's codes in place after the decision
-                    ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok && lane == 0) give_up(C, p.device_status);
-                }
+            if (codes_wait) {
+                // three formats, 128x128 blocks: the compute threads put the chosen format's codes in place
+                // after the decision
+                bool ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok && lane == 0) give_up(C, p.device_status);
                 if (ok && lane == 0) {
                     tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
                     bulk_commit();
                     stores_pending = true;
-                    bulk_wait_read<0>();      // the staging buffer may be overwritten from here on
                 }
             }
+            if (STORE && lane == 0 && stores_pending) bulk_wait_read<0>();   // the staging buffer may be overwritten from here on
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&C.out_empty[b]);
