@@ -88,8 +88,9 @@ typedef struct mor_tensor_desc {
     int64_t rows, cols;     /* >= 0; an empty tensor is valid                                */
     int64_t ld;             /* elements between row starts; >= cols; multiple of 8           */
     int32_t block_rows;     /* partition: (0,0) whole tensor, (1,128) sub-channel rows,      */
-    int32_t block_cols;     /*            (128,128) 2-D blocks.  Edge blocks may overhang:
-                                           missing elements take part in nothing             */
+    int32_t block_cols;     /*            (128,128) or (64,64) 2-D blocks (Section 4.1.2 runs
+                                           the smaller size as an ablation).  Edge blocks may
+                                           overhang: missing elements take part in nothing   */
     int32_t n_formats;      /* 2 or 3                                                        */
     int32_t formats[3];     /* {E4M3,BF16} or {E4M3,E5M2,BF16}, in this order                */
     int32_t criterion;      /* mor_criterion_t; three formats need BLOCK_VS_E5M2             */

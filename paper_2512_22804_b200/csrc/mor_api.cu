@@ -27,6 +27,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     if (d.block_rows == 0 && d.block_cols == 0) s.kind = KIND_TENSOR;
     else if (d.block_rows == 1 && d.block_cols == 128) s.kind = KIND_ROW128;
     else if (d.block_rows == 128 && d.block_cols == 128) s.kind = KIND_BLK128;
+    else if (d.block_rows == 64 && d.block_cols == 64) s.kind = KIND_BLK64;
     else return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     const uint64_t nbc = empty ? 0 : (uint64_t)(d.cols + 127) / 128;
@@ -39,6 +40,11 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     if (s.kind == KIND_BLK128) {
         s.n_units = s.n_tiles;
         s.n_blocks = s.n_units;
+    } else if (s.kind == KIND_BLK64) {
+        const uint64_t nb = empty ? 0 : ((uint64_t)(d.rows + 63) / 64) * ((uint64_t)(d.cols + 63) / 64);
+        if (nb >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
+        s.n_units = (uint32_t)nb;
+        s.n_blocks = nb;
     } else {
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
@@ -184,6 +190,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.key_stride = it.s.kind == KIND_ROW128 ? (uint32_t)kTileRows : 4u;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
+    r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
     r.tile_begin = it.tile_begin;
     r.criterion = d.criterion; r.scale_mode = d.scale_mode; r.n_formats = d.n_formats;
     r.flags = d.flags; r.threshold = d.threshold;

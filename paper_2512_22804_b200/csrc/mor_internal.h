@@ -12,8 +12,8 @@
 namespace mor {
 
 // The main kernel works on tiles of 128 rows x 128 columns (32 KiB of BF16), whatever the
-// partition: a tile is one 128x128 block, or 128 one-row blocks of 128 elements, or a piece of
-// the single block of the per-tensor partition.  Tiles are numbered row-major over the tile
+// partition: a tile is one 128x128 block, or four 64x64 blocks, or 128 one-row blocks of 128
+// elements, or a piece of the single block of the per-tensor partition.  Tiles are numbered row-major over the tile
 // grid [ceil(rows/128), ceil(cols/128)].  The amax pre-pass uses the same tiles.
 constexpr int kTileRows = 128;
 constexpr int kTileCols = 128;
@@ -23,7 +23,7 @@ constexpr int kThreads = 256;          // amax and finalise kernels; compute thr
 constexpr int kMainThreads = 320;      // 8 compute warps + load warp + store warp
 constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor maps travel as kernel parameters
 
-enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2 };
+enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3 };
 
 // Per-tile partial results, reduced in tile order by the finalise kernel.
 struct Partial {
@@ -48,10 +48,13 @@ struct TensorRec {
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
-    uint32_t key_stride;          // words per tile in `keys`: 128 (one key per row piece) or 4 (one per tile)
+    uint32_t key_stride;          // words per tile in `keys`: 128 (one key per row piece) or 4 (one per tile, or one
+                                  // per 64x64 quadrant in the order top-left, top-right, bottom-left, bottom-right)
     int64_t rows, cols, ld, codes_ld;
     uint32_t nbc;                 // tile columns = ceil(cols / 128)
     uint32_t nbr;                 // tile rows = ceil(rows / 128)
+    uint32_t nbc_blk;             // KIND_BLK64: block columns = ceil(cols / 64)
+    int32_t kind;                 // Kind
     uint32_t n_units;             // blocks of the partition (KIND_TENSOR: row pieces, used by the pre-pass)
     uint32_t n_tiles;
     uint32_t tile_begin;          // index of the tensor's first Partial

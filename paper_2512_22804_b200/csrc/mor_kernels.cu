@@ -113,6 +113,7 @@ __global__ void __launch_bounds__(kThreads)
 mor_amax_kernel(const __grid_constant__ BatchParams p)
 {
     __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32];
+    __shared__ uint32_t s_qkey[kThreads / 32][4], s_qnf[kThreads / 32][4];   // 64x64 blocks: per warp and quadrant
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     uint32_t local;
@@ -196,6 +197,30 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             if (k == 0) R.keys[(size_t)local * kTileRows + (t >> 4) + 16 * j] = kk;
         }
     }
+    if (R.keys != nullptr && R.kind == KIND_BLK64) {
+        // one key per 64x64 quadrant: this thread's chunk lies in column half (k >> 3); its first four rows
+        // are in the upper half of the tile, the other four in the lower half
+        uint32_t kq[2], nq[2] = {0u, 0u};
+        if (warp_nf) {
+            kq[0] = key_max(key_max(key[0], key[1]), key_max(key[2], key[3]));
+            kq[1] = key_max(key_max(key[4], key[5]), key_max(key[6], key[7]));
+            nq[0] = nf_piece & 0xFu; nq[1] = nf_piece >> 4;
+        } else {
+            kq[0] = key_max(key_max(key_of_chunk(v[0]), key_of_chunk(v[1])), key_max(key_of_chunk(v[2]), key_of_chunk(v[3])));
+            kq[1] = key_max(key_max(key_of_chunk(v[4]), key_of_chunk(v[5])), key_max(key_of_chunk(v[6]), key_of_chunk(v[7])));
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            // lanes with the same (lane >> 3) & 1 share a column half
+#pragma unroll
+            for (int o = 1; o <= 16; o <<= 1) {
+                if (o == 8) continue;
+                kq[r] = key_max(kq[r], __shfl_xor_sync(0xFFFFFFFFu, kq[r], o));
+                nq[r] |= __shfl_xor_sync(0xFFFFFFFFu, nq[r], o);
+            }
+            if ((lane & 7) == 0 && lane < 16) { s_qkey[warp][2 * r + (lane >> 3)] = kq[r]; s_qnf[warp][2 * r + (lane >> 3)] = nq[r]; }
+        }
+    }
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
     if (lane == 0) { s_wkey[warp] = (hi << 16) | lo; s_wnf[warp] = nf; }
@@ -203,7 +228,15 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     if (t == 0) {
         uint32_t kk = s_wkey[0];
         for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; }
-        if (R.keys != nullptr && R.key_stride != (uint32_t)kTileRows) R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
+        if (R.keys != nullptr && R.kind == KIND_BLK64) {
+            for (int q = 0; q < 4; ++q) {
+                uint32_t kq = s_qkey[0][q], nq = s_qnf[0][q];
+                for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, s_qkey[i][q]); nq |= s_qnf[i][q]; }
+                R.keys[(size_t)local * 4 + q] = kq | (nq ? 0x80000000u : 0u);
+            }
+        } else if (R.keys != nullptr && R.key_stride != (uint32_t)kTileRows) {
+            R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
+        }
         // non-negative binary32 patterns order like the values
         atomicMax(reinterpret_cast<unsigned int*>(R.amax_slot), (kk >> 16) << 16);
         if (nf) atomicAdd(R.nonfinite_slot, nf);
@@ -333,6 +366,7 @@ cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int k
         case KIND_TENSOR: mor_finalise_kernel<KIND_TENSOR><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_ROW128: mor_finalise_kernel<KIND_ROW128><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_BLK128: mor_finalise_kernel<KIND_BLK128><<<grid, kThreads, 0, s>>>(p, partials); break;
+        case KIND_BLK64: mor_finalise_kernel<KIND_BLK64><<<grid, kThreads, 0, s>>>(p, partials); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

@@ -72,10 +72,11 @@ struct Control {
     TileMeta meta[kStages];
     uint32_t keys[kStages][kTileRows];                   // block keys of the tile from the pre-pass (arrive with the tile)
     Entry entry[2][kThreads];
-    uint32_t wmax[2][2][kComputeWarps];                  // BLK128: per tile parity, per pass: warp amax | inverted min
-    uint32_t tile_scale[2][2];                           // BLK128: scale bits (E4M3, E5M2) of the tile
-    uint32_t tile_key[2];                                // BLK128: amax bits << 16 | 0xFFFF - (min - 1)
-    uint32_t dec_sel[2];
+    // 128x128 and 64x64 blocks (a tile holds one block, or four: index q = 2 * (row >= 64) + (column >= 64))
+    uint32_t wmax[2][2][2 * kComputeWarps];              // per tile parity, per pass: warp (and column half) amax | inverted min
+    uint32_t tile_scale[2][4][2];                        // scale bits (E4M3, E5M2) of the tile's blocks
+    uint32_t tile_key[2][4];                             // amax bits << 16 | 0xFFFF - (min - 1)
+    uint32_t dec_sel[2][4];
     uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
     uint32_t issued;                                     // tile loads issued so far by this CTA
     volatile uint32_t abort;
@@ -659,8 +660,9 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const uint32_t b = it & 1u, n = it >> 1;
         const TileId t = locate_tile(p.b, tile);        // before the wait: off the critical path
         const TensorRec& R = p.b.t[t.ti];
-        const bool need_dec = KIND == KIND_BLK128 && (THREE || (STORE && R.fallback != nullptr));
-        const bool codes_wait = STORE && KIND == KIND_BLK128 && THREE;
+        constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
+        const bool need_dec = kTileBlocks && (THREE || (STORE && R.fallback != nullptr));
+        const bool codes_wait = STORE && kTileBlocks && THREE;
         out_full_sync(b);                                // sleeps until every compute thread has arrived
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
             if (STORE && !codes_wait && lane == 0) {
@@ -670,27 +672,39 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 stores_pending = true;
             }
 
-            // the threads' sums in a fixed order: lane-strided in binary32, then a butterfly in double
-            float f43 = 0.0f, f52 = 0.0f;
-            uint32_t nnz = 0, nonf = 0, n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
+            // the threads' sums in a fixed order: lane-strided in binary32, then a butterfly in double.
+            // With 64x64 blocks a lane's entries belong to one column half (lane & 1) and to the upper
+            // (k < 4) or lower rows: two sets of sums per lane, combined over the lanes of equal parity.
+            constexpr int NR = KIND == KIND_BLK64 ? 2 : 1;
+            float f43[NR], f52[NR];
+            uint32_t nnz[NR], nonf[NR], n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
+#pragma unroll
+            for (int r = 0; r < NR; ++r) { f43[r] = 0.0f; f52[r] = 0.0f; nnz[r] = 0; nonf[r] = 0; }
 #pragma unroll
             for (int k = 0; k < kEntries / 32; ++k) {
                 const Entry e = C.entry[b][lane + 32 * k];
-                f43 += e.e43;
-                f52 += e.e52;
-                nnz += e.nnz_nonf & 0xFFFFu;
-                nonf += e.nnz_nonf >> 16;
+                const int r = (NR == 2 && k >= 4) ? 1 : 0;
+                f43[r] += e.e43;
+                f52[r] += e.e52;
+                nnz[r] += e.nnz_nonf & 0xFFFFu;
+                nonf[r] += e.nnz_nonf >> 16;
                 if (KIND == KIND_ROW128) {
                     const uint32_t sel = e.sel_min & 0xFFFFu;
                     n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
                 }
                 mn = min(mn, e.sel_min >> 16);
             }
-            double s43 = (double)f43, s52 = (double)f52;
+            double s43[NR], s52[NR];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
-            nnz = __reduce_add_sync(0xFFFFFFFFu, nnz);
-            nonf = __reduce_add_sync(0xFFFFFFFFu, nonf);
+            for (int r = 0; r < NR; ++r) {
+                s43[r] = (double)f43[r]; s52[r] = (double)f52[r];
+#pragma unroll
+                for (int o = 16; o > (NR == 2 ? 1 : 0); o >>= 1) {
+                    s43[r] += shfl_xor_f64(s43[r], o); s52[r] += shfl_xor_f64(s52[r], o);
+                    if (NR == 2) { nnz[r] += __shfl_xor_sync(0xFFFFFFFFu, nnz[r], o); nonf[r] += __shfl_xor_sync(0xFFFFFFFFu, nonf[r], o); }
+                }
+                if (NR == 1) { nnz[r] = __reduce_add_sync(0xFFFFFFFFu, nnz[r]); nonf[r] = __reduce_add_sync(0xFFFFFFFFu, nonf[r]); }
+            }
             mn = __reduce_min_sync(0xFFFFFFFFu, mn);
             if (KIND == KIND_ROW128) {
                 n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
@@ -698,28 +712,58 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 nb = __reduce_add_sync(0xFFFFFFFFu, nb);
             }
 
-            if (lane == 0) {
-                if (KIND == KIND_BLK128) {
-                    const uint32_t key = C.tile_key[b], s4b = C.tile_scale[b][0], s5b = C.tile_scale[b][1];
-                    const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
-                    const uint32_t bsel = decide_block(R, s43, s52, nnz, nonf, amax_bits, minm1, (uint32_t)(t.vrows * t.vcols));
-                    if (need_dec) { C.dec_sel[b] = bsel; mbar_arrive(&C.dec_full[b]); }   // first: compute threads may be waiting
-                    const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
-                    if (R.sel) R.sel[t.local] = (uint8_t)bsel;
-                    if (R.scale_e8m0) R.scale_e8m0[t.local] = (uint8_t)(sb >> 23);
-                    if (R.scale_f32) R.scale_f32[t.local] = __uint_as_float(sb);
-                    if (R.block_stats) {
-                        mor_block_stats_t bs;
-                        bs.amax = __uint_as_float(amax_bits << 16);
-                        bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                        bs.nnz = nnz; bs.n_nonfinite = nonf;
-                        bs.sum_rel_e4m3 = (float)s43; bs.sum_rel_e5m2 = (float)s52;
-                        R.block_stats[t.local] = bs;
+            // tile totals (64x64: the four blocks in the order q = 0..3, taken from lanes 0 and 1)
+            double t43 = s43[0], t52 = s52[0];
+            uint32_t tnnz = nnz[0], tnonf = nonf[0];
+            if (NR == 2) {
+                const double a1 = __shfl_sync(0xFFFFFFFFu, s43[0], 1), b1 = __shfl_sync(0xFFFFFFFFu, s52[0], 1);
+                const double a3 = __shfl_sync(0xFFFFFFFFu, s43[NR - 1], 1), b3 = __shfl_sync(0xFFFFFFFFu, s52[NR - 1], 1);
+                t43 = ((s43[0] + a1) + s43[NR - 1]) + a3;
+                t52 = ((s52[0] + b1) + s52[NR - 1]) + b3;
+                tnnz = nnz[0] + nnz[NR - 1]; tnnz += __shfl_xor_sync(0xFFFFFFFFu, tnnz, 1);
+                tnonf = nonf[0] + nonf[NR - 1]; tnonf += __shfl_xor_sync(0xFFFFFFFFu, tnonf, 1);
+            }
+
+            if (kTileBlocks && lane < (NR == 2 ? 2 : 1)) {
+                // Algorithm 2 for the tile's block(s): lane 0 decides block(s) of the left column half, lane 1 of the right
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    const int q = NR == 2 ? 2 * r + lane : 0;
+                    const int br = NR == 2 ? 64 : 128;
+                    const int vr = min(br, t.vrows - (NR == 2 ? 64 * r : 0)), vc = min(br, t.vcols - (NR == 2 ? 64 * lane : 0));
+                    uint32_t bsel = kSelNone;
+                    if (vr > 0 && vc > 0) {
+                        const uint32_t key = C.tile_key[b][q], s4b = C.tile_scale[b][q][0], s5b = C.tile_scale[b][q][1];
+                        const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
+                        bsel = decide_block(R, s43[r], s52[r], nnz[r], nonf[r], amax_bits, minm1, (uint32_t)(vr * vc));
+                        const uint32_t blk = NR == 2 ? (uint32_t)(t.row0 / 64 + r) * R.nbc_blk + (uint32_t)(t.col0 / 64 + lane) : t.local;
+                        const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
+                        if (R.sel) R.sel[blk] = (uint8_t)bsel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
+                        if (R.block_stats) {
+                            mor_block_stats_t bs;
+                            bs.amax = __uint_as_float(amax_bits << 16);
+                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                            bs.nnz = nnz[r]; bs.n_nonfinite = nonf[r];
+                            bs.sum_rel_e4m3 = (float)s43[r]; bs.sum_rel_e5m2 = (float)s52[r];
+                            R.block_stats[blk] = bs;
+                        }
                     }
-                    n4 = bsel == MOR_FMT_E4M3; n5 = bsel == MOR_FMT_E5M2; nb = bsel == MOR_FMT_BF16;
+                    if (need_dec) C.dec_sel[b][q] = bsel;
+                    n4 += bsel == MOR_FMT_E4M3; n5 += bsel == MOR_FMT_E5M2; nb += bsel == MOR_FMT_BF16;
                 }
+            }
+            if (NR == 2) {
+                n4 += __shfl_xor_sync(0xFFFFFFFFu, n4, 1); n5 += __shfl_xor_sync(0xFFFFFFFFu, n5, 1); nb += __shfl_xor_sync(0xFFFFFFFFu, nb, 1);
+            }
+            if (need_dec) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&C.dec_full[b]);      // compute threads may be waiting for the decision
+            }
+            if (lane == 0) {
                 Partial P;
-                P.sum43 = s43; P.sum52 = s52; P.nnz = nnz; P.nonfinite = nonf;
+                P.sum43 = t43; P.sum52 = t52; P.nnz = tnnz; P.nonfinite = tnonf;
                 P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
                 partials[R.tile_begin + t.local] = P;
             }
@@ -773,6 +817,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     // this choice the 8 threads of a 128-bit load phase and the 16 threads of a 64-bit store phase
     // touch distinct banks.
     const int swz = (row & 7) ^ (h << 2);
+    const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
     const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
     const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
     const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
@@ -828,7 +873,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         uint32_t key = 0u;
         if (!SCAN) {
             // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (KIND == KIND_ROW128 ? (uint32_t)row * 4u : 0u)));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (KIND == KIND_ROW128 ? (uint32_t)row * 4u : (uint32_t)q * 4u)));
         }
         stage_free_arrive(s);                           // this thread's copy of the stage is in registers
 
@@ -837,7 +882,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         if (!SCAN) {
             nonfin = (key >> 31) != 0u;
             key &= 0x7FFFFFFFu;
-            if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);
+            if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);   // warp-uniform (a tile-wide key is CTA-uniform already)
         } else if (KIND == KIND_ROW128) {
             key = scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
@@ -846,17 +891,32 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = scan_words_finite(w);
                 key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             }
-        } else if (KIND == KIND_BLK128) {
+        } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
             key = scan_words(w);
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
-                const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, key >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, key & 0xFFFFu);
-                if (lane == 0) C.wmax[b][pass][warp] = (hi << 16) | lo;
+                // the warps exchange their keys; with 64x64 blocks a warp has one per column half (lane parity)
+                const uint32_t part = KIND == KIND_BLK64 ? (h ? 0xAAAAAAAAu : 0x55555555u) : 0xFFFFFFFFu;
+                const uint32_t hi = __reduce_max_sync(part, key >> 16), lo = __reduce_max_sync(part, key & 0xFFFFu);
+                if (KIND == KIND_BLK64) { if (lane < 2) C.wmax[b][pass][2 * warp + h] = (hi << 16) | lo; }
+                else if (lane == 0) C.wmax[b][pass][warp] = (hi << 16) | lo;
                 dead = compute_bar_or(dead);                                       // also spreads the word that a wait ran out
-                const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]);
-                const uint4 k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
-                key = key_max(key_max(__vimax3_u16x2(k0.x, k0.y, k0.z), k0.w), key_max(__vimax3_u16x2(k1.x, k1.y, k1.z), k1.w));
-                nonfin = pass == 1 || (key >> 16) >= kBf16Inf;                     // CTA-uniform
+                uint32_t any;                                                      // the largest key of the tile: CTA-uniform
+                if (KIND == KIND_BLK64) {
+                    const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]), k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
+                    const uint4 k2 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][8]), k3 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][12]);
+                    // entries 2 * warp + h: warps 0-3 hold the upper rows, 4-7 the lower
+                    const uint32_t u0 = __vimax3_u16x2(k0.x, k0.z, key_max(k1.x, k1.z)), u1 = __vimax3_u16x2(k0.y, k0.w, key_max(k1.y, k1.w));
+                    const uint32_t l0 = __vimax3_u16x2(k2.x, k2.z, key_max(k3.x, k3.z)), l1 = __vimax3_u16x2(k2.y, k2.w, key_max(k3.y, k3.w));
+                    key = (row >> 6) ? (h ? l1 : l0) : (h ? u1 : u0);
+                    any = key_max(key_max(u0, u1), key_max(l0, l1));
+                } else {
+                    const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]);
+                    const uint4 k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
+                    key = key_max(key_max(__vimax3_u16x2(k0.x, k0.y, k0.z), k0.w), key_max(__vimax3_u16x2(k1.x, k1.y, k1.z), k1.w));
+                    any = key;
+                }
+                nonfin = pass == 1 || (any >> 16) >= kBf16Inf;                     // CTA-uniform
                 if (dead) { key = 0u; nonfin = false; }
                 if (pass == 1 || !nonfin) break;
                 key = scan_words_finite(w);
@@ -927,15 +987,15 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             } else {
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
-                if (KIND == KIND_BLK128 && tid == 0) {
-                    C.tile_scale[b][0] = s4b; C.tile_scale[b][1] = s5b; C.tile_key[b] = key;
+                if ((KIND == KIND_BLK128 && tid == 0) || (KIND == KIND_BLK64 && (row & 63) == 0)) {
+                    C.tile_scale[b][q][0] = s4b; C.tile_scale[b][q][1] = s5b; C.tile_key[b][q] = key;
                 }
             }
             if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
         }
         out_full_arrive(b);
 
-        if (KIND == KIND_BLK128) {
+        if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
             const bool need_dec = THREE || has_fallback;
             if (need_dec) {
                 if (!dead) {
@@ -943,7 +1003,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
                 }
-                if (!dead) sel = C.dec_sel[b];
+                if (!dead) sel = C.dec_sel[b][q];
                 if (THREE && STORE) {
                     if (!dead && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
                     fence_async_smem();
@@ -1043,6 +1103,7 @@ cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* part
         case KIND_TENSOR: return launch_main_k<KIND_TENSOR>(v, p, partials, s);
         case KIND_ROW128: return launch_main_k<KIND_ROW128>(v, p, partials, s);
         case KIND_BLK128: return launch_main_k<KIND_BLK128>(v, p, partials, s);
+        case KIND_BLK64: return launch_main_k<KIND_BLK64>(v, p, partials, s);
     }
     return cudaErrorInvalidValue;
 }

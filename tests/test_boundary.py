@@ -50,7 +50,7 @@ def test_workspace_bytes(lib):
     assert both >= big
     assert mb.mor_workspace_bytes([desc(0, 128)]) > 0                     # empty tensors still get their slots
     assert lib.mor_workspace_bytes(None, 1) == 0
-    assert mb.mor_workspace_bytes([desc(128, 128, block=(64, 64))]) == 0  # unsupported block shape
+    assert mb.mor_workspace_bytes([desc(128, 128, block=(32, 32))]) == 0  # unsupported block shape
 
 
 def out_struct(codes=0x2000, codes_ld=256, ts=0x3000):
@@ -61,7 +61,7 @@ def out_struct(codes=0x2000, codes_ld=256, ts=0x3000):
 
 
 @pytest.mark.parametrize("d,o,want", [
-    (desc(block=(64, 64)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
+    (desc(block=(32, 32)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
     (desc(block=(128, 1)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
     (desc(formats=(1, 0, 2)), out_struct(), mb.MOR_ERR_UNSUPPORTED),       # order is fixed: E4M3 first
     (desc(formats=(0, 1)), out_struct(), mb.MOR_ERR_UNSUPPORTED),

@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 
 TWO = (mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16)
 THREE = (mb.MOR_FMT_E4M3, mb.MOR_FMT_E5M2, mb.MOR_FMT_BF16)
-KINDS = [(0, 0), (1, 128), (128, 128)]
+KINDS = [(0, 0), (1, 128), (128, 128), (64, 64)]
 
 
 def recipe(block, formats=TWO, criterion=mb.MOR_CRIT_BLOCK_VS_E5M2, threshold=0.045, scale_mode=mb.MOR_SCALE_GAM, flags=0):
@@ -39,7 +39,7 @@ def test_every_partition_with_every_criterion(block, crit):
     parity.run_and_compare(g, recipe(block, TWO, crit, threshold=0.2))
 
 
-@pytest.mark.parametrize("block", [(1, 128), (128, 128)])
+@pytest.mark.parametrize("block", [(1, 128), (128, 128), (64, 64)])
 @pytest.mark.parametrize("flags", [0, mb.MOR_FLAG_STRICT_TIES, mb.MOR_FLAG_RANGE_MIN_INCLUDES_ZERO,
                                    mb.MOR_FLAG_STRICT_TIES | mb.MOR_FLAG_RANGE_MIN_INCLUDES_ZERO])
 def test_three_way_with_flags(block, flags):
@@ -121,6 +121,16 @@ def test_nonfinite_inputs(block):
     fm = THREE if block != (0, 0) else TWO
     parity.run_and_compare(x, recipe(block, fm))
     parity.run_and_compare(x, recipe(block, TWO, mb.MOR_CRIT_TENSOR_MEAN_REL))
+    # with the group amax supplied the main kernel finds the block amax itself (no keys from the pre-pass)
+    parity.run_and_compare(x, recipe(block, fm), group_amax_supplied=True)
+
+
+@pytest.mark.parametrize("block", KINDS)
+def test_supplied_group_amax_on_ragged_gradient_data(block):
+    g = wl.gradient_like(300, 1000, seed=47)
+    fm = THREE if block != (0, 0) else TWO
+    rep = parity.run_and_compare(g, recipe(block, fm), group_amax_supplied=True, pad_to=1008)
+    assert rep.n_exempt <= 2
 
 
 # ------------------------------------------------------------ the cast itself, exhaustively
@@ -137,7 +147,7 @@ def test_every_bf16_pattern_through_the_cast(amax_bits):
         b = bits.copy()
         if clean:
             b[(b & 0x7F80) == 0x7F80] = 0
-        for block, fm in (((0, 0), TWO), ((1, 128), THREE), ((128, 128), THREE)):
+        for block, fm in (((0, 0), TWO), ((1, 128), THREE), ((128, 128), THREE), ((64, 64), THREE)):
             r = recipe(block, fm)
             ref = orc.run(b, r.block, list(r.formats), r.criterion, r.threshold, group_amax=amax)
             ga = torch.tensor([amax], dtype=torch.float32, device="cuda")
@@ -165,7 +175,7 @@ def test_select_stats_matches_analyze_quantize():
 
     g = wl.gradient_like(256, 1024, seed=53)
     x = parity.to_device(g)
-    for block in [(1, 128), (128, 128)]:
+    for block in [(1, 128), (128, 128), (64, 64)]:
         r = recipe(block, THREE)
         a = mb.analyze_quantize(x, r, block_stats=True)
         s = mb.select_stats(x, r)
@@ -183,7 +193,7 @@ def test_bf16_fallback_copies_only_rejected_blocks():
     g = np.concatenate([wl.gradient_like(150, 1000, seed=54), wl.weight_like(150, 1000, seed=57)])
     host = np.zeros((300, 1008), dtype=np.uint16); host[:, :1000] = g
     x = parity.to_device(host)
-    for block in [(1, 128), (128, 128)]:
+    for block in [(1, 128), (128, 128), (64, 64)]:
         r = recipe(block, THREE)
         out = mb.analyze_quantize(x, r, cols=1000, fallback=True)
         torch.cuda.synchronize()
@@ -225,7 +235,7 @@ def test_many_tensors_exceeding_one_launch():
     rng = np.random.default_rng(60)
     bits = [wl.weight_like(int(rng.integers(1, 300)), int(rng.integers(1, 40)) * 8, seed=61 + i) for i in range(47)]
     xs = [parity.to_device(b) for b in bits]
-    recipes = [recipe(KINDS[i % 3]) for i in range(47)]
+    recipes = [recipe(KINDS[i % 4]) for i in range(47)]
     plan = mb.BatchPlan(xs, recipes)
     plan.run()
     torch.cuda.synchronize()
@@ -282,7 +292,7 @@ def test_invalid_arguments_launch_nothing():
 
     x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(mb.MorError) as e:
-        mb.analyze_quantize(x, recipe((64, 64)))
+        mb.analyze_quantize(x, recipe((32, 32)))
     assert e.value.status == mb.MOR_ERR_UNSUPPORTED
     with pytest.raises(mb.MorError) as e:
         mb.analyze_quantize(x, recipe((1, 128), (mb.MOR_FMT_E5M2, mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16)))
