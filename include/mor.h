@@ -89,8 +89,11 @@ typedef struct mor_tensor_desc {
     int64_t ld;             /* elements between row starts; >= cols; multiple of 8           */
     int32_t block_rows;     /* partition: (0,0) whole tensor, (1,128) sub-channel rows,      */
     int32_t block_cols;     /*            (128,128) or (64,64) 2-D blocks (Section 4.1.2 runs
-                                           the smaller size as an ablation).  Edge blocks may
-                                           overhang: missing elements take part in nothing   */
+                                           the smaller size as an ablation), (1,0) per channel:
+                                           one block per row (Section 3; the paper's most
+                                           FP8-efficient partition), with the tensor-level
+                                           criterion only.  Edge blocks may overhang: missing
+                                           elements take part in nothing                     */
     int32_t n_formats;      /* 2 or 3                                                        */
     int32_t formats[3];     /* {E4M3,BF16} or {E4M3,E5M2,BF16}, in this order                */
     int32_t criterion;      /* mor_criterion_t; three formats need BLOCK_VS_E5M2             */
@@ -150,7 +153,7 @@ typedef struct mor_outputs {
                                block that selected BF16 (other blocks are left untouched).
                                NULL = the fallback is the input itself.  Per-block criteria
                                only                                                          */
-    mor_block_stats_t*  block_stats;  /* [n_blocks] optional                                 */
+    mor_block_stats_t*  block_stats;  /* [n_blocks] optional; not with the (1,0) partition   */
     mor_tensor_stats_t* tensor_stats; /* required                                            */
 } mor_outputs_t;
 

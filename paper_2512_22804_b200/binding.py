@@ -211,6 +211,8 @@ def grid_of(rows: int, cols: int, block) -> tuple:
         return (0, 0)
     if tuple(block) == (0, 0):
         return (1, 1)
+    if tuple(block) == (1, 0):          # per-channel: one block per row
+        return (rows, 1)
     return (-(-rows // block[0]), -(-cols // block[1]))
 
 

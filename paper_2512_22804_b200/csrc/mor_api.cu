@@ -28,6 +28,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     else if (d.block_rows == 1 && d.block_cols == 128) s.kind = KIND_ROW128;
     else if (d.block_rows == 128 && d.block_cols == 128) s.kind = KIND_BLK128;
     else if (d.block_rows == 64 && d.block_cols == 64) s.kind = KIND_BLK64;
+    else if (d.block_rows == 1 && d.block_cols == 0) s.kind = KIND_CHANNEL;
     else return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     const uint64_t nbc = empty ? 0 : (uint64_t)(d.cols + 127) / 128;
@@ -45,11 +46,15 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         if (nb >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
         s.n_units = (uint32_t)nb;
         s.n_blocks = nb;
+    } else if (s.kind == KIND_CHANNEL) {
+        s.n_units = empty ? 0u : (uint32_t)d.rows;
+        s.n_blocks = s.n_units;
     } else {
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
-    s.key_words = (uint64_t)s.n_tiles * (s.kind == KIND_ROW128 ? (uint64_t)kTileRows : 4u);
+    s.key_words = (uint64_t)s.n_tiles * ((s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL) ? (uint64_t)kTileRows : 4u);
+    if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows;      // + one key per row
     return MOR_OK;
 }
 
@@ -74,6 +79,9 @@ mor_status_t check_desc(const mor_tensor_desc_t& d, Shape& s)
         return MOR_ERR_INVALID_ARG;
     }
     if (d.criterion < MOR_CRIT_TENSOR_MEAN_REL || d.criterion > MOR_CRIT_BLOCK_MEAN_REL) return MOR_ERR_INVALID_ARG;
+    // per-channel blocks span many tiles: this build gives them the tensor-level decision only (the recipe the
+    // paper evaluates them with, Section 4.1)
+    if (s.kind == KIND_CHANNEL && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || d.n_formats != 2)) return MOR_ERR_UNSUPPORTED;
     if (d.scale_mode < MOR_SCALE_GAM || d.scale_mode > MOR_SCALE_FP32_AMAX) return MOR_ERR_INVALID_ARG;
     if (!(d.threshold >= 0.0f) || std::isinf(d.threshold)) return MOR_ERR_INVALID_ARG;
     if (d.flags & ~(uint32_t)(MOR_FLAG_STRICT_TIES | MOR_FLAG_RANGE_MIN_INCLUDES_ZERO)) return MOR_ERR_INVALID_ARG;
@@ -85,6 +93,7 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
 {
     if (o.tensor_stats == nullptr) return MOR_ERR_INVALID_ARG;
     if (!aligned(o.tensor_stats, 8) || !aligned(o.block_stats, 4) || !aligned(o.scale_f32, 4)) return MOR_ERR_ALIGNMENT;
+    if (s.kind == KIND_CHANNEL && o.block_stats != nullptr) return MOR_ERR_UNSUPPORTED;   // would need sums across tiles
     const bool empty = d.rows == 0 || d.cols == 0;
     if (store) {
         if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
@@ -187,7 +196,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
     r.keys = it.prepass ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
-    r.key_stride = it.s.kind == KIND_ROW128 ? (uint32_t)kTileRows : 4u;
+    r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kTileRows : 4u;
+    r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kTileRows : nullptr;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
@@ -231,7 +241,10 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         uint32_t t_end = 0;
         auto flush = [&]() -> bool {
             if (bp.n == 0) return true;
-            const bool ok = launch_amax(bp, t_end, stream) == cudaSuccess;
+            bool ok = launch_amax(bp, t_end, stream) == cudaSuccess;
+            bool channel = false;
+            for (int k = 0; k < bp.n; ++k) channel = channel || bp.t[k].kind == KIND_CHANNEL;
+            if (ok && channel) ok = launch_row_keys(bp, stream) == cudaSuccess;
             bp.n = 0; t_end = 0;
             return ok;
         };
@@ -309,7 +322,7 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.store = store;
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
-    it.prepass = it.s.n_tiles != 0 && !(d->group_amax != nullptr && it.s.kind != KIND_TENSOR);
+    it.prepass = it.s.n_tiles != 0 && !(d->group_amax != nullptr && it.s.kind != KIND_TENSOR && it.s.kind != KIND_CHANNEL);
     it.v.scan = !it.prepass;
     return MOR_OK;
 }

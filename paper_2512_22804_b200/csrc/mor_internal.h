@@ -23,7 +23,7 @@ constexpr int kThreads = 256;          // amax and finalise kernels; compute thr
 constexpr int kMainThreads = 320;      // 8 compute warps + load warp + store warp
 constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor maps travel as kernel parameters
 
-enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3 };
+enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3, KIND_CHANNEL = 4 };
 
 // Per-tile partial results, reduced in tile order by the finalise kernel.
 struct Partial {
@@ -48,6 +48,7 @@ struct TensorRec {
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
+    uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows
     uint32_t key_stride;          // words per tile in `keys`: 128 (one key per row piece) or 4 (one per tile, or one
                                   // per 64x64 quadrant in the order top-left, top-right, bottom-left, bottom-right)
     int64_t rows, cols, ld, codes_ld;
@@ -88,6 +89,7 @@ struct MainVariant {
 };
 
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
+cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s);
 

@@ -243,6 +243,23 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     }
 }
 
+// Per-channel partition: a block is a whole row, so its key is the combination of the keys of the row's
+// 128-element pieces over all tiles of the tile row.  One CTA of 128 threads per (tile row, tensor).
+__global__ void __launch_bounds__(kTileRows)
+mor_row_keys_kernel(const __grid_constant__ BatchParams p)
+{
+    const TensorRec& R = p.t[blockIdx.y];
+    if (R.kind != KIND_CHANNEL || R.row_keys == nullptr || blockIdx.x >= R.nbr) return;
+    const uint32_t* src = R.keys + ((size_t)blockIdx.x * R.nbc) * kTileRows + threadIdx.x;
+    uint32_t k = 0u, flag = 0u;
+    for (uint32_t j = 0; j < R.nbc; ++j, src += kTileRows) {
+        const uint32_t v = *src;
+        flag |= v & 0x80000000u;
+        k = key_max(k, v & 0x7FFFFFFFu);
+    }
+    R.row_keys[(size_t)blockIdx.x * kTileRows + threadIdx.x] = k | flag;
+}
+
 // ----------------------------------------------------------------------- finalise ----
 
 // One CTA per (tensor, slice).  Every slice repeats the reduction over the tensor's tile
@@ -354,6 +371,16 @@ cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t
     return cudaGetLastError();
 }
 
+cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s)
+{
+    uint32_t nbr = 0;
+    for (int i = 0; i < p.n; ++i)
+        if (p.t[i].kind == KIND_CHANNEL && p.t[i].nbr > nbr) nbr = p.t[i].nbr;
+    if (nbr == 0) return cudaSuccess;
+    mor_row_keys_kernel<<<dim3(nbr, (unsigned)p.n), kTileRows, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s)
 {
     if (p.n == 0) return cudaSuccess;
@@ -367,6 +394,7 @@ cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int k
         case KIND_ROW128: mor_finalise_kernel<KIND_ROW128><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_BLK128: mor_finalise_kernel<KIND_BLK128><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_BLK64: mor_finalise_kernel<KIND_BLK64><<<grid, kThreads, 0, s>>>(p, partials); break;
+        case KIND_CHANNEL: mor_finalise_kernel<KIND_CHANNEL><<<grid, kThreads, 0, s>>>(p, partials); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

@@ -613,13 +613,17 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     TileMeta m;
     m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
     m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
+    if (p.b.t[t.ti].kind == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
     m.pad = 0;
     C.meta[s] = m;
     const TensorRec& R = p.b.t[t.ti];
     const uint32_t key_bytes = R.keys != nullptr ? R.key_stride * 4u : 0u;
     mbar_arrive_expect_tx(&C.full[s], kInBytes + key_bytes);
     tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
-    if (key_bytes) bulk_load(&C.keys[s][0], R.keys + (size_t)t.local * R.key_stride, key_bytes, &C.full[s]);
+    if (key_bytes) {
+        const uint32_t* src = R.kind == KIND_CHANNEL ? R.row_keys + t.row0 : R.keys + (size_t)t.local * R.key_stride;
+        bulk_load(&C.keys[s][0], src, key_bytes, &C.full[s]);
+    }
     C.issued = it + 1;
 }
 
@@ -873,7 +877,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         uint32_t key = 0u;
         if (!SCAN) {
             // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (KIND == KIND_ROW128 ? (uint32_t)row * 4u : (uint32_t)q * 4u)));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + ((KIND == KIND_ROW128 || KIND == KIND_CHANNEL) ? (uint32_t)row * 4u : (uint32_t)q * 4u)));
         }
         stage_free_arrive(s);                           // this thread's copy of the stage is in registers
 
@@ -987,6 +991,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             } else {
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
+                if (KIND == KIND_CHANNEL && h == 0 && m.blk_base != 0xFFFFFFFFu && row < m.vrows) {
+                    // per-channel: the row's scale, written by the tile that holds the row's first columns
+                    const uint32_t blk = m.blk_base + (uint32_t)row;
+                    if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(s4b >> 23);
+                    if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(s4b);
+                }
                 if ((KIND == KIND_BLK128 && tid == 0) || (KIND == KIND_BLK64 && (row & 63) == 0)) {
                     C.tile_scale[b][q][0] = s4b; C.tile_scale[b][q][1] = s5b; C.tile_key[b][q] = key;
                 }
@@ -1104,6 +1114,8 @@ cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* part
         case KIND_ROW128: return launch_main_k<KIND_ROW128>(v, p, partials, s);
         case KIND_BLK128: return launch_main_k<KIND_BLK128>(v, p, partials, s);
         case KIND_BLK64: return launch_main_k<KIND_BLK64>(v, p, partials, s);
+        case KIND_CHANNEL:   // the row amax spans tiles: always taken from the pre-pass
+            return v.scan ? cudaErrorInvalidValue : launch_main_ks<KIND_CHANNEL, false>(v, p, partials, s);
     }
     return cudaErrorInvalidValue;
 }

@@ -59,6 +59,38 @@ def test_scale_modes(block, mode):
     parity.run_and_compare(x, recipe(block, TWO, scale_mode=mode))
 
 
+# ------------------------------------------------------------ per-channel partition (one block per row)
+
+@pytest.mark.parametrize("shape", [(256, 512), (130, 1000), (1, 128), (300, 72), (5, 2049)])
+@pytest.mark.parametrize("mode", [mb.MOR_SCALE_GAM, mb.MOR_SCALE_E8M0, mb.MOR_SCALE_FP32_AMAX])
+def test_per_channel_partition_with_the_tensor_level_decision(shape, mode):
+    x = wl.activation_like(shape[0], shape[1], n_outlier_cols=min(4, shape[1]), seed=48)
+    x[shape[0] // 2, :] = 0                                        # an all-zero channel
+    ld = (shape[1] + 7) // 8 * 8 + 8
+    for th in (0.045, 0.01):
+        r = recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL, threshold=th, scale_mode=mode)
+        rep = parity.run_and_compare(x, r, pad_to=ld, block_stats=False)
+        assert rep.n_blocks == shape[0]
+    if shape[0] > 3:
+        x[3, shape[1] // 2] = 0x7FC0                               # a NaN in one channel
+        parity.run_and_compare(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL, scale_mode=mode), pad_to=ld, block_stats=False)
+        parity.run_and_compare(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL, scale_mode=mode), pad_to=ld, block_stats=False,
+                               group_amax_supplied=True)
+
+
+def test_per_channel_partition_supports_the_tensor_level_recipe_only():
+    import torch
+
+    x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
+    for bad in (recipe((1, 0), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2), recipe((1, 0), THREE, mb.MOR_CRIT_BLOCK_VS_E5M2)):
+        with pytest.raises(mb.MorError) as e:
+            mb.analyze_quantize(x, bad)
+        assert e.value.status == mb.MOR_ERR_UNSUPPORTED
+    with pytest.raises(mb.MorError) as e:
+        mb.analyze_quantize(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), block_stats=True)
+    assert e.value.status == mb.MOR_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------ ragged, padded, tiny and empty shapes
 
 @pytest.mark.parametrize("block", KINDS)
