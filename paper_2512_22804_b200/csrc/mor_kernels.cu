@@ -185,6 +185,8 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     }
     if (per_piece) {
         // one key per row piece: combine the 16 lanes that share the piece
+        const uint32_t half = (lane & 16) ? 0xFFFF0000u : 0x0000FFFFu;
+        uint32_t* kp = R.keys + (size_t)local * kTileRows + (t >> 4);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t kk = key[j];
@@ -192,9 +194,9 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             for (int o = 8; o > 0; o >>= 1) kk = key_max(kk, __shfl_xor_sync(0xFFFFFFFFu, kk, o));
             if (warp_nf) {
                 const uint32_t b = __ballot_sync(0xFFFFFFFFu, (nf_piece >> j) & 1u);
-                if ((b >> (lane & 16)) & 0xFFFFu) kk |= 0x80000000u;
+                if (b & half) kk |= 0x80000000u;
             }
-            if (k == 0) R.keys[(size_t)local * kTileRows + (t >> 4) + 16 * j] = kk;
+            if (k == 0) kp[16 * j] = kk;
         }
     }
     if (R.keys != nullptr && R.kind == KIND_BLK64) {
