@@ -59,6 +59,24 @@ def test_scale_modes(block, mode):
     parity.run_and_compare(x, recipe(block, TWO, scale_mode=mode))
 
 
+@pytest.mark.parametrize("block", [(1, 128), (128, 128), (64, 64)])
+@pytest.mark.parametrize("formats", [TWO, THREE])
+def test_narrow_range_blocks_next_to_wide_range_blocks(block, formats):
+    """Narrow-range blocks (all non-zeros within E4M3's normal range after scaling) keep E4M3 by
+    construction (every element's E5M2 error is at least its E4M3 error there); they sit next to
+    wide-range blocks that go to E5M2 or BF16.  With and without block statistics, with and without
+    strict ties."""
+    rng = np.random.default_rng(49)
+    a = rng.uniform(0.5, 4.0, size=(384, 512)) * rng.choice([-1.0, 1.0], size=(384, 512))
+    a[:, 256:] = wl.bf16_bits_to_float(wl.gradient_like(384, 256, seed=50))      # wide-range half
+    a[5, 17] = 0.0
+    x = wl.to_bf16_bits(a)
+    for stats in (False, True):
+        for flags in (0, mb.MOR_FLAG_STRICT_TIES):
+            rep = parity.run_and_compare(x, recipe(block, formats, flags=flags), block_stats=stats)
+            assert rep.n_exempt <= 1
+
+
 # ------------------------------------------------------------ per-channel partition (one block per row)
 
 @pytest.mark.parametrize("shape", [(256, 512), (130, 1000), (1, 128), (300, 72), (5, 2049)])
