@@ -47,6 +47,12 @@
  *       paper fixes this case.
  *   R10 blocks that overhang the tensor edge are filled with absent elements, which take
  *       part in nothing.
+ *   R11 fake quantisation (Section 4: "quantise, dequantise, de-scale", BF16 out): the FP8
+ *       value divided by the scale in one binary32 division, then rounded to BF16 (nearest
+ *       even).  A block that stays in BF16, and any NaN/inf element, is copied unchanged.  Where
+ *       the decision is taken for the whole tensor (tensor-level criterion, per-tensor
+ *       partition) the E4M3 values are written and the caller keeps the input when the tensor
+ *       falls back.
  */
 #include <math.h>
 #include <stdint.h>
@@ -463,6 +469,43 @@ int orc_run(const orc_cfg_t* cfg, const uint16_t* x, uint8_t* codes, int64_t cod
             orc_tensor_t* tensor, int n_threads)
 {
     return orc_run_blocks(cfg, x, NULL, 0, codes, codes_ld, scale_e8m0, sel, scale_f32, blocks, tensor, n_threads);
+}
+
+/* ------------------------------------------------------------- fake quantisation --- */
+
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u = f32_bits(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x0040u);   /* NaN stays NaN */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* R11.  `sel` and `scale_f32` are the per-block results of orc_run (selected format and its
+ * scale).  out has the layout of x with leading dimension out_ld. */
+int orc_fake_quant(const orc_cfg_t* cfg, const uint16_t* x, const uint8_t* sel, const float* scale_f32,
+                   uint16_t* out, int64_t out_ld)
+{
+    build_tables();
+    int64_t nbr, nbc; grid_dims(cfg, &nbr, &nbc);
+    int whole = cfg->criterion == ORC_CRIT_TENSOR_MEAN_REL || (cfg->block_rows == 0 && cfg->block_cols == 0);
+    for (int64_t bi = 0; bi < nbr; ++bi)
+        for (int64_t bj = 0; bj < nbc; ++bj) {
+            int64_t r0, r1, c0, c1, id = bi * nbc + bj;
+            block_bounds(cfg, bi, bj, &r0, &r1, &c0, &c1);
+            int fmt = whole ? ORC_FMT_E4M3 : sel[id];
+            float s = scale_f32[id];
+            for (int64_t r = r0; r < r1; ++r)
+                for (int64_t c = c0; c < c1; ++c) {
+                    uint16_t h = x[r * cfg->ld + c];
+                    if (fmt == ORC_FMT_BF16 || bf16_is_nonfinite(h)) { out[r * out_ld + c] = h; continue; }
+                    float y = scale_value(orc_bf16_to_float(h), s);
+                    float q = fmt == ORC_FMT_E5M2 ? (float)orc_decode_e5m2(orc_encode_e5m2(y))
+                                                  : (float)orc_decode_e4m3(orc_encode_e4m3(y));
+                    out[r * out_ld + c] = f32_to_bf16_rne(q / s);      /* one binary32 division */
+                }
+        }
+    return 0;
 }
 
 /* Element-level helpers exported for the pins. */

@@ -95,6 +95,8 @@ def lib():
         L.orc_run_blocks.argtypes = [C.POINTER(Cfg), C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.POINTER(Tensor), C.c_int]
+        L.orc_fake_quant.restype = C.c_int
+        L.orc_fake_quant.argtypes = [C.POINTER(Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
         L.orc_scale_value.restype = C.c_float
         L.orc_scale_value.argtypes = [C.c_float, C.c_float]
         for n in ("orc_rel_err_e4m3", "orc_rel_err_e5m2"):
@@ -220,6 +222,21 @@ def run(bits: np.ndarray, block, formats, criterion, threshold=0.045, scale_mode
         raise ValueError(f"oracle rejected the recipe (rc={rc})")
     td = {k: getattr(t, k) for k, _ in Tensor._fields_}
     return Result(codes, scale[:nb], sel[:nb], sf32[:nb], blocks[:n], td, grid, ids_arr)
+
+
+def fake_quant(bits: np.ndarray, res: Result, block, formats, criterion, threshold=0.045, scale_mode=SCALE_GAM,
+               flags=0, cols=None) -> np.ndarray:
+    """BF16 bit patterns of the fake-quantised tensor (quantise, dequantise, de-scale) for a finished run."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    rows, ld_ = bits.shape
+    cols = ld_ if cols is None else cols
+    cfg = make_cfg(rows, cols, ld_, tuple(block), formats, criterion, threshold, scale_mode, flags, None)
+    out = np.zeros((rows, cols), dtype=np.uint16)
+    sel = np.ascontiguousarray(res.sel, dtype=np.uint8)
+    sf = np.ascontiguousarray(res.scale_f32, dtype=np.float32)
+    rc = lib().orc_fake_quant(C.byref(cfg), bits.ctypes.data, sel.ctypes.data, sf.ctypes.data, out.ctypes.data, cols)
+    assert rc == 0
+    return out
 
 
 def tensor_amax(bits: np.ndarray) -> float:
