@@ -155,6 +155,14 @@ typedef struct mor_outputs {
                                only                                                          */
     mor_block_stats_t*  block_stats;  /* [n_blocks] optional; not with the (1,0) partition   */
     mor_tensor_stats_t* tensor_stats; /* required                                            */
+    void*    fake_quant;    /* optional, BF16 [rows, ld] like x: the tensor after "quantise,
+                               dequantise, de-scale" (Section 4, the form the paper trains with).
+                               Per element: the FP8 value of the block's selected format divided
+                               by the block's scale (one binary32 division), rounded to BF16;
+                               blocks that stay in BF16 and NaN/inf elements are copied.  Where the
+                               decision is taken for the whole tensor (tensor-level criterion,
+                               (0,0) and (1,0) partitions) the E4M3 values are written: keep the
+                               input instead when tensor_format says BF16                        */
 } mor_outputs_t;
 
 /* Bytes of DEVICE scratch the calls below need for these `n` descriptors (one partial result per

@@ -64,7 +64,7 @@ class mor_tensor_stats_t(C.Structure):
 class mor_outputs_t(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("codes_ld", C.c_int64), ("scale_e8m0", C.c_void_p),
                 ("sel", C.c_void_p), ("scale_f32", C.c_void_p), ("bf16_fallback", C.c_void_p),
-                ("block_stats", C.c_void_p), ("tensor_stats", C.c_void_p)]
+                ("block_stats", C.c_void_p), ("tensor_stats", C.c_void_p), ("fake_quant", C.c_void_p)]
 
 
 class mor_stage_events_t(C.Structure):
@@ -249,6 +249,7 @@ class Outputs:
     sel: object = None            # uint8 [grid]
     scale_f32: object = None      # float32 [grid]
     bf16_fallback: object = None  # bfloat16, shaped like x
+    fake_quant: object = None     # bfloat16, shaped like x
     block_stats: object = None    # uint8 [n_blocks * 24]
     tensor_stats: object = None   # uint8 [80]
     cols: int = 0
@@ -267,7 +268,7 @@ class Outputs:
 
 
 def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, block_stats=False, fallback_like=None,
-                  scale_f32=False) -> Outputs:
+                  scale_f32=False, fake_quant_like=None) -> Outputs:
     import torch
 
     g = grid_of(rows, cols, recipe.block)
@@ -283,6 +284,8 @@ def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, b
         o.scale_f32 = torch.empty(g, dtype=torch.float32, device=device)
     if fallback_like is not None:
         o.bf16_fallback = torch.zeros_like(fallback_like)
+    if fake_quant_like is not None:
+        o.fake_quant = torch.zeros_like(fake_quant_like)
     if block_stats:
         o.block_stats = torch.empty((max(nb, 1) * BLOCK_STATS_DTYPE.itemsize,), **u8)
     o.tensor_stats = torch.empty((TENSOR_STATS_DTYPE.itemsize,), **u8)
@@ -293,6 +296,7 @@ def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, b
     s.sel = o.sel.data_ptr() if nb else None
     s.scale_f32 = o.scale_f32.data_ptr() if o.scale_f32 is not None and nb else None
     s.bf16_fallback = o.bf16_fallback.data_ptr() if o.bf16_fallback is not None else None
+    s.fake_quant = o.fake_quant.data_ptr() if o.fake_quant is not None else None
     s.block_stats = o.block_stats.data_ptr() if o.block_stats is not None else None
     s.tensor_stats = o.tensor_stats.data_ptr()
     return o
@@ -311,11 +315,11 @@ def _workspace(nbytes: int, device):
 
 
 def analyze_quantize(x, recipe: Recipe, *, cols=None, group_amax=None, block_stats=False, fallback=False,
-                     scale_f32=False, stream=None) -> Outputs:
+                     scale_f32=False, fake_quant=False, stream=None) -> Outputs:
     """Run mor_analyze_quantize on one BF16 CUDA tensor; allocates outputs and workspace."""
     d = desc_for(x, recipe, cols, group_amax)
     o = alloc_outputs(d.rows, d.cols, recipe, x.device, block_stats=block_stats,
-                      fallback_like=x if fallback else None, scale_f32=scale_f32)
+                      fallback_like=x if fallback else None, scale_f32=scale_f32, fake_quant_like=x if fake_quant else None)
     nbytes = mor_workspace_bytes([d])
     ws = _workspace(nbytes, x.device)
     st = mor_analyze_quantize(d, o.c_struct, ws.data_ptr(), ws.numel(), _stream_ptr(stream))

@@ -100,6 +100,7 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
         if (o.codes_ld < (int64_t)round_up((size_t)d.cols, 16)) return MOR_ERR_INVALID_ARG;
         if (o.codes_ld % 16 != 0 || !aligned(o.codes, 16)) return MOR_ERR_ALIGNMENT;
         if (d.scale_mode == MOR_SCALE_FP32_AMAX && o.scale_f32 == nullptr && s.n_blocks) return MOR_ERR_INVALID_ARG;
+        if (o.fake_quant && !aligned(o.fake_quant, 16)) return MOR_ERR_ALIGNMENT;
         if (o.bf16_fallback) {
             if (s.kind == KIND_TENSOR || d.criterion == MOR_CRIT_TENSOR_MEAN_REL) return MOR_ERR_UNSUPPORTED;
             if (!aligned(o.bf16_fallback, 16)) return MOR_ERR_ALIGNMENT;
@@ -189,6 +190,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.sel = it.o.sel;
     r.scale_f32 = it.o.scale_f32;
     r.fallback = static_cast<uint16_t*>(it.o.bf16_fallback);
+    r.fake_quant = static_cast<uint16_t*>(it.o.fake_quant);
     r.block_stats = it.o.block_stats;
     r.tensor_stats = it.o.tensor_stats;
     r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
@@ -467,6 +469,7 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
     if (host_desc == nullptr || host_out == nullptr) return MOR_ERR_INVALID_ARG;
     if (host_desc->group_amax != nullptr) return MOR_ERR_INVALID_ARG;
     if (host_out->bf16_fallback != nullptr) return MOR_ERR_UNSUPPORTED;   // the fallback is the caller's own host tensor
+    if (host_out->fake_quant != nullptr) return MOR_ERR_UNSUPPORTED;
     if (host_desc->rows < 0 || host_desc->cols < 0 || host_desc->ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t dev_codes_ld = (int64_t)round_up((size_t)host_desc->cols, 16);

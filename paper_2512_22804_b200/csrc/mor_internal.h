@@ -41,6 +41,7 @@ struct TensorRec {
     uint8_t* sel;
     float* scale_f32;
     uint16_t* fallback;
+    uint16_t* fake_quant;
     mor_block_stats_t* block_stats;
     mor_tensor_stats_t* tensor_stats;
     const float* amax;            // group amax on the device (workspace slot or the caller's)

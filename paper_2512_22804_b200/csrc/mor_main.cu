@@ -665,7 +665,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const TileId t = locate_tile(p.b, tile);        // before the wait: off the critical path
         const TensorRec& R = p.b.t[t.ti];
         constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
-        const bool need_dec = kTileBlocks && (THREE || (STORE && R.fallback != nullptr));
+        const bool need_dec = kTileBlocks && (THREE || (STORE && (R.fallback != nullptr || R.fake_quant != nullptr)));
         const bool codes_wait = STORE && kTileBlocks && THREE;
         out_full_sync(b);                                // sleeps until every compute thread has arrived
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
@@ -812,6 +812,53 @@ __device__ __forceinline__ void write_fallback(const TensorRec& R, const uint32_
     }
 }
 
+// Fake quantisation of a thread's 64 elements (Section 4: quantise, dequantise, de-scale; BF16 out): the FP8
+// value of format `fmt` divided by the scale in one binary32 division, rounded to BF16; a block that stays
+// in BF16 and NaN/inf elements are copied.  Straight from the registers, like the fallback copy.
+__device__ __noinline__ void fake_quant_chunk(uint4 v, uint32_t fmt, float s, uint32_t (&o)[4])
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t ww = w[i];
+        const float xlo = __uint_as_float(ww << 16), xhi = __uint_as_float(ww & 0xFFFF0000u);
+        const float ylo = __fmul_rn(xlo, s), yhi = __fmul_rn(xhi, s);
+        const uint32_t q = fmt == MOR_FMT_E5M2 ? e5m2x2_to_f16x2(cvt_e5m2x2(yhi, ylo)) : e4m3x2_to_f16x2(cvt_e4m3x2(yhi, ylo));
+        const float2 qf = __half22float2(*reinterpret_cast<const __half2*>(&q));
+        const float tlo = __fdiv_rn(qf.x, s), thi = __fdiv_rn(qf.y, s);
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(thi), "f"(tlo));
+        if ((ww & 0x7F80u) == 0x7F80u) r = (r & 0xFFFF0000u) | (ww & 0xFFFFu);             // NaN / inf: as they are
+        if ((ww & 0x7F800000u) == 0x7F800000u) r = (r & 0xFFFFu) | (ww & 0xFFFF0000u);
+        o[i] = r;
+    }
+}
+__device__ __forceinline__ void write_fake_quant(const TensorRec& R, const uint32_t (&w)[32], const TileMeta& m, int row, int h, int swz,
+                                                 uint32_t fmt, uint32_t s4b, uint32_t s5b)
+{
+    if (row >= m.vrows) return;
+    const float s = __uint_as_float(fmt == MOR_FMT_E5M2 ? s5b : s4b);
+    uint16_t* dst_row = R.fake_quant + (long long)(m.row0 + row) * R.ld + m.col0 + h * 64;
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) {
+        const int c = (j ^ swz) * 8;
+        const int left = m.vcols - (h * 64 + c);
+        if (left <= 0) continue;
+        // chunk j of the registers, selected without indexing them dynamically
+        uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+        for (int k = 1; k < 8; ++k)
+            if (j == k) v = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+        uint32_t o[4] = {v.x, v.y, v.z, v.w};
+        if (fmt != MOR_FMT_BF16) fake_quant_chunk(v, fmt, s, o);
+        if (left >= 8) {
+            *reinterpret_cast<uint4*>(dst_row + c) = make_uint4(o[0], o[1], o[2], o[3]);
+        } else {
+            for (int i = 0; i < left; ++i) dst_row[c + i] = (uint16_t)(o[i >> 1] >> (16 * (i & 1)));
+        }
+    }
+}
+
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
 __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
 {
@@ -831,6 +878,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     uint32_t m_g = 0;            // Algorithm 1, group part
     int scale_mode = 0;
     bool has_fallback = false;
+    bool has_fq = false, fq_e4m3 = false;   // fake-quantised output wanted; ... with E4M3 values whatever the block's selection
     uint32_t tensor_amax_bits = 0;
     const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
@@ -865,12 +913,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             cur_ti = m.ti;
             scale_mode = R.scale_mode;
             has_fallback = STORE && R.fallback != nullptr;
+            has_fq = STORE && R.fake_quant != nullptr;
+            fq_e4m3 = KIND == KIND_TENSOR || KIND == KIND_CHANNEL || R.criterion == MOR_CRIT_TENSOR_MEAN_REL;
             if (!dead) {
                 m_g = group_mantissa(*R.amax, scale_mode);
                 if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
             }
         }
-        if (has_fallback) {      // the copy of BF16 blocks needs the tile's position too
+        if (has_fallback || has_fq) {      // the BF16 outputs need the tile's position too
             const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
             m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z;
         }
@@ -988,9 +1038,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                     }
                 }
                 if (has_fallback && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                if (has_fq) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
             } else {
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
+                if ((KIND == KIND_TENSOR || KIND == KIND_CHANNEL) && has_fq)
+                    write_fake_quant(R, w, m, row, h, swz, (uint32_t)MOR_FMT_E4M3, s4b, s5b);
                 if (KIND == KIND_CHANNEL && h == 0 && m.blk_base != 0xFFFFFFFFu && row < m.vrows) {
                     // per-channel: the row's scale, written by the tile that holds the row's first columns
                     const uint32_t blk = m.blk_base + (uint32_t)row;
@@ -1006,7 +1059,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         out_full_arrive(b);
 
         if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
-            const bool need_dec = THREE || has_fallback;
+            const bool need_dec = THREE || has_fallback || has_fq;
             if (need_dec) {
                 if (!dead) {
                     bool ok = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
@@ -1021,6 +1074,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                     if (lane == 0) mbar_arrive(&C.codes_full[b]);
                 }
                 if (has_fallback && !dead && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                if (has_fq && !dead) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
             }
         }
     }

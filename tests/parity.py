@@ -139,7 +139,7 @@ def compare(bits: np.ndarray, recipe: mb.Recipe, out: "mb.Outputs", ref: "orc.Re
 
 
 def run_and_compare(bits: np.ndarray, recipe: mb.Recipe, *, cols=None, block_stats=True, scale_mode=None,
-                    group_amax_supplied=False, pad_to=None) -> Report:
+                    group_amax_supplied=False, pad_to=None, fake_quant=False) -> Report:
     """CUDA run + full oracle run on the same bytes, compared."""
     import torch
 
@@ -157,6 +157,25 @@ def run_and_compare(bits: np.ndarray, recipe: mb.Recipe, *, cols=None, block_sta
     if group_amax_supplied:
         ga = torch.tensor([ref.tensor["group_amax"]], dtype=torch.float32, device="cuda")
     out = mb.analyze_quantize(x, recipe, cols=cols, group_amax=ga, block_stats=block_stats,
-                              scale_f32=True)
+                              scale_f32=True, fake_quant=fake_quant)
     torch.cuda.synchronize()
-    return compare(host, recipe, out, ref, cols=cols)
+    rep = compare(host, recipe, out, ref, cols=cols)
+    if fake_quant:
+        # the fake-quantised tensor, bit for bit, outside blocks whose decision is within the tolerance band;
+        # padding columns must stay untouched (zero-initialised output)
+        c = host.shape[1] if cols is None else cols
+        ob = oracle_block(recipe.block, c)
+        want = orc.fake_quant(host, ref, ob, list(recipe.formats), recipe.criterion, recipe.threshold, recipe.scale_mode,
+                              recipe.flags, cols=cols)
+        got = out.fake_quant.view(torch.int16).cpu().numpy().view(np.uint16)
+        ex = exempt_blocks(ref, recipe)
+        if not ex.any():
+            np.testing.assert_array_equal(got[:, :c], want)
+        else:
+            br, bc = ob if tuple(recipe.block) != (0, 0) else host.shape
+            for b in np.nonzero(~ex)[0]:
+                bi, bj = divmod(int(b), ref.grid[1])
+                sl = (slice(bi * br, min((bi + 1) * br, host.shape[0])), slice(bj * bc, min((bj + 1) * bc, c)))
+                np.testing.assert_array_equal(got[sl], want[sl])
+        assert (got[:, c:] == 0).all()
+    return rep

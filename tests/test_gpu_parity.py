@@ -77,6 +77,23 @@ def test_narrow_range_blocks_next_to_wide_range_blocks(block, formats):
             assert rep.n_exempt <= 1
 
 
+# ------------------------------------------------------------ fake quantisation (Section 4)
+
+@pytest.mark.parametrize("block", KINDS + [(1, 0)])
+def test_fake_quant_output(block):
+    g = np.concatenate([wl.gradient_like(150, 1000, seed=58), wl.weight_like(170, 1000, seed=59)])
+    g[7, 13] = 0x7FC0
+    g[200, 999] = 0xFF80
+    whole = block in ((0, 0), (1, 0))
+    recipes = [recipe(block, TWO, mb.MOR_CRIT_TENSOR_MEAN_REL)]
+    if not whole:
+        recipes += [recipe(block, THREE), recipe(block, TWO), recipe(block, TWO, mb.MOR_CRIT_BLOCK_MEAN_REL, threshold=0.03),
+                    recipe(block, THREE, scale_mode=mb.MOR_SCALE_E8M0)]
+    for r in recipes:
+        parity.run_and_compare(g, r, pad_to=1008, block_stats=block != (1, 0), fake_quant=True)
+        parity.run_and_compare(g, r, pad_to=1008, block_stats=False, fake_quant=True, group_amax_supplied=True)
+
+
 # ------------------------------------------------------------ per-channel partition (one block per row)
 
 @pytest.mark.parametrize("shape", [(256, 512), (130, 1000), (1, 128), (300, 72), (5, 2049)])
