@@ -92,8 +92,11 @@ typedef struct mor_tensor_desc {
                                            the smaller size as an ablation), (1,0) per channel:
                                            one block per row (Section 3; the paper's most
                                            FP8-efficient partition), with the tensor-level
-                                           criterion only.  Edge blocks may overhang: missing
-                                           elements take part in nothing                     */
+                                           criterion only; (128,1) sub-column blocks, for the
+                                           operand whose dot-product dimension runs down the
+                                           rows (its codes come out transposed, see codes).
+                                           Edge blocks may overhang: missing elements take part
+                                           in nothing                                        */
     int32_t n_formats;      /* 2 or 3                                                        */
     int32_t formats[3];     /* {E4M3,BF16} or {E4M3,E5M2,BF16}, in this order                */
     int32_t criterion;      /* mor_criterion_t; three formats need BLOCK_VS_E5M2             */
@@ -138,7 +141,9 @@ typedef struct mor_tensor_stats {
  * mor_tensor_stats_t.group_mantissa).  All DEVICE pointers.  Block arrays are row-major
  * over the block grid [ceil(rows/block_rows), ceil(cols/block_cols)]. */
 typedef struct mor_outputs {
-    uint8_t* codes;         /* [rows, codes_ld] FP8 codes, 16-byte aligned.  E4M3 codes
+    uint8_t* codes;         /* [rows, codes_ld] FP8 codes, 16-byte aligned ((128,1) blocks:
+                               transposed, [cols, codes_ld] with codes_ld >= roundup(rows,16),
+                               so that every block is contiguous).  E4M3 codes
                                everywhere except in blocks that selected E5M2; blocks that
                                selected BF16 still hold their E4M3 codes.  Bytes in columns
                                cols..codes_ld-1 of each row are left untouched               */
@@ -149,7 +154,8 @@ typedef struct mor_outputs {
     uint8_t* sel;           /* [n_blocks] mor_format_t chosen for the block                  */
     float*   scale_f32;     /* [n_blocks] optional (required for MOR_SCALE_FP32_AMAX): the
                                selected format's scale as a binary32                         */
-    void*    bf16_fallback; /* optional, BF16 [rows, ld] like x: receives a copy of every
+    void*    bf16_fallback; /* optional (not with (128,1) blocks, nor is fake_quant),
+                               BF16 [rows, ld] like x: receives a copy of every
                                block that selected BF16 (other blocks are left untouched).
                                NULL = the fallback is the input itself.  Per-block criteria
                                only                                                          */

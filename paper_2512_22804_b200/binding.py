@@ -253,9 +253,14 @@ class Outputs:
     block_stats: object = None    # uint8 [n_blocks * 24]
     tensor_stats: object = None   # uint8 [80]
     cols: int = 0
+    rows: int = 0
+    transposed: bool = False      # (128, 1) sub-column blocks: codes are stored [cols, rows]
     c_struct: mor_outputs_t = field(default_factory=mor_outputs_t)
 
     def codes_view(self):
+        """The codes as a [rows, cols] view, whatever the stored layout."""
+        if self.transposed:
+            return self.codes[:, :self.rows].t()
         return self.codes[:, :self.cols]
 
     def tensor_stats_dict(self) -> dict:
@@ -273,11 +278,12 @@ def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, b
 
     g = grid_of(rows, cols, recipe.block)
     nb = g[0] * g[1]
-    o = Outputs(cols=cols)
-    ld = (cols + 15) // 16 * 16
+    transposed = tuple(recipe.block) == (128, 1)
+    o = Outputs(cols=cols, rows=rows, transposed=transposed)
+    ld = ((rows if transposed else cols) + 15) // 16 * 16
     u8 = dict(dtype=torch.uint8, device=device)
     if codes:
-        o.codes = torch.empty((rows, ld), **u8)
+        o.codes = torch.empty((cols if transposed else rows, ld), **u8)
     o.scale_e8m0 = torch.empty(g, **u8)
     o.sel = torch.empty(g, **u8)
     if scale_f32 or recipe.scale_mode == MOR_SCALE_FP32_AMAX:

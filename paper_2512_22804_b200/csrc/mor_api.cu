@@ -29,6 +29,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     else if (d.block_rows == 128 && d.block_cols == 128) s.kind = KIND_BLK128;
     else if (d.block_rows == 64 && d.block_cols == 64) s.kind = KIND_BLK64;
     else if (d.block_rows == 1 && d.block_cols == 0) s.kind = KIND_CHANNEL;
+    else if (d.block_rows == 128 && d.block_cols == 1) s.kind = KIND_COL128;
     else return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     const uint64_t nbc = empty ? 0 : (uint64_t)(d.cols + 127) / 128;
@@ -43,6 +44,11 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         s.n_blocks = s.n_units;
     } else if (s.kind == KIND_BLK64) {
         const uint64_t nb = empty ? 0 : ((uint64_t)(d.rows + 63) / 64) * ((uint64_t)(d.cols + 63) / 64);
+        if (nb >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
+        s.n_units = (uint32_t)nb;
+        s.n_blocks = nb;
+    } else if (s.kind == KIND_COL128) {
+        const uint64_t nb = empty ? 0 : nbr * (uint64_t)d.cols;
         if (nb >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
         s.n_units = (uint32_t)nb;
         s.n_blocks = nb;
@@ -97,7 +103,9 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
     const bool empty = d.rows == 0 || d.cols == 0;
     if (store) {
         if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
-        if (o.codes_ld < (int64_t)round_up((size_t)d.cols, 16)) return MOR_ERR_INVALID_ARG;
+        // sub-column blocks leave their codes transposed: [cols, codes_ld] with the rows along the contiguous dimension
+        if (o.codes_ld < (int64_t)round_up((size_t)(s.kind == KIND_COL128 ? d.rows : d.cols), 16)) return MOR_ERR_INVALID_ARG;
+        if (s.kind == KIND_COL128 && (o.bf16_fallback != nullptr || o.fake_quant != nullptr)) return MOR_ERR_UNSUPPORTED;
         if (o.codes_ld % 16 != 0 || !aligned(o.codes, 16)) return MOR_ERR_ALIGNMENT;
         if (d.scale_mode == MOR_SCALE_FP32_AMAX && o.scale_f32 == nullptr && s.n_blocks) return MOR_ERR_INVALID_ARG;
         if (o.fake_quant && !aligned(o.fake_quant, 16)) return MOR_ERR_ALIGNMENT;
@@ -146,7 +154,9 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
         return false;
     if (store) {
         const cuuint64_t out_stride[1] = {(cuuint64_t)o.codes_ld};
-        if (enc(&out_map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, o.codes, dims, out_stride, box, estr,
+        const cuuint64_t dims_t[2] = {(cuuint64_t)d.rows, (cuuint64_t)d.cols};      // transposed codes of sub-column blocks
+        const bool transposed = d.block_rows == 128 && d.block_cols == 1;
+        if (enc(&out_map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, o.codes, transposed ? dims_t : dims, out_stride, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return false;
@@ -197,7 +207,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
-    r.keys = it.prepass ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
+    r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
     r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kTileRows : 4u;
     r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kTileRows : nullptr;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
@@ -325,7 +335,7 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
     it.prepass = it.s.n_tiles != 0 && !(d->group_amax != nullptr && it.s.kind != KIND_TENSOR && it.s.kind != KIND_CHANNEL);
-    it.v.scan = !it.prepass;
+    it.v.scan = !it.prepass || it.s.kind == KIND_COL128;       // sub-column blocks: the main kernel always scans
     return MOR_OK;
 }
 
@@ -470,6 +480,7 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
     if (host_desc->group_amax != nullptr) return MOR_ERR_INVALID_ARG;
     if (host_out->bf16_fallback != nullptr) return MOR_ERR_UNSUPPORTED;   // the fallback is the caller's own host tensor
     if (host_out->fake_quant != nullptr) return MOR_ERR_UNSUPPORTED;
+    if (host_desc->block_rows == 128 && host_desc->block_cols == 1) return MOR_ERR_UNSUPPORTED;   // transposed codes: device entry points only
     if (host_desc->rows < 0 || host_desc->cols < 0 || host_desc->ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t dev_codes_ld = (int64_t)round_up((size_t)host_desc->cols, 16);

@@ -397,6 +397,7 @@ cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int k
         case KIND_BLK128: mor_finalise_kernel<KIND_BLK128><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_BLK64: mor_finalise_kernel<KIND_BLK64><<<grid, kThreads, 0, s>>>(p, partials); break;
         case KIND_CHANNEL: mor_finalise_kernel<KIND_CHANNEL><<<grid, kThreads, 0, s>>>(p, partials); break;
+        case KIND_COL128: mor_finalise_kernel<KIND_COL128><<<grid, kThreads, 0, s>>>(p, partials); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

@@ -613,6 +613,7 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     TileMeta m;
     m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
     m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
+    if (p.b.t[t.ti].kind == KIND_COL128) m.blk_base = (uint32_t)(t.row0 / kTileRows) * (uint32_t)p.b.t[t.ti].cols + (uint32_t)t.col0;
     if (p.b.t[t.ti].kind == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
     m.pad = 0;
     C.meta[s] = m;
@@ -655,7 +656,8 @@ template <int KIND, bool THREE, bool STORE>
 __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsigned char* out, Partial* __restrict__ partials,
                                            int lane)
 {
-    constexpr int kEntries = (KIND == KIND_ROW128) ? kTileRows : kThreads;
+    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;   // 128 one-line blocks per tile
+    constexpr int kEntries = kLineBlocks ? kTileRows : kThreads;
     bool stores_pending = false;
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
@@ -671,7 +673,8 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
             if (STORE && !codes_wait && lane == 0) {
                 // the codes are complete: start the tile store at once, it runs while the sums are formed
-                tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
+                // (sub-column blocks: the staging tile and the code tensor are transposed)
+                tma_store_tile(&p.out_map[t.ti], KIND == KIND_COL128 ? t.row0 : t.col0, KIND == KIND_COL128 ? t.col0 : t.row0, out + b * kOutBytes);
                 bulk_commit();
                 stores_pending = true;
             }
@@ -692,7 +695,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 f52[r] += e.e52;
                 nnz[r] += e.nnz_nonf & 0xFFFFu;
                 nonf[r] += e.nnz_nonf >> 16;
-                if (KIND == KIND_ROW128) {
+                if (kLineBlocks) {
                     const uint32_t sel = e.sel_min & 0xFFFFu;
                     n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
                 }
@@ -710,7 +713,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 if (NR == 1) { nnz[r] = __reduce_add_sync(0xFFFFFFFFu, nnz[r]); nonf[r] = __reduce_add_sync(0xFFFFFFFFu, nonf[r]); }
             }
             mn = __reduce_min_sync(0xFFFFFFFFu, mn);
-            if (KIND == KIND_ROW128) {
+            if (kLineBlocks) {
                 n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
                 n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
                 nb = __reduce_add_sync(0xFFFFFFFFu, nb);
@@ -868,6 +871,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     // this choice the 8 threads of a 128-bit load phase and the 16 threads of a 64-bit store phase
     // touch distinct banks.
     const int swz = (row & 7) ^ (h << 2);
+    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;
     const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
     const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
     const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
@@ -900,7 +904,18 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             m.local = 0; m.row0 = 0; m.col0 = 0; m.pad = 0;
         }
         uint32_t w[32];
-        {
+        if (KIND == KIND_COL128) {
+            // sub-column blocks: this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows
+            // per word, so that everything after this point works on the block as on a row piece
+            const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                uint32_t lo, hi;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
+                w[i] = lo | (hi << 16);
+            }
+        } else {
             const uint32_t a = in_base + s * kInBytes + in_off;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -937,7 +952,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             nonfin = (key >> 31) != 0u;
             key &= 0x7FFFFFFFu;
             if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);   // warp-uniform (a tile-wide key is CTA-uniform already)
-        } else if (KIND == KIND_ROW128) {
+        } else if (kLineBlocks) {
             key = scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
@@ -1010,20 +1025,20 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             if (careful) convert_words<YARD, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
             else         convert_words<YARD, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
 
-            if (KIND == KIND_ROW128) {
+            if (kLineBlocks) {
                 // ---- block sums, decision, metadata ----
                 e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
                 e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
                 uint32_t nz = nnz | (nonf << 16);
                 nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
-                const bool valid = row < m.vrows;
-                sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)m.vcols);
+                const bool valid = row < (KIND == KIND_COL128 ? m.vcols : m.vrows);
+                sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
                 if (THREE && STORE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
                 if (h == 0) {
                     sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
                            make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
                     if (valid) {
-                        const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
+                        const uint32_t blk = m.blk_base + (uint32_t)row * (KIND == KIND_COL128 ? 1u : R.nbc);
                         const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
                         if (R.sel) R.sel[blk] = (uint8_t)sel;
                         if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
@@ -1168,6 +1183,8 @@ cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* part
         case KIND_ROW128: return launch_main_k<KIND_ROW128>(v, p, partials, s);
         case KIND_BLK128: return launch_main_k<KIND_BLK128>(v, p, partials, s);
         case KIND_BLK64: return launch_main_k<KIND_BLK64>(v, p, partials, s);
+        case KIND_COL128:    // sub-column blocks: the main kernel always scans (the pre-pass leaves no column keys)
+            return v.scan ? launch_main_ks<KIND_COL128, true>(v, p, partials, s) : cudaErrorInvalidValue;
         case KIND_CHANNEL:   // the row amax spans tiles: always taken from the pre-pass
             return v.scan ? cudaErrorInvalidValue : launch_main_ks<KIND_CHANNEL, false>(v, p, partials, s);
     }

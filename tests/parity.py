@@ -78,7 +78,7 @@ def compare(bits: np.ndarray, recipe: mb.Recipe, out: "mb.Outputs", ref: "orc.Re
     ts = out.tensor_stats_dict()
     sel = out.sel.cpu().numpy().reshape(-1)
     scale = out.scale_e8m0.cpu().numpy().reshape(-1)
-    codes = None if out.codes is None else out.codes.cpu().numpy()[:, :cols]
+    codes = None if out.codes is None else out.codes_view().cpu().numpy()
     idx = np.arange(nb) if ids is None else np.asarray(ids)
     th = float(np.float32(recipe.threshold))
 

@@ -77,6 +77,36 @@ def test_narrow_range_blocks_next_to_wide_range_blocks(block, formats):
             assert rep.n_exempt <= 1
 
 
+# ------------------------------------------------------------ sub-column blocks (128 x 1), transposed codes
+
+@pytest.mark.parametrize("shape", [(256, 256), (128, 1), (300, 200), (1, 130), (517, 72)])
+@pytest.mark.parametrize("formats", [TWO, THREE])
+def test_sub_column_blocks_with_transposed_codes(shape, formats):
+    g = wl.gradient_like(shape[0], shape[1], seed=63) if shape[0] > 1 else wl.weight_like(1, shape[1], seed=63)
+    if shape[0] > 200:
+        g[130:, : shape[1] // 2] = wl.weight_like(shape[0] - 130, shape[1] // 2, seed=64)    # blocks that keep E4M3
+        g[3, 5] = 0x7FC0
+    ld = (shape[1] + 7) // 8 * 8 + 8
+    for flags in (0, mb.MOR_FLAG_STRICT_TIES | mb.MOR_FLAG_RANGE_MIN_INCLUDES_ZERO):
+        for mode in (mb.MOR_SCALE_GAM, mb.MOR_SCALE_FP32_AMAX):
+            rep = parity.run_and_compare(g, recipe((128, 1), formats, flags=flags, scale_mode=mode), pad_to=ld)
+            assert rep.n_exempt <= 2
+    parity.run_and_compare(g, recipe((128, 1), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), pad_to=ld, group_amax_supplied=True)
+
+
+def test_sub_column_codes_are_the_transpose_of_what_row_blocks_give_for_the_transposed_tensor():
+    import torch
+
+    g = wl.activation_like(256, 384, seed=65)
+    x = parity.to_device(g)
+    xt = parity.to_device(np.ascontiguousarray(g.T))
+    a = mb.analyze_quantize(x, recipe((128, 1), THREE))
+    b = mb.analyze_quantize(xt, recipe((1, 128), THREE))
+    torch.cuda.synchronize()
+    assert a.codes.shape == (384, 256) and torch.equal(a.codes, b.codes)          # stored transposed: same bytes
+    assert torch.equal(a.sel.t().contiguous(), b.sel) and torch.equal(a.scale_e8m0.t().contiguous(), b.scale_e8m0)
+
+
 # ------------------------------------------------------------ fake quantisation (Section 4)
 
 @pytest.mark.parametrize("block", KINDS + [(1, 0)])
