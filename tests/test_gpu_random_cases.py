@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 
 TWO = (mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16)
 THREE = (mb.MOR_FMT_E4M3, mb.MOR_FMT_E5M2, mb.MOR_FMT_BF16)
-PARTITIONS = [(0, 0), (1, 128), (128, 128), (64, 64), (1, 0)]
+PARTITIONS = [(0, 0), (1, 128), (128, 128), (64, 64), (1, 0), (128, 1)]
 
 
 def draw_case(rng):
@@ -46,7 +46,7 @@ def draw_case(rng):
     return bits, recipe, ld, bool(rng.random() < 0.3)
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(60))
 def test_random_case(seed):
     rng = np.random.default_rng(1000 + seed)
     bits, recipe, ld, supplied = draw_case(rng)
