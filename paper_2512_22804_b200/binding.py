@@ -366,16 +366,23 @@ class BatchPlan:
     """Descriptors, outputs and workspace of a fixed list of tensors, built once so that a
     step is a single call of mor_analyze_quantize_batched."""
 
-    def __init__(self, xs: Sequence, recipes: Sequence[Recipe], *, group_amax=None, block_stats=False):
+    def __init__(self, xs: Sequence, recipes: Sequence[Recipe], *, group_amax=None, block_stats=False,
+                 fallback=False, fake_quant=False):
+        """`fallback` and `fake_quant` are one flag for all tensors or one flag per tensor."""
         assert len(xs) == len(recipes) and len(xs) > 0
         self.xs = list(xs)
         self.group_amax = group_amax
+        per = lambda f: list(f) if isinstance(f, (list, tuple)) else [bool(f)] * len(xs)
+        fallback, fake_quant = per(fallback), per(fake_quant)
+        assert len(fallback) == len(xs) == len(fake_quant)
         descs, self.outs = [], []
         for i, (x, r) in enumerate(zip(xs, recipes)):
             ga = None if group_amax is None else group_amax[i:i + 1]
             d = desc_for(x, r, None, ga)
             descs.append(d)
-            self.outs.append(alloc_outputs(d.rows, d.cols, r, x.device, block_stats=block_stats))
+            self.outs.append(alloc_outputs(d.rows, d.cols, r, x.device, block_stats=block_stats,
+                                           fallback_like=x if fallback[i] else None,
+                                           fake_quant_like=x if fake_quant[i] else None))
         self.descs = (mor_tensor_desc_t * len(descs))(*descs)
         self.couts = (mor_outputs_t * len(descs))(*[o.c_struct for o in self.outs])
         self.n = len(descs)

@@ -667,7 +667,10 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const TileId t = locate_tile(p.b, tile);        // before the wait: off the critical path
         const TensorRec& R = p.b.t[t.ti];
         constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
-        const bool need_dec = kTileBlocks && (THREE || (STORE && (R.fallback != nullptr || R.fake_quant != nullptr)));
+        // the decision is handed back every tile of a launch with whole-tile blocks, whether this
+        // tensor's compute threads wait for it or not: the barrier's phase then follows the tile count,
+        // also when tensors with and without a BF16 copy share a launch
+        constexpr bool need_dec = kTileBlocks;
         const bool codes_wait = STORE && kTileBlocks && THREE;
         out_full_sync(b);                                // sleeps until every compute thread has arrived
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {

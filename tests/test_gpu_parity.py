@@ -306,6 +306,38 @@ def test_bf16_fallback_copies_only_rejected_blocks():
         assert (fb[:, 1000:] == 0).all()
 
 
+@pytest.mark.parametrize("block", [(128, 128), (64, 64)])
+@pytest.mark.parametrize("formats", [TWO, THREE])
+def test_batched_call_mixes_tensors_with_and_without_bf16_copy(block, formats):
+    """One launch whose thread blocks walk through tiles of tensors that ask for the BF16 copy or the
+    fake-quantised output and of tensors that do not: every tensor equals its own single call."""
+    import torch
+
+    n = 6
+    host = [wl.gradient_like(2048, 2048, seed=300 + i) if i % 2 else wl.weight_like(2048, 2048, seed=300 + i)
+            for i in range(n)]
+    xs = [parity.to_device(h) for h in host]
+    r = recipe(block, formats)
+    fb = [False, True, False, False, True, False]
+    fq = [False, False, True, False, True, False]
+    plan = mb.BatchPlan(xs, [r] * n, block_stats=True, fallback=fb, fake_quant=fq)
+    plan.run()
+    plan.run()
+    torch.cuda.synchronize()
+    for i in range(n):
+        single = mb.analyze_quantize(xs[i], r, block_stats=True, fallback=fb[i], fake_quant=fq[i])
+        torch.cuda.synchronize()
+        o = plan.outs[i]
+        assert o.tensor_stats_dict() == single.tensor_stats_dict() and o.tensor_stats_dict()["status"] == 0
+        assert torch.equal(o.codes, single.codes) and torch.equal(o.sel, single.sel)
+        if fb[i]:
+            assert torch.equal(o.bf16_fallback, single.bf16_fallback)
+        if fq[i]:
+            assert torch.equal(o.fake_quant.view(torch.int16), single.fake_quant.view(torch.int16))
+    ref = orc.run(host[4], r.block, list(r.formats), r.criterion, r.threshold, n_threads=8)
+    parity.compare(host[4], r, plan.outs[4], ref)
+
+
 def test_batched_call_equals_single_calls():
     import torch
 
