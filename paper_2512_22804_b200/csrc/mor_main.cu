@@ -9,14 +9,17 @@
 //                  two-stage ring of 32 KiB buffers to registers, then one thread starts the TMA
 //                  tile load (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) of the
 //                  tile that uses the stage next; an mbarrier per stage tells when it has landed;
-//   compute warps  8 warps, two threads per tile row.  A thread copies its 64 elements from the
-//                  stage to registers, scans them for amax / smallest non-zero, derives the scale,
-//                  converts and accumulates the error terms from the registers, and writes its
-//                  codes to a 16 KiB staging buffer;
+//   compute warps  8 warps, two threads per tile row (per tile column with 128x1 blocks).  A thread
+//                  copies its 64 elements from the stage to registers, takes the block's amax and
+//                  smallest non-zero from the key that the amax pre-pass left for the block and
+//                  that arrived with the tile (or scans its registers for them where the caller
+//                  supplied the group amax and no pre-pass ran), derives the scale, converts and
+//                  accumulates the error terms from the registers, and writes its codes to a
+//                  16 KiB staging buffer;
 //   store warp     sleeps on a hardware barrier until the staging buffer is complete, issues the
 //                  TMA tile store of the codes (clipped at the tensor's edge by the hardware),
 //                  adds up the threads' sums in a fixed order, and writes the tile's partial and,
-//                  for 128x128 blocks, the block's decision and metadata.
+//                  for 128x128 and 64x64 blocks, the blocks' decisions and metadata.
 // Every wait on an mbarrier is bounded; a wait that runs out sets a status word that the
 // finalise kernel copies into mor_tensor_stats_t.status.  From then on the CTA's threads skip
 // the work and the waits but keep every barrier arrival, so that nobody is left waiting.
@@ -873,7 +876,10 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     // Chunk order: thread (row, h) holds the 16-byte chunk c of its 128 bytes as chunk c ^ swz.  With
     // this choice the 8 threads of a 128-bit load phase and the 16 threads of a 64-bit store phase
     // touch distinct banks.
-    const int swz = (row & 7) ^ (h << 2);
+    // Sub-column blocks read 16-bit pieces down a column; all rows of a column share a bank, so there
+    // the two columns that share a 32-bit word get the same order (they then read the same word) at the
+    // price of a two-way conflict on the stores.
+    const int swz = KIND == KIND_COL128 ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
     constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;
     const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
     const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
