@@ -246,8 +246,13 @@ def main():
         for name, rec in (("128x128, tensor-level Eq.2 (E4M3 only)", mb.Recipe((128, 128), recipe.formats, T, 0.045)),
                           ("1x128, two-way Eq.3", mb.Recipe((1, 128), recipe.formats, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)),
                           ("1x128, tensor-level Eq.2 (E4M3 only)", mb.Recipe((1, 128), recipe.formats, T, 0.045)),
-                          ("per channel, tensor-level Eq.2 (E4M3 only)", mb.Recipe((1, 0), recipe.formats, T, 0.045))):
-            vp = mb.BatchPlan(xs, [rec] * B)
+                          ("per channel, tensor-level Eq.2 (E4M3 only)", mb.Recipe((1, 0), recipe.formats, T, 0.045)),
+                          ("128x128, two-way Eq.3, group amax supplied by the caller (no pre-pass: the main kernel scans the blocks itself)", recipe),
+                          ("1x128, two-way Eq.3, group amax supplied by the caller (no pre-pass)", mb.Recipe((1, 128), recipe.formats, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045))):
+            supplied = None
+            if "supplied" in name:
+                supplied = torch.tensor([o.tensor_stats_dict()["group_amax"] for o in plan.outs], dtype=torch.float32, device=dev)
+            vp = mb.BatchPlan(xs, [rec] * B, group_amax=supplied)
             ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             ea.record(stream); eb.record(stream)
             sv = mb.mor_stage_events_t()
