@@ -269,6 +269,28 @@ def main():
             variants.append({"recipe": name, "main_kernel_GBs": gbs, "frac_of_measured_copy": gbs / peak, "frac_of_8TBs": gbs / 8000.0})
             del vp
 
+    # ---- configs[0]: one 1024x1024 tensor, per-tensor partition: latency of a step, launched directly and
+    #      replayed as a CUDA graph (the step is launch-bound at this size)
+    small = None
+    if rank == 0 and not args.no_variants:
+        sb = wl.gaussian_outlier_rows()
+        sx = torch.from_numpy(sb.view(np.int16)).view(torch.bfloat16).to(dev)
+        sp = mb.BatchPlan([sx], [mb.Recipe((0, 0), recipe.formats, mb.MOR_CRIT_TENSOR_MEAN_REL, 0.045)])
+        graph = sp.capture()
+        small = {"workload": "BASELINE configs[0]: one 1024x1024 tensor, per-tensor partition, Eq.2"}
+        for key, fn in (("direct_us", lambda: sp.run(torch.cuda.current_stream())), ("cuda_graph_us", graph.replay)):
+            for _ in range(5):
+                fn()
+            torch.cuda.synchronize()
+            ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ts = []
+            for _ in range(20):
+                ea.record(); fn(); eb.record()
+                torch.cuda.synchronize()
+                ts.append(ea.elapsed_time(eb) * 1e3)
+            small[key] = statistics.median(ts)
+        del graph, sp
+
     # ---- end to end through the host-memory entry point: pinned inputs in, codes/scales/selection/stats out
     e2e = None
     if not args.no_e2e:
@@ -356,7 +378,7 @@ def main():
                 "elements_per_s": elements * world / (ms_step * 1e-3),
                 "frac_of_hbm_peak_8TBs": value / 8000.0, "frac_of_measured_copy": value / peak,
                 "fp8_block_fraction": fp8_frac, "fp8_tensor_fraction_eq2": tensor_fp8,
-                "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "other_recipes_same_tensors": variants,
+                "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "other_recipes_same_tensors": variants, "small_tensor_latency": small,
                 "paper_context": "the paper reports no throughput and names no hardware; its own figures are FP8 tensor fractions "
                                  "(98.38 % / 95.93 % per channel, tensor-level MoR, Nemotron-3 8B), see BASELINE.md",
                 "gpu_launches": 3 * K, "clocks": clocks}

@@ -394,3 +394,17 @@ class BatchPlan:
                       None if events is None else C.byref(events))
         if st != MOR_OK:
             raise MorError(st, "mor_analyze_quantize_batched")
+
+    def capture(self):
+        """The step as a CUDA graph (memset, amax pre-pass, main kernel, finalise as graph nodes), for
+        launch-bound cases such as a single small tensor.  One ordinary step runs first, so that the library's
+        per-device set-up happens outside the capture.  Replay with ``graph.replay()``; the tensors, outputs
+        and workspace of this plan are baked in."""
+        import torch
+
+        self.run()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.run(torch.cuda.current_stream())
+        return graph

@@ -81,6 +81,8 @@ struct alignas(64) MainParams {
     uint32_t* device_status;
 };
 
+static_assert(sizeof(MainParams) <= 32764, "kernel parameters are limited to 32764 bytes");
+
 struct MainVariant {
     int kind;        // Kind
     bool yard;       // evaluate E5M2 as well (Eq. 3, or statistics asked for)

@@ -373,6 +373,25 @@ def test_many_tensors_exceeding_one_launch():
         parity.compare(b, r, o, ref)
 
 
+def test_step_captured_as_cuda_graph_replays_identically():
+    """BatchPlan.capture(): the memset and the three kernels as one CUDA graph; two replays, each checked
+    against the oracle after the outputs were overwritten."""
+    import torch
+
+    bits = wl.gradient_like(300, 992, seed=77)
+    r = recipe((1, 128), THREE)
+    plan = mb.BatchPlan([parity.to_device(bits)], [r], block_stats=True)
+    graph = plan.capture()
+    ref = orc.run(bits, r.block, list(r.formats), r.criterion, r.threshold)
+    for _ in range(2):
+        plan.outs[0].codes.zero_()
+        plan.outs[0].sel.fill_(9)
+        plan.outs[0].tensor_stats.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        parity.compare(bits, r, plan.outs[0], ref)
+
+
 def test_runs_are_deterministic():
     import torch
 
