@@ -269,6 +269,33 @@ def main():
             variants.append({"recipe": name, "main_kernel_GBs": gbs, "frac_of_measured_copy": gbs / peak, "frac_of_8TBs": gbs / 8000.0})
             del vp
 
+    # ---- mor_select_stats (decisions and statistics, no codes) on the same tensors: one call per tensor
+    if rank == 0 and not args.no_variants:
+        sd = [mb.desc_for(x, recipe) for x in xs]
+        so = [mb.alloc_outputs(ROWS, COLS, recipe, dev, codes=False, block_stats=True) for _ in xs]
+        sw = torch.empty((mb.mor_workspace_bytes([sd[0]]),), dtype=torch.uint8, device=dev)
+
+        def stats_step():
+            for d, o in zip(sd, so):
+                st = mb.mor_select_stats(d, o.c_struct.block_stats, o.c_struct.tensor_stats, o.c_struct.sel,
+                                         o.c_struct.scale_e8m0, sw.data_ptr(), sw.numel(), stream.cuda_stream)
+                if st != mb.MOR_OK:
+                    raise mb.MorError(st, "mor_select_stats")
+
+        for _ in range(3):
+            stats_step()
+        torch.cuda.synchronize()
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        tms = []
+        for _ in range(5):
+            ea.record(stream); stats_step(); eb.record(stream)
+            torch.cuda.synchronize()
+            tms.append(ea.elapsed_time(eb))
+        gbs = elements * 4.0 / (statistics.median(tms) * 1e-3) / 1e9      # the tensor is read twice, nothing else of size moves
+        variants.append({"recipe": "mor_select_stats, 128x128 two-way Eq.3 with block statistics, one call per tensor (whole calls, 4 B/element)",
+                         "whole_call_GBs": gbs, "frac_of_measured_copy": gbs / peak, "frac_of_8TBs": gbs / 8000.0})
+        del so, sw
+
     # ---- configs[0]: one 1024x1024 tensor, per-tensor partition: latency of a step, launched directly and
     #      replayed as a CUDA graph (the step is launch-bound at this size)
     small = None
