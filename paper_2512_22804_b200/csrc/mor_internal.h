@@ -91,6 +91,28 @@ struct MainVariant {
     bool scan;       // the kernel scans the data for amax / smallest non-zero itself (no keys from the pre-pass)
 };
 
+// Programmatic dependent launch: a kernel launched with launch_dependent() may become resident while the
+// kernel before it in the stream is still draining; it runs its prologue and then blocks in pdl_wait() until that
+// kernel has completed and its writes are visible.  A kernel lets its successor in early with pdl_trigger()
+// (called by every CTA at its start, so the successor's CTAs only take what finishing CTAs free).  Every CTA of
+// a kernel launched this way passes pdl_wait(), so completion of a kernel implies completion of all before it.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+#endif
+
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);

@@ -115,6 +115,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32];
     __shared__ uint32_t s_qkey[kThreads / 32][4], s_qnf[kThreads / 32][4];   // 64x64 blocks: per warp and quadrant
 
+    pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     uint32_t local;
     const TensorRec& R = p.t[find_tensor(p, blockIdx.x, local)];
@@ -250,6 +251,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
 __global__ void __launch_bounds__(kTileRows)
 mor_row_keys_kernel(const __grid_constant__ BatchParams p)
 {
+    pdl_trigger();
     const TensorRec& R = p.t[blockIdx.y];
     if (R.kind != KIND_CHANNEL || R.row_keys == nullptr || blockIdx.x >= R.nbr) return;
     const uint32_t* src = R.keys + ((size_t)blockIdx.x * R.nbc) * kTileRows + threadIdx.x;
@@ -273,6 +275,7 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
 {
     __shared__ WarpPart s_wp[kThreads / 32];
     __shared__ WarpPart s_tot;
+    pdl_wait();                                          // the main kernel's partials and outputs are complete
     const TensorRec& R = p.t[blockIdx.x];
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
 
@@ -391,16 +394,17 @@ cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int k
     for (int i = 0; i < p.n; ++i)
         if (kind != KIND_TENSOR && p.t[i].criterion == MOR_CRIT_TENSOR_MEAN_REL && p.t[i].sel && p.t[i].n_units > 65536u) slices = 16;
     dim3 grid((unsigned)p.n, slices);
+    cudaError_t e = cudaSuccess;
     switch (kind) {
-        case KIND_TENSOR: mor_finalise_kernel<KIND_TENSOR><<<grid, kThreads, 0, s>>>(p, partials); break;
-        case KIND_ROW128: mor_finalise_kernel<KIND_ROW128><<<grid, kThreads, 0, s>>>(p, partials); break;
-        case KIND_BLK128: mor_finalise_kernel<KIND_BLK128><<<grid, kThreads, 0, s>>>(p, partials); break;
-        case KIND_BLK64: mor_finalise_kernel<KIND_BLK64><<<grid, kThreads, 0, s>>>(p, partials); break;
-        case KIND_CHANNEL: mor_finalise_kernel<KIND_CHANNEL><<<grid, kThreads, 0, s>>>(p, partials); break;
-        case KIND_COL128: mor_finalise_kernel<KIND_COL128><<<grid, kThreads, 0, s>>>(p, partials); break;
+        case KIND_TENSOR: e = launch_dependent(mor_finalise_kernel<KIND_TENSOR>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_ROW128: e = launch_dependent(mor_finalise_kernel<KIND_ROW128>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_BLK128: e = launch_dependent(mor_finalise_kernel<KIND_BLK128>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_BLK64: e = launch_dependent(mor_finalise_kernel<KIND_BLK64>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_CHANNEL: e = launch_dependent(mor_finalise_kernel<KIND_CHANNEL>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_COL128: e = launch_dependent(mor_finalise_kernel<KIND_COL128>, grid, dim3(kThreads), 0, s, p, partials); break;
         default: return cudaErrorInvalidValue;
     }
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace mor

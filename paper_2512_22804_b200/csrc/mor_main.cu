@@ -1132,6 +1132,10 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     // done here once per CTA with the IEEE divide and looked up per block afterwards
     if (tid < 128) C.rtab[tid] = __float_as_uint(__fdiv_rn(448.0f, 1.0f + (float)tid * 0.0078125f));
     __syncthreads();
+    // Up to here nothing was read that an earlier kernel of the stream writes: this CTA may have become resident
+    // while the amax pre-pass was still draining.  From here on its amax and keys are needed.
+    pdl_trigger();
+    pdl_wait();
 
     if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE, SCAN>(p, C, in, out, tid);
     else if (warp == kLoadWarp) load_warp(p, C, in, lane);
@@ -1157,8 +1161,7 @@ cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s
     }
     const uint32_t resident = 2u * (uint32_t)sm_count[dev];
     const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
-    kfn<<<grid, kMainThreads, kSmemBytes, s>>>(p, partials);
-    return cudaGetLastError();
+    return launch_dependent(kfn, dim3(grid), dim3(kMainThreads), (size_t)kSmemBytes, s, p, partials);
 }
 
 template <int KIND, bool SCAN>
