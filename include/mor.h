@@ -107,8 +107,10 @@ typedef struct mor_tensor_desc {
                                already: it fixes the shared mantissa; block amaxes are still
                                taken from the data, so a stale value cannot cause saturation.
                                NULL = the library computes it with one extra read of the
-                               tensor (always done for the (0,0) partition, whose block amax
-                               is the tensor amax)                                           */
+                               tensor (always done for the (0,0) and (1,0) partitions, whose
+                               block amax spans tiles; never needed for the E8M0 and FP32-amax
+                               scale modes of the other partitions, which have no shared
+                               mantissa: those read the tensor once)                         */
 } mor_tensor_desc_t;
 
 /* Per-block quantities behind the decisions (Eq. 3 sums, Eq. 4 range). */

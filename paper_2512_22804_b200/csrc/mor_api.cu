@@ -334,7 +334,10 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.store = store;
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
-    it.prepass = it.s.n_tiles != 0 && !(d->group_amax != nullptr && it.s.kind != KIND_TENSOR && it.s.kind != KIND_CHANNEL);
+    // Nor is it needed where the scale has no shared mantissa (E8M0 and FP32-amax modes): those need the block
+    // amax only, which the main kernel finds in the tile it has just read, so the tensor is read once.
+    const bool whole_rows = it.s.kind == KIND_TENSOR || it.s.kind == KIND_CHANNEL;
+    it.prepass = it.s.n_tiles != 0 && (whole_rows || (d->group_amax == nullptr && d->scale_mode == MOR_SCALE_GAM));
     it.v.scan = !it.prepass || it.s.kind == KIND_COL128;       // sub-column blocks: the main kernel always scans
     return MOR_OK;
 }

@@ -241,7 +241,9 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
         }
         // non-negative binary32 patterns order like the values
-        atomicMax(reinterpret_cast<unsigned int*>(R.amax_slot), (kk >> 16) << 16);
+        // (atomics on one address are served one at a time: read first, most tiles end there)
+        unsigned int* slot = reinterpret_cast<unsigned int*>(R.amax_slot);
+        if (__ldcg(slot) < ((kk >> 16) << 16)) atomicMax(slot, (kk >> 16) << 16);
         if (nf) atomicAdd(R.nonfinite_slot, nf);
     }
 }

@@ -381,6 +381,16 @@ __device__ __forceinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
 
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
 
+// Raise the tensor amax slot to the BF16 magnitude `bits` (non-negative binary32 patterns order like the
+// values).  Atomics on one address are served one at a time, so the slot is read first: after the first
+// tiles of a tensor almost every call ends there.
+__device__ __forceinline__ void raise_amax(float* slot, uint32_t bits, bool active)
+{
+    if (!active || bits == 0u) return;
+    unsigned int* p = reinterpret_cast<unsigned int*>(slot);
+    if (__ldcg(p) < (bits << 16)) atomicMax(p, bits << 16);
+}
+
 // ------------------------------------------------------------------ conversion ----
 
 // Fast path for one BF16 pair: two E4M3 codes (and two E5M2 codes) with their terms of
@@ -969,8 +979,13 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = scan_words_finite(w);
                 key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             }
+            // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
+            // patterns order like the values)
+            const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
+            raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
         } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
             key = scan_words(w);
+            uint32_t tile_amax = 0u;
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
                 // the warps exchange their keys; with 64x64 blocks a warp has one per column half (lane parity)
@@ -996,9 +1011,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 }
                 nonfin = pass == 1 || (any >> 16) >= kBf16Inf;                     // CTA-uniform
                 if (dead) { key = 0u; nonfin = false; }
+                tile_amax = any >> 16;
                 if (pass == 1 || !nonfin) break;
                 key = scan_words_finite(w);
             }
+            // no pre-pass ran: the tensor amax that the summary reports is gathered here
+            raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead);
         } else {
             key = scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
