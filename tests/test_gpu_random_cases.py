@@ -53,3 +53,57 @@ def test_random_case(seed):
     stats = tuple(recipe.block) != (1, 0) and seed % 2 == 0
     rep = parity.run_and_compare(bits, recipe, pad_to=ld, block_stats=stats, group_amax_supplied=supplied)
     assert rep.n_exempt <= max(1, rep.n_blocks // 500)
+
+
+def draw_batch(rng):
+    """Several mid-sized tensors for one batched call: one or two partitions (so that launches hold several
+    tensors and every thread block walks through many tiles), random recipes, BF16 copy and fake-quantised
+    output asked for on some tensors only."""
+    n = int(rng.integers(2, 8))
+    parts = [PARTITIONS[int(rng.integers(len(PARTITIONS)))] for _ in range(2)]
+    hosts, recipes, fallback, fake = [], [], [], []
+    for _ in range(n):
+        rows, cols = int(rng.integers(300, 2600)), int(rng.integers(300, 2600)) // 8 * 8
+        seed = int(rng.integers(1 << 30))
+        gen = int(rng.integers(0, 3))
+        bits = (wl.weight_like(rows, cols, seed=seed) if gen == 0 else wl.gradient_like(rows, cols, seed=seed) if gen == 1
+                else wl.activation_like(rows, cols, n_outlier_cols=3, seed=seed))
+        if rng.random() < 0.3:
+            bits[int(rng.integers(rows)), int(rng.integers(cols))] = [0x7F80, 0x7FC0, 0x0001][int(rng.integers(3))]
+        block = parts[int(rng.integers(2))]
+        if block in ((1, 0), (0, 0)):
+            formats, crit = TWO, mb.MOR_CRIT_TENSOR_MEAN_REL
+        else:
+            formats = THREE if rng.random() < 0.4 else TWO
+            crit = mb.MOR_CRIT_BLOCK_VS_E5M2 if formats is THREE else int(rng.integers(0, 3))
+        recipes.append(mb.Recipe(block, formats, crit, 0.045, int(rng.integers(0, 3)), int(rng.integers(0, 4))))
+        hosts.append(bits)
+        fallback.append(bool(rng.random() < 0.3) and block != (128, 1) and crit != mb.MOR_CRIT_TENSOR_MEAN_REL)
+        fake.append(bool(rng.random() < 0.3) and block != (128, 1))
+    return hosts, recipes, fallback, fake, (1, 0) in parts
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_batch(seed):
+    import torch
+
+    from oracle import mor_oracle as orc
+
+    hosts, recipes, fallback, fake, has_channel = draw_batch(np.random.default_rng(90000 + seed))
+    stats = bool(seed % 2) and not has_channel
+    plan = mb.BatchPlan([parity.to_device(h) for h in hosts], recipes, block_stats=stats, fallback=fallback, fake_quant=fake)
+    plan.run()
+    plan.run()
+    torch.cuda.synchronize()
+    for host, r, out, fb, fq in zip(hosts, recipes, plan.outs, fallback, fake):
+        ob = parity.oracle_block(r.block, host.shape[1])
+        ref = orc.run(host, ob, list(r.formats), r.criterion, r.threshold, r.scale_mode, r.flags, n_threads=8)
+        rep = parity.compare(host, r, out, ref, check_block_stats=stats)
+        assert rep.n_exempt <= max(2, rep.n_blocks // 500)
+        if fq and not parity.exempt_blocks(ref, r).any():
+            want = orc.fake_quant(host, ref, ob, list(r.formats), r.criterion, r.threshold, r.scale_mode, r.flags)
+            np.testing.assert_array_equal(out.fake_quant.view(torch.int16).cpu().numpy().view(np.uint16), want)
+        if fb:
+            sel = out.sel.cpu().numpy()
+            mask = np.kron(sel == mb.MOR_FMT_BF16, np.ones(ob, dtype=bool))[:host.shape[0], :host.shape[1]]
+            np.testing.assert_array_equal(out.bf16_fallback.view(torch.int16).cpu().numpy().view(np.uint16), np.where(mask, host, 0))
