@@ -186,7 +186,13 @@ size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n);
 mor_status_t mor_analyze_quantize(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* The same analysis for `n` tensors with one set of launches per block shape. */
+/* The same analysis for `n` tensors with one set of launches per block shape.
+ * Section 3 applies the method to a tensor and to its transpose (the operand layouts of the forward
+ * and the backward GEMM).  Two neighbouring entries that name the same tensor (same x, shape, ld,
+ * recipe, group_amax) with block shape (1,128) first and (128,1) second, codes wanted, no BF16 copy or
+ * fake-quantised output on the first, are served by one main kernel that reads every tile of the tensor
+ * once and converts it along the rows and along the columns; every output equals that of two separate
+ * calls. */
 mor_status_t mor_analyze_quantize_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
                                           int n, void* workspace, size_t workspace_bytes, void* cuda_stream);
 

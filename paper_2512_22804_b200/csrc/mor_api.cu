@@ -188,6 +188,8 @@ struct Item {
     uint32_t tile_begin;
     uint64_t key_begin;      // first word of the tensor's keys
     bool prepass;            // the amax pre-pass runs for this tensor (and leaves keys)
+    int dual;                // 1, 2: first (1x128 blocks) and second (128x1 blocks) item of a pair on the same tensor
+                             // that the main kernel serves from one read of each tile; 0: not part of a pair
     int index;
 };
 
@@ -238,6 +240,26 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         it.key_begin = key_words; key_words += it.s.key_words;
     }
     if (tiles >= (1ull << 31)) return MOR_ERR_UNSUPPORTED;
+    // Two neighbouring items that ask for the same tensor under the same recipe, once with 1x128 blocks and once
+    // with 128x1 blocks (the operand layouts of the forward and the backward GEMM), are served by one main
+    // kernel that reads every tile once.  Nothing in the results depends on it.
+    for (int i = 0; i + 1 < n; ++i) {
+        Item& a = items[i];
+        Item& b = items[i + 1];
+        if (a.dual || b.dual || a.s.kind != KIND_ROW128 || b.s.kind != KIND_COL128 || a.s.n_tiles == 0) continue;
+        const mor_tensor_desc_t& da = *a.d;
+        const mor_tensor_desc_t& db = *b.d;
+        const bool same = da.x == db.x && da.rows == db.rows && da.cols == db.cols && da.ld == db.ld &&
+                          da.n_formats == db.n_formats && da.criterion == db.criterion && da.threshold == db.threshold &&
+                          da.scale_mode == db.scale_mode && da.flags == db.flags && da.group_amax == db.group_amax;
+        const bool plain = a.v.store && b.v.store && a.o.bf16_fallback == nullptr && a.o.fake_quant == nullptr &&
+                           a.v.yard == b.v.yard && a.v.three == b.v.three;
+        if (!same || !plain) continue;
+        a.dual = 1; b.dual = 2;
+        b.prepass = false;                 // the columns are scanned by the main kernel; the tensor amax is the rows' item's
+        a.v.kind = b.v.kind = KIND_DUAL;
+        b.v.scan = a.v.scan;
+    }
     const Layout l = layout_of(n, tiles, key_words);
     if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign)) return MOR_ERR_ALIGNMENT;
@@ -304,7 +326,12 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
             } else {
                 fill_rec(items[j], ws, l, bp.t[bp.n]);
                 if (!encode_maps(*items[j].d, items[j].o, v.store, mp.in_map[bp.n], mp.out_map[bp.n])) return MOR_ERR_CUDA;
-                t_end += items[j].s.n_tiles;
+                if (items[j].dual == 2) {
+                    // the columns' record shares the tiles and the group amax of the rows' record before it
+                    if (items[j].d->group_amax == nullptr) bp.t[bp.n].amax = bp.t[bp.n - 1].amax_slot;
+                } else {
+                    t_end += items[j].s.n_tiles;
+                }
                 bp.tile_end[bp.n++] = t_end;
             }
             if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
@@ -312,8 +339,19 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         if (!flush()) return MOR_ERR_CUDA;
     }
     if (ev && !record(ev->main_end)) return MOR_ERR_CUDA;
-    for (const Chunk& c : chunks)
-        if (launch_finalise(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
+    for (const Chunk& c : chunks) {
+        if (c.kind != KIND_DUAL) {
+            if (launch_finalise(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
+            continue;
+        }
+        // a launch of pairs: the rows' records and the columns' records are summarised as what they are
+        for (int dir = 0; dir < 2; ++dir) {
+            BatchParams half;
+            half.n = 0;
+            for (int k = dir; k < c.bp.n; k += 2) { half.t[half.n] = c.bp.t[k]; half.tile_end[half.n] = 0; ++half.n; }
+            if (launch_finalise(half, partials, dir ? KIND_COL128 : KIND_ROW128, stream) != cudaSuccess) return MOR_ERR_CUDA;
+        }
+    }
     if (ev && !record(ev->finalise_end)) return MOR_ERR_CUDA;
     return MOR_OK;
 }
@@ -339,6 +377,7 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     const bool whole_rows = it.s.kind == KIND_TENSOR || it.s.kind == KIND_CHANNEL;
     it.prepass = it.s.n_tiles != 0 && (whole_rows || (d->group_amax == nullptr && d->scale_mode == MOR_SCALE_GAM));
     it.v.scan = !it.prepass || it.s.kind == KIND_COL128;       // sub-column blocks: the main kernel always scans
+    it.dual = 0;
     return MOR_OK;
 }
 

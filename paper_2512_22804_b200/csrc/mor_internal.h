@@ -23,7 +23,10 @@ constexpr int kThreads = 256;          // amax and finalise kernels; compute thr
 constexpr int kMainThreads = 320;      // 8 compute warps + load warp + store warp
 constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor maps travel as kernel parameters
 
-enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3, KIND_CHANNEL = 4, KIND_COL128 = 5 };
+enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3, KIND_CHANNEL = 4, KIND_COL128 = 5,
+                  // main kernel only: 1x128 blocks and 128x1 blocks of the same tensor from one read of each tile; the
+                  // launch's records come in pairs (rows, columns) that share their tiles
+                  KIND_DUAL = 6 };
 
 // Per-tile partial results, reduced in tile order by the finalise kernel.
 struct Partial {

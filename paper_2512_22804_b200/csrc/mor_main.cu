@@ -669,15 +669,18 @@ template <int KIND, bool THREE, bool STORE>
 __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsigned char* out, Partial* __restrict__ partials,
                                            int lane)
 {
-    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;   // 128 one-line blocks per tile
+    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128 || KIND == KIND_DUAL;   // 128 one-line blocks per tile
     constexpr int kEntries = kLineBlocks ? kTileRows : kThreads;
     bool stores_pending = false;
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        // both directions from one read: two conversions per tile, rows (record ti) then columns (record ti + 1)
+        const uint32_t tile = blockIdx.x + (KIND == KIND_DUAL ? it >> 1 : it) * gridDim.x;
         if (tile >= p.total_tiles) break;
         const uint32_t b = it & 1u, n = it >> 1;
-        const TileId t = locate_tile(p.b, tile);        // before the wait: off the critical path
+        const bool columns = KIND == KIND_COL128 || (KIND == KIND_DUAL && (it & 1u));
+        TileId t = locate_tile(p.b, tile);              // before the wait: off the critical path
+        if (KIND == KIND_DUAL && columns) t.ti += 1;
         const TensorRec& R = p.b.t[t.ti];
         constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
         // the decision is handed back every tile of a launch with whole-tile blocks, whether this
@@ -690,7 +693,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
             if (STORE && !codes_wait && lane == 0) {
                 // the codes are complete: start the tile store at once, it runs while the sums are formed
                 // (sub-column blocks: the staging tile and the code tensor are transposed)
-                tma_store_tile(&p.out_map[t.ti], KIND == KIND_COL128 ? t.row0 : t.col0, KIND == KIND_COL128 ? t.col0 : t.row0, out + b * kOutBytes);
+                tma_store_tile(&p.out_map[t.ti], columns ? t.row0 : t.col0, columns ? t.col0 : t.row0, out + b * kOutBytes);
                 bulk_commit();
                 stores_pending = true;
             }
@@ -1122,6 +1125,144 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     }
 }
 
+// ------------------------------------------------------------------ both directions from one read ----
+
+// KIND_DUAL: the tensor is wanted with 1x128 blocks and with 128x1 blocks (the two operand layouts of the forward
+// and backward GEMMs).  A tile is loaded once; the compute threads take it from the stage twice, first as rows
+// (record ti, exactly the 1x128 path), then as columns (record ti + 1, exactly the 128x1 path, codes transposed),
+// and hand each direction to the store warp as a tile of its own, so the two staging buffers alternate between
+// the directions.  The stage is released after the second copy to registers.
+template <bool YARD, bool THREE, bool SCAN>
+__device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
+{
+    const int lane = tid & 31;
+    const int row = tid >> 1, h = tid & 1;
+    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
+    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
+    int cur_ti = -1;
+    uint32_t m_g = 0;
+    int scale_mode = 0;
+    bool dead = false;
+#pragma unroll 1
+    for (uint32_t it = 0;; ++it) {
+        const uint32_t tile = blockIdx.x + it * gridDim.x;
+        if (tile >= p.total_tiles) break;
+        const uint32_t s = it % kStages;
+        if (!dead) {
+            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+        }
+        TileMeta m;
+        {
+            const uint4 q0 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
+            const uint4 q1 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
+            m.ti = dead ? 0 : (int32_t)q0.x; m.vrows = (int32_t)q0.y; m.vcols = (int32_t)q0.z; m.blk_base = q0.w;
+            m.local = q1.x; m.row0 = (int32_t)q1.y; m.col0 = (int32_t)q1.z; m.pad = 0;
+        }
+        if (m.ti != cur_ti) {
+            cur_ti = m.ti;
+            scale_mode = p.b.t[m.ti].scale_mode;
+            if (!dead) m_g = group_mantissa(*p.b.t[m.ti].amax, scale_mode);
+        }
+#pragma unroll
+        for (int dir = 0; dir < 2; ++dir) {
+            const TensorRec& R = p.b.t[m.ti + dir];
+            const uint32_t b = (uint32_t)dir, n2 = it;        // conversion number 2 * it + dir
+            const int swz = dir ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
+            uint32_t w[32];
+            uint32_t key = 0u;
+            if (dir == 0) {
+                const uint32_t a = in_base + s * kInBytes + (uint32_t)(row * 256 + h * 128 + (swz << 4));
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 v = lds128(a ^ (j << 4));
+                    w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+                }
+                if (!SCAN) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)row * 4u));
+            } else {
+                // this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows per word
+                const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    uint32_t lo, hi;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
+                    w[i] = lo | (hi << 16);
+                }
+                stage_free_arrive(s);                       // both copies of the stage are in registers
+            }
+
+            // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
+            bool nonfin;
+            if (dir == 0 && !SCAN) {
+                nonfin = __any_sync(0xFFFFFFFFu, (key >> 31) != 0u);
+                key &= 0x7FFFFFFFu;
+            } else {
+                key = scan_words(w);
+                key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
+                nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
+                if (nonfin) {
+                    key = scan_words_finite(w);
+                    key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
+                }
+                if (dir == 0) {                             // no pre-pass ran: gather the tensor amax for the summaries
+                    const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
+                    raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
+                }
+            }
+            const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
+            uint32_t s4b, s5b;
+            block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
+            bool careful = nonfin;
+            if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
+            careful = __any_sync(0xFFFFFFFFu, careful);
+
+            // ---- staging buffer and entries of the same direction of the tile before must have been consumed ----
+            if (n2 > 0 && !dead) {
+                bool ok = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+            }
+            const uint32_t oa = out_base + b * kOutBytes + (uint32_t)(row * 128 + h * 64 + (swz << 3));
+            if (!dead) {
+                float e43, e52;
+                uint32_t nnz, nonf;
+                if (careful) convert_words<YARD, true, true>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
+                else         convert_words<YARD, false, true>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
+                e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
+                e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
+                uint32_t nz = nnz | (nonf << 16);
+                nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
+                const bool valid = row < (dir ? m.vcols : m.vrows);
+                const uint32_t sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(dir ? m.vrows : m.vcols));
+                if (THREE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
+                if (h == 0) {
+                    sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
+                           make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
+                    if (valid) {
+                        const uint32_t blk = dir ? (uint32_t)(m.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)m.col0 + (uint32_t)row
+                                                 : m.blk_base + (uint32_t)row * R.nbc;
+                        const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
+                        if (R.sel) R.sel[blk] = (uint8_t)sel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
+                        if (R.block_stats) {
+                            mor_block_stats_t bs;
+                            bs.amax = __uint_as_float(amax_bits << 16);
+                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
+                            bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
+                            R.block_stats[blk] = bs;
+                        }
+                    }
+                }
+                fence_async_smem();                      // the codes must be visible to the TMA store
+            }
+            out_full_arrive(b);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ kernel ----
 
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
@@ -1155,7 +1296,10 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     pdl_trigger();
     pdl_wait();
 
-    if (warp < kComputeWarps) compute_warps<KIND, YARD, THREE, STORE, SCAN>(p, C, in, out, tid);
+    if (warp < kComputeWarps) {
+        if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
+        else compute_warps<KIND, YARD, THREE, STORE, SCAN>(p, C, in, out, tid);
+    }
     else if (warp == kLoadWarp) load_warp(p, C, in, lane);
     else store_warp<KIND, THREE, STORE>(p, C, out, partials, lane);
 }
@@ -1215,6 +1359,16 @@ cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* part
         case KIND_BLK64: return launch_main_k<KIND_BLK64>(v, p, partials, s);
         case KIND_COL128:    // sub-column blocks: the main kernel always scans (the pre-pass leaves no column keys)
             return v.scan ? launch_main_ks<KIND_COL128, true>(v, p, partials, s) : cudaErrorInvalidValue;
+        case KIND_DUAL:      // rows and columns of the same tensors from one read: codes are always stored
+            if (!v.store) return cudaErrorInvalidValue;
+            if (v.scan) {
+                return v.three ? launch_main_t<KIND_DUAL, true, true, true, true>(p, partials, s)
+                     : v.yard  ? launch_main_t<KIND_DUAL, true, false, true, true>(p, partials, s)
+                               : launch_main_t<KIND_DUAL, false, false, true, true>(p, partials, s);
+            }
+            return v.three ? launch_main_t<KIND_DUAL, true, true, true, false>(p, partials, s)
+                 : v.yard  ? launch_main_t<KIND_DUAL, true, false, true, false>(p, partials, s)
+                           : launch_main_t<KIND_DUAL, false, false, true, false>(p, partials, s);
         case KIND_CHANNEL:   // the row amax spans tiles: always taken from the pre-pass
             return v.scan ? cudaErrorInvalidValue : launch_main_ks<KIND_CHANNEL, false>(v, p, partials, s);
     }
