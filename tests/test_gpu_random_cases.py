@@ -107,3 +107,38 @@ def test_random_batch(seed):
             sel = out.sel.cpu().numpy()
             mask = np.kron(sel == mb.MOR_FMT_BF16, np.ones(ob, dtype=bool))[:host.shape[0], :host.shape[1]]
             np.testing.assert_array_equal(out.bf16_fallback.view(torch.int16).cpu().numpy().view(np.uint16), np.where(mask, host, 0))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_pair_rows_and_columns(seed):
+    """The same tensor with 1x128 and with 128x1 blocks in one call (one read of each tile), one to three
+    pairs per call, random shape, recipe, scale mode and flags; both results against the oracle."""
+    import torch
+
+    from oracle import mor_oracle as orc
+
+    rng = np.random.default_rng(70000 + seed)
+    bits, _, _, supplied = draw_case(rng)
+    if seed % 6 == 0:
+        bits = wl.gradient_like(int(rng.integers(600, 2400)), int(rng.integers(600, 2400)), seed=seed)
+    formats = THREE if rng.random() < 0.5 else TWO
+    crit = mb.MOR_CRIT_BLOCK_VS_E5M2 if formats is THREE else int(rng.integers(0, 3))
+    mode, flags = int(rng.integers(0, 3)), int(rng.integers(0, 4))
+    recipes = [mb.Recipe((1, 128), formats, crit, 0.045, mode, flags), mb.Recipe((128, 1), formats, crit, 0.045, mode, flags)]
+    rows, cols = bits.shape
+    host = np.full((rows, (cols + 7) // 8 * 8 + 8 * int(rng.integers(0, 2))), 0x7FC1, dtype=np.uint16)
+    host[:, :cols] = bits
+    x = parity.to_device(host)[:, :cols]
+    n_pairs = int(rng.integers(1, 4))
+    ga = torch.tensor([orc.tensor_amax(bits)] * (2 * n_pairs), dtype=torch.float32, device="cuda") if supplied else None
+    stats = bool(seed % 2)
+    plan = mb.BatchPlan([x, x] * n_pairs, recipes * n_pairs, block_stats=stats, group_amax=ga)
+    plan.run()
+    plan.run()
+    torch.cuda.synchronize()
+    bits = np.ascontiguousarray(bits)
+    refs = [orc.run(bits, parity.oracle_block(r.block, cols), list(r.formats), r.criterion, r.threshold, r.scale_mode, r.flags)
+            for r in recipes]
+    for k, out in enumerate(plan.outs):
+        rep = parity.compare(bits, recipes[k & 1], out, refs[k & 1], check_block_stats=stats)
+        assert rep.n_exempt <= max(2, rep.n_blocks // 500)
