@@ -296,6 +296,33 @@ def main():
                          "whole_call_GBs": gbs, "frac_of_measured_copy": gbs / peak, "frac_of_8TBs": gbs / 8000.0})
         del so, sw
 
+    # ---- the same tensors wanted along the rows (1x128) and along the columns (128x1): one call with a pair of
+    #      entries per tensor (one read of each tile) against the two calls it replaces; whole calls
+    if rank == 0 and not args.no_variants:
+        nb2 = min(B, 8)
+        rr = mb.Recipe((1, 128), recipe.formats, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+        rc = mb.Recipe((128, 1), recipe.formats, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+        plans = {"one_call_us": [mb.BatchPlan([x for x in xs[:nb2] for _ in (0, 1)], [rr, rc] * nb2)],
+                 "two_calls_us": [mb.BatchPlan(xs[:nb2], [rr] * nb2), mb.BatchPlan(xs[:nb2], [rc] * nb2)]}
+        both = {"workload": "%d of the tensors, 1x128 and 128x1 blocks, two-way Eq.3" % nb2}
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for key, pl in plans.items():
+            for _ in range(3):
+                for q in pl:
+                    q.run(stream)
+            torch.cuda.synchronize()
+            tms = []
+            for _ in range(5):
+                ea.record(stream)
+                for q in pl:
+                    q.run(stream)
+                eb.record(stream)
+                torch.cuda.synchronize()
+                tms.append(ea.elapsed_time(eb) * 1e3)
+            both[key] = statistics.median(tms)
+        variants.append({"recipe": "rows and columns of the same tensors", **both})
+        del plans
+
     # ---- configs[0]: one 1024x1024 tensor, per-tensor partition: latency of a step, launched directly and
     #      replayed as a CUDA graph (the step is launch-bound at this size)
     small = None
