@@ -1165,7 +1165,7 @@ __device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control&
             scale_mode = p.b.t[m.ti].scale_mode;
             if (!dead) m_g = group_mantissa(*p.b.t[m.ti].amax, scale_mode);
         }
-#pragma unroll
+#pragma unroll 1
         for (int dir = 0; dir < 2; ++dir) {
             const TensorRec& R = p.b.t[m.ti + dir];
             const uint32_t b = (uint32_t)dir, n2 = it;        // conversion number 2 * it + dir
