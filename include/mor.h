@@ -113,6 +113,8 @@ typedef struct mor_tensor_desc {
                                mantissa: those read the tensor once)                         */
 } mor_tensor_desc_t;
 
+#define MOR_ERROR_BINS 12
+
 /* Per-block quantities behind the decisions (Eq. 3 sums, Eq. 4 range). */
 typedef struct mor_block_stats {
     float    amax;          /* max|x| over the block's finite elements                       */
@@ -171,6 +173,12 @@ typedef struct mor_outputs {
                                decision is taken for the whole tensor (tensor-level criterion,
                                (0,0) and (1,0) partitions) the E4M3 values are written: keep the
                                input instead when tensor_format says BF16                        */
+    uint32_t* error_histogram; /* optional, DEVICE, [MOR_ERROR_BINS] counters of the relative-error
+                               histogram of Section 4.1.3: the call adds one to the bin that holds the
+                               tensor's error of Eq. 1 (tensor_stats.mean_rel_e4m3).  Bin k covers
+                               [0.5 k %, 0.5 (k+1) %), the last bin everything from 5.5 % up.  The
+                               caller zeroes the counters when a period starts and may hand the same
+                               array to many calls (one row of the paper's heat map per tensor)      */
 } mor_outputs_t;
 
 /* Bytes of DEVICE scratch the calls below need for these `n` descriptors (one partial result per

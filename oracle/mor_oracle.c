@@ -483,6 +483,16 @@ static uint16_t f32_to_bf16_rne(float f)
 
 /* R11.  `sel` and `scale_f32` are the per-block results of orc_run (selected format and its
  * scale).  out has the layout of x with leading dimension out_ld. */
+/* Section 4.1.3: the relative-error histogram has bins of 0.5 %: bin k holds errors in
+ * [0.5 k %, 0.5 (k+1) %), the twelfth and last bin everything from 5.5 % up.  One tensor and
+ * mini-batch contribute one count. */
+int orc_error_bin(double mean_rel)
+{
+    int k = 0;
+    while (k < 11 && mean_rel >= 0.005 * (double)(k + 1)) ++k;
+    return k;
+}
+
 int orc_fake_quant(const orc_cfg_t* cfg, const uint16_t* x, const uint8_t* sel, const float* scale_f32,
                    uint16_t* out, int64_t out_ld)
 {

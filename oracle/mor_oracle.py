@@ -95,6 +95,8 @@ def lib():
         L.orc_run_blocks.argtypes = [C.POINTER(Cfg), C.c_void_p, C.c_void_p, C.c_int64,
                                      C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.POINTER(Tensor), C.c_int]
+        L.orc_error_bin.restype = C.c_int
+        L.orc_error_bin.argtypes = [C.c_double]
         L.orc_fake_quant.restype = C.c_int
         L.orc_fake_quant.argtypes = [C.POINTER(Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
         L.orc_scale_value.restype = C.c_float
@@ -222,6 +224,11 @@ def run(bits: np.ndarray, block, formats, criterion, threshold=0.045, scale_mode
         raise ValueError(f"oracle rejected the recipe (rc={rc})")
     td = {k: getattr(t, k) for k, _ in Tensor._fields_}
     return Result(codes, scale[:nb], sel[:nb], sf32[:nb], blocks[:n], td, grid, ids_arr)
+
+
+def error_bin(mean_rel: float) -> int:
+    """Bin of the 12-bin relative-error histogram (Section 4.1.3) that a tensor-level error falls into."""
+    return int(lib().orc_error_bin(float(mean_rel)))
 
 
 def fake_quant(bits: np.ndarray, res: Result, block, formats, criterion, threshold=0.045, scale_mode=SCALE_GAM,

@@ -32,6 +32,7 @@ MOR_FMT_E4M3, MOR_FMT_E5M2, MOR_FMT_BF16 = 0, 1, 2
 MOR_SCALE_GAM, MOR_SCALE_E8M0, MOR_SCALE_FP32_AMAX = 0, 1, 2
 MOR_CRIT_TENSOR_MEAN_REL, MOR_CRIT_BLOCK_VS_E5M2, MOR_CRIT_BLOCK_MEAN_REL = 0, 1, 2
 MOR_FLAG_STRICT_TIES, MOR_FLAG_RANGE_MIN_INCLUDES_ZERO = 1, 2
+MOR_ERROR_BINS = 12
 
 
 class MorError(RuntimeError):
@@ -64,7 +65,8 @@ class mor_tensor_stats_t(C.Structure):
 class mor_outputs_t(C.Structure):
     _fields_ = [("codes", C.c_void_p), ("codes_ld", C.c_int64), ("scale_e8m0", C.c_void_p),
                 ("sel", C.c_void_p), ("scale_f32", C.c_void_p), ("bf16_fallback", C.c_void_p),
-                ("block_stats", C.c_void_p), ("tensor_stats", C.c_void_p), ("fake_quant", C.c_void_p)]
+                ("block_stats", C.c_void_p), ("tensor_stats", C.c_void_p), ("fake_quant", C.c_void_p),
+                ("error_histogram", C.c_void_p)]
 
 
 class mor_stage_events_t(C.Structure):
@@ -250,6 +252,7 @@ class Outputs:
     scale_f32: object = None      # float32 [grid]
     bf16_fallback: object = None  # bfloat16, shaped like x
     fake_quant: object = None     # bfloat16, shaped like x
+    error_histogram: object = None  # the caller's 12 counters (Section 4.1.3), if given
     block_stats: object = None    # uint8 [n_blocks * 24]
     tensor_stats: object = None   # uint8 [80]
     cols: int = 0
@@ -273,7 +276,7 @@ class Outputs:
 
 
 def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, block_stats=False, fallback_like=None,
-                  scale_f32=False, fake_quant_like=None) -> Outputs:
+                  scale_f32=False, fake_quant_like=None, error_histogram=None) -> Outputs:
     import torch
 
     g = grid_of(rows, cols, recipe.block)
@@ -303,6 +306,10 @@ def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, b
     s.scale_f32 = o.scale_f32.data_ptr() if o.scale_f32 is not None and nb else None
     s.bf16_fallback = o.bf16_fallback.data_ptr() if o.bf16_fallback is not None else None
     s.fake_quant = o.fake_quant.data_ptr() if o.fake_quant is not None else None
+    if error_histogram is not None:      # the caller's counters (int32 or uint32, MOR_ERROR_BINS of them), kept across calls
+        assert error_histogram.numel() == MOR_ERROR_BINS and error_histogram.element_size() == 4 and error_histogram.is_cuda
+        o.error_histogram = error_histogram
+        s.error_histogram = error_histogram.data_ptr()
     s.block_stats = o.block_stats.data_ptr() if o.block_stats is not None else None
     s.tensor_stats = o.tensor_stats.data_ptr()
     return o
@@ -321,11 +328,12 @@ def _workspace(nbytes: int, device):
 
 
 def analyze_quantize(x, recipe: Recipe, *, cols=None, group_amax=None, block_stats=False, fallback=False,
-                     scale_f32=False, fake_quant=False, stream=None) -> Outputs:
+                     scale_f32=False, fake_quant=False, error_histogram=None, stream=None) -> Outputs:
     """Run mor_analyze_quantize on one BF16 CUDA tensor; allocates outputs and workspace."""
     d = desc_for(x, recipe, cols, group_amax)
     o = alloc_outputs(d.rows, d.cols, recipe, x.device, block_stats=block_stats,
-                      fallback_like=x if fallback else None, scale_f32=scale_f32, fake_quant_like=x if fake_quant else None)
+                      fallback_like=x if fallback else None, scale_f32=scale_f32, fake_quant_like=x if fake_quant else None,
+                      error_histogram=error_histogram)
     nbytes = mor_workspace_bytes([d])
     ws = _workspace(nbytes, x.device)
     st = mor_analyze_quantize(d, o.c_struct, ws.data_ptr(), ws.numel(), _stream_ptr(stream))
@@ -367,8 +375,9 @@ class BatchPlan:
     step is a single call of mor_analyze_quantize_batched."""
 
     def __init__(self, xs: Sequence, recipes: Sequence[Recipe], *, group_amax=None, block_stats=False,
-                 fallback=False, fake_quant=False):
-        """`fallback` and `fake_quant` are one flag for all tensors or one flag per tensor."""
+                 fallback=False, fake_quant=False, error_histograms=None):
+        """`fallback` and `fake_quant` are one flag for all tensors or one flag per tensor; `error_histograms`
+        is one tensor of MOR_ERROR_BINS 32-bit counters per tensor (or None)."""
         assert len(xs) == len(recipes) and len(xs) > 0
         self.xs = list(xs)
         self.group_amax = group_amax
@@ -382,7 +391,8 @@ class BatchPlan:
             descs.append(d)
             self.outs.append(alloc_outputs(d.rows, d.cols, r, x.device, block_stats=block_stats,
                                            fallback_like=x if fallback[i] else None,
-                                           fake_quant_like=x if fake_quant[i] else None))
+                                           fake_quant_like=x if fake_quant[i] else None,
+                                           error_histogram=None if error_histograms is None else error_histograms[i]))
         self.descs = (mor_tensor_desc_t * len(descs))(*descs)
         self.couts = (mor_outputs_t * len(descs))(*[o.c_struct for o in self.outs])
         self.n = len(descs)

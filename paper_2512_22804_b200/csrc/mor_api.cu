@@ -98,6 +98,7 @@ mor_status_t check_desc(const mor_tensor_desc_t& d, Shape& s)
 mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_outputs_t& o, bool store)
 {
     if (o.tensor_stats == nullptr) return MOR_ERR_INVALID_ARG;
+    if (o.error_histogram && !aligned(o.error_histogram, 4)) return MOR_ERR_ALIGNMENT;
     if (!aligned(o.tensor_stats, 8) || !aligned(o.block_stats, 4) || !aligned(o.scale_f32, 4)) return MOR_ERR_ALIGNMENT;
     if (s.kind == KIND_CHANNEL && o.block_stats != nullptr) return MOR_ERR_UNSUPPORTED;   // would need sums across tiles
     const bool empty = d.rows == 0 || d.cols == 0;
@@ -205,6 +206,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.fake_quant = static_cast<uint16_t*>(it.o.fake_quant);
     r.block_stats = it.o.block_stats;
     r.tensor_stats = it.o.tensor_stats;
+    r.hist = it.o.error_histogram;
     r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
@@ -522,6 +524,7 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
     if (host_desc->group_amax != nullptr) return MOR_ERR_INVALID_ARG;
     if (host_out->bf16_fallback != nullptr) return MOR_ERR_UNSUPPORTED;   // the fallback is the caller's own host tensor
     if (host_out->fake_quant != nullptr) return MOR_ERR_UNSUPPORTED;
+    if (host_out->error_histogram != nullptr) return MOR_ERR_UNSUPPORTED;  // a device array that outlives the call
     if (host_desc->block_rows == 128 && host_desc->block_cols == 1) return MOR_ERR_UNSUPPORTED;   // transposed codes: device entry points only
     if (host_desc->rows < 0 || host_desc->cols < 0 || host_desc->ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

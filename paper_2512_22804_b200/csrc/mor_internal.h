@@ -47,6 +47,7 @@ struct TensorRec {
     uint16_t* fake_quant;
     mor_block_stats_t* block_stats;
     mor_tensor_stats_t* tensor_stats;
+    uint32_t* hist;               // optional 12-bin histogram of the tensor-level error (Section 4.1.3)
     const float* amax;            // group amax on the device (workspace slot or the caller's)
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass

@@ -355,6 +355,12 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
             ts.status = *R.device_status ? MOR_ERR_TIMEOUT : MOR_OK;
             ts.n_blocks = n_blocks; ts.n_e4m3 = c[2]; ts.n_e5m2 = c[3]; ts.n_bf16 = c[4]; ts.n_nonfinite = c[1];
             *R.tensor_stats = ts;
+            if (R.hist) {
+                // Section 4.1.3: bins of 0.5 % of relative error, the last one open-ended
+                uint32_t bin = 0;
+                while (bin < MOR_ERROR_BINS - 1 && mean >= 0.005 * (double)(bin + 1)) ++bin;
+                atomicAdd(&R.hist[bin], 1u);
+            }
         }
         s_fmt = fmt;
         (void)s_tot;

@@ -419,6 +419,44 @@ def test_many_tensors_exceeding_one_launch():
         parity.compare(b, r, o, ref)
 
 
+def test_error_histogram_counts_one_per_tensor_and_call():
+    """Section 4.1.3: every call adds one count to the bin of the tensor's error; the counters persist
+    across calls and may be shared by the tensors of a batch."""
+    import torch
+
+    cases = [wl.weight_like(512, 512, seed=81), wl.gradient_like(384, 640, seed=82), wl.gaussian_outlier_rows(),
+             wl.activation_like(256, 512, seed=83), np.zeros((128, 128), dtype=np.uint16)]
+    hist = torch.zeros((mb.MOR_ERROR_BINS,), dtype=torch.int32, device="cuda")
+    want = np.zeros(mb.MOR_ERROR_BINS, dtype=np.int64)
+    r = recipe((128, 128), TWO)
+    for bits in cases:
+        out = mb.analyze_quantize(parity.to_device(bits), r, error_histogram=hist)
+        torch.cuda.synchronize()
+        ref = orc.run(bits, r.block, list(r.formats), r.criterion, r.threshold)
+        mean = ref.tensor["mean_rel_e4m3"]
+        edge = min(abs(mean - 0.005 * k) for k in range(1, 12))
+        assert edge > 1e-5 * max(mean, 1e-30), "a case on a bin edge proves nothing"
+        want[orc.error_bin(mean)] += 1
+        assert out.tensor_stats_dict()["status"] == 0
+    assert hist.cpu().numpy().tolist() == want.tolist() and want.sum() == len(cases)
+    assert len(set(np.nonzero(want)[0])) >= 3                          # the cases spread over several bins
+    # one shared row of counters for a whole batch, two steps
+    per = [torch.zeros((mb.MOR_ERROR_BINS,), dtype=torch.int32, device="cuda") for _ in cases[:4]]
+    plan = mb.BatchPlan([parity.to_device(b) for b in cases[:4]], [r] * 4, error_histograms=[hist] * 2 + per[2:])
+    plan.run()
+    plan.run()
+    torch.cuda.synchronize()
+    want2 = want.copy()
+    for i, bits in enumerate(cases[:4]):
+        ref = orc.run(bits, r.block, list(r.formats), r.criterion, r.threshold)
+        k = orc.error_bin(ref.tensor["mean_rel_e4m3"])
+        if i < 2:
+            want2[k] += 2
+        else:
+            assert per[i].cpu().numpy().tolist() == [2 if j == k else 0 for j in range(mb.MOR_ERROR_BINS)]
+    assert hist.cpu().numpy().tolist() == want2.tolist()
+
+
 def test_step_captured_as_cuda_graph_replays_identically():
     """BatchPlan.capture(): the memset and the three kernels as one CUDA graph; two replays, each checked
     against the oracle after the outputs were overwritten."""

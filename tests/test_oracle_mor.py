@@ -301,3 +301,24 @@ def test_unsupported_recipes_are_rejected():
         orc.run(x, (1, 128), [orc.FMT_E5M2, orc.FMT_E4M3, orc.FMT_BF16], orc.CRIT_BLOCK_VS_E5M2)
     with pytest.raises(ValueError):
         orc.run(x, (1, 128), THREE, orc.CRIT_TENSOR_MEAN_REL)
+
+
+def test_error_histogram_bins_of_section_4_1_3():
+    """Twelve bins of 0.5 % of relative error: the first below 0.5 %, the second from 0.5 % to below 1.0 %,
+    the last from 5.5 % up; the 4.5 % threshold is the left edge of the tenth bin."""
+    assert orc.error_bin(0.0) == 0 and orc.error_bin(0.0049999) == 0
+    assert orc.error_bin(0.005) == 1 and orc.error_bin(0.0099999) == 1
+    assert orc.error_bin(0.045) == 9 and orc.error_bin(0.0449999) == 8
+    assert orc.error_bin(0.0549999) == 10 and orc.error_bin(0.055) == 11
+    assert orc.error_bin(1.0) == 11 and orc.error_bin(37.5) == 11
+    # every bin is hit once by its midpoint, and the bin never decreases with the error
+    mids = [(k + 0.5) * 0.005 for k in range(12)]
+    assert [orc.error_bin(m) for m in mids] == list(range(12))
+    xs = np.linspace(0.0, 0.08, 2001)
+    bins = [orc.error_bin(float(x)) for x in xs]
+    assert all(b1 >= b0 for b0, b1 in zip(bins, bins[1:]))
+    # brute force against the definition with exact rationals (edges k/200)
+    from fractions import Fraction
+    for x in xs:
+        k = min(11, int(Fraction(float(x)) / Fraction(0.005)))
+        assert orc.error_bin(float(x)) == k
