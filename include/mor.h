@@ -41,8 +41,8 @@ typedef enum {
                                   the built-in array holds                                    */
 } mor_status_t;
 
-/* Representation types (Section 3: ordered "from most aggressive (e.g. E4M3) to least
- * aggressive (e.g. BF16)").  E4M3: 4 exponent / 3 mantissa bits, finite range 2^-9..448.
+/* Representation types.  Section 3 orders the candidates by how much precision they give up,
+ * E4M3 first and BF16 last.  E4M3: 4 exponent / 3 mantissa bits, finite range 2^-9..448.
  * E5M2: 5 / 2 bits, 2^-16..57344 (Sections 1-2).  Casts round to nearest even and
  * saturate to the largest finite value. */
 typedef enum { MOR_FMT_E4M3 = 0, MOR_FMT_E5M2 = 1, MOR_FMT_BF16 = 2 } mor_format_t;
@@ -60,7 +60,7 @@ typedef enum { MOR_SCALE_GAM = 0, MOR_SCALE_E8M0 = 1, MOR_SCALE_FP32_AMAX = 2 } 
 /* Acceptance metric for E4M3.
  *   TENSOR_MEAN_REL  Section 3.1, Eq. 1-2: one decision for the whole tensor; mean over its
  *                    non-zero elements of |x - Q(x)| / |x| must be < threshold.  The scales
- *                    may still be per block ("aggregate the local errors into the global").
+ *                    may still be per block: the block sums are added up into the tensor's error.
  *   BLOCK_VS_E5M2    Section 3.2, Eq. 3: per block, E4M3 is kept when its summed relative
  *                    error does not exceed that of E5M2.  With three formats a rejected
  *                    block takes E5M2 when Eq. 4 holds (max|b|/min|b| < 57344/2^-14).
@@ -227,7 +227,7 @@ mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_block_stat
                               mor_tensor_stats_t* tensor_stats, uint8_t* sel, uint8_t* scale_e8m0,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* Step "g_amax <- max(abs(g))" of Algorithm 1 alone, with the whole tensor as the group:
+/* The first step of Algorithm 1 alone (the group's largest magnitude), with the whole tensor as the group:
  * writes max|x| over finite elements of tensor i to amax_out[i] (DEVICE, n floats), so
  * that later calls can pass it as group_amax. */
 mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* amax_out,

@@ -16,8 +16,8 @@
  *
  * The method is its own definition (it approximates nothing else), so the oracle takes
  * the algorithm's steps in the paper's order, one element at a time, with every sum in
- * double.  Two quantities are FP32 by the paper's wording ("ideal FP32 scaling factor",
- * Section 2): the scale q_amax/amax and the scaled value x*scale that is then rounded
+ * double.  Two quantities are FP32 by the paper's wording (Section 2 calls the scaling factor
+ * an FP32 number): the scale q_amax/amax and the scaled value x*scale that is then rounded
  * to FP8.  Both are formed here as one correctly rounded FP32 operation.
  *
  * FP8 encoding is done from the format definition: the table of finite values is built
@@ -195,7 +195,7 @@ uint8_t orc_encode_e5m2_exhaustive(float y) { return encode_with_table(y, tab_e5
 
 #define Q_AMAX_E4M3 448.0f
 
-/* "ideal FP32 scaling factor" q_amax / amax: one binary32 division.  R5: an overflowing
+/* Algorithm 1's FP32 scaling factor q_amax / amax: one binary32 division.  R5: an overflowing
  * quotient is replaced by the largest finite binary32. */
 static float ideal_scale(float q_amax, float amax)
 {

@@ -1,6 +1,6 @@
 // The two small kernels around the fused main kernel (mor_main.cu).
 //
-//   mor_amax_kernel      Algorithm 1, "g_amax <- max(abs(g))" with the tensor as one group
+//   mor_amax_kernel      Algorithm 1, first step: the largest magnitude of the group, the tensor being one group
 //   mor_finalise_kernel  tensor-wide aggregate of the per-tile partials and the Eq. 2 decision
 #include <cuda_bf16.h>
 #include <float.h>
@@ -17,7 +17,7 @@ struct WarpPart {
     uint32_t nnz, nonfinite, n4, n5, nb, mn;
 };
 
-// "ideal FP32 scaling factor" 448 / amax: one IEEE division; a quotient above the largest
+// Algorithm 1's binary32 scaling factor 448 / amax: one IEEE division; a quotient above the largest
 // finite binary32 is replaced by it
 __device__ __forceinline__ uint32_t ideal_scale_bits(float amax)
 {
@@ -103,7 +103,7 @@ __device__ __noinline__ uint2 key_of_chunk_finite(uint4 v)
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
 
 // One 128 x 128 tile per CTA (the tiling of the main kernel); 16-byte loads straight to registers,
-// 16 lanes per 256-byte row piece.  Results: the tensor's amax (Algorithm 1, "g_amax <- max(abs(g))"
+// 16 lanes per 256-byte row piece.  Results: the tensor's amax (Algorithm 1, first step,
 // with the tensor as one group) by atomicMax, the count of NaN/inf elements, and, when the tensor
 // record has a key array, the key of every row piece of the tile (1x128 partition: that is the
 // block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main

@@ -274,7 +274,7 @@ __device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, un
 
 // ------------------------------------------------------------------ Algorithm 1 ----
 
-// "ideal FP32 scaling factor" 448 / amax by one IEEE division; a quotient above the largest
+// Algorithm 1's binary32 scaling factor 448 / amax by one IEEE division; a quotient above the largest
 // finite binary32 is replaced by it
 __device__ __forceinline__ uint32_t ideal_scale_bits_div(float amax)
 {
