@@ -127,7 +127,7 @@ def run_reference(args, rank):
     line = {"impl": "reference", "metric": "analyse+quantise throughput (algorithmic bytes)", "value": gbs, "unit": "GB/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "BASELINE configs[1]: 4096x4096 weight-like BF16, 128x128 blocks, [E4M3,BF16] vs E5M2",
+            "config": {"workload": "configs[1]: 4096x4096 weight-like BF16, 128x128 blocks, [E4M3,BF16] vs E5M2",
                        "sample": f"first {sample_rows} rows of one tensor per step"},
             "elements_per_s": el / dt,
             "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
@@ -331,7 +331,7 @@ def main():
         sx = torch.from_numpy(sb.view(np.int16)).view(torch.bfloat16).to(dev)
         sp = mb.BatchPlan([sx], [mb.Recipe((0, 0), recipe.formats, mb.MOR_CRIT_TENSOR_MEAN_REL, 0.045)])
         graph = sp.capture()
-        small = {"workload": "BASELINE configs[0]: one 1024x1024 tensor, per-tensor partition, Eq.2"}
+        small = {"workload": "configs[0]: one 1024x1024 tensor, per-tensor partition, Eq.2"}
         for key, fn in (("direct_us", lambda: sp.run(torch.cuda.current_stream())), ("cuda_graph_us", graph.replay)):
             for _ in range(5):
                 fn()
@@ -424,7 +424,7 @@ def main():
         line = {"metric": "analyse+quantise throughput (algorithmic bytes)", "value": value, "unit": "GB/s",
                 "n_gpus": world, "steps": K, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": "BASELINE configs[1]: 4096x4096 weight-like BF16 N(0,0.02) x per-column 10^U(-1,1), "
+                "config": {"workload": "configs[1]: 4096x4096 weight-like BF16 N(0,0.02) x per-column 10^U(-1,1), "
                                        "128x128 blocks, candidates [E4M3,BF16], Eq.3 against E5M2, GAM scaling",
                            "tensors_per_step_per_gpu": B, "elements_per_step_per_gpu": elements,
                            "l2": "inputs (512 MiB per step at the default batch) exceed L2; no flush needed",
@@ -434,7 +434,7 @@ def main():
                 "fp8_block_fraction": fp8_frac, "fp8_tensor_fraction_eq2": tensor_fp8,
                 "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "other_recipes_same_tensors": variants, "small_tensor_latency": small,
                 "paper_context": "the paper reports no throughput and names no hardware; its own figures are FP8 tensor fractions "
-                                 "(98.38 % / 95.93 % per channel, tensor-level MoR, Nemotron-3 8B), see BASELINE.md",
+                                 "(98.38 % / 95.93 % per channel, tensor-level MoR, Nemotron-3 8B)",
                 "gpu_launches": 3 * K, "clocks": clocks}
         print(json.dumps(line), flush=True)
     if world > 1:
