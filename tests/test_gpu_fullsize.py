@@ -116,3 +116,29 @@ def test_config4_llama_layer_one_batched_call():
         ts = o.tensor_stats_dict()
         assert ts["n_blocks"] == nb == ts["n_e4m3"] + ts["n_e5m2"] + ts["n_bf16"], c.name
         assert ts["nnz"] == int(np.count_nonzero(c.bits & 0x7FFF)), c.name
+
+
+@pytest.mark.parametrize("block,formats", [((128, 128), TWO), ((1, 128), THREE)])
+def test_tensor_with_more_than_2_31_elements(block, formats):
+    """70000 x 33000 (2.31 G elements, 4.6 GB): element offsets pass 2^31 and 2^32 bytes.  Sampled blocks, among
+    them the first, the middle and the last ones, against the oracle; counts over the whole tensor."""
+    import torch
+
+    rows, cols = 70000, 33000
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    x = (torch.randn((rows, cols), device="cuda", generator=gen, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+    x[rows - 1, cols - 1] = 3.0                     # the amax sits at the very end
+    x[12345, 6789] = 0.0
+    host = x.view(torch.int16).cpu().numpy().view(np.uint16)
+    r = mb.Recipe(block, formats, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+    out = mb.analyze_quantize(x, r, block_stats=True, scale_f32=True)
+    torch.cuda.synchronize()
+    ts = out.tensor_stats_dict()
+    grid = mb.grid_of(rows, cols, block)
+    nb = grid[0] * grid[1]
+    rng = np.random.default_rng(3)
+    ids = np.unique(np.concatenate([rng.choice(nb, 200, replace=False), [0, nb - 1, nb - 2, nb // 2]]))
+    ref = orc.run(host, block, list(formats), r.criterion, r.threshold, ids=ids)
+    parity.compare(host, r, out, ref, ids=ids)
+    assert ts["n_blocks"] == nb == ts["n_e4m3"] + ts["n_e5m2"] + ts["n_bf16"] and ts["status"] == 0
+    assert ts["group_amax"] == 3.0 and ts["nnz"] == int(torch.count_nonzero(x).item())
