@@ -1,6 +1,7 @@
 // Host side of the C boundary: argument checks, workspace layout, grouping of tensors by
 // partition kind and launch sequence.  No device code lives here.
 #include <cmath>
+#include <atomic>
 #include <cstring>
 #include <vector>
 
@@ -127,13 +128,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 EncodeTiledFn encode_tiled_fn()
 {
-    static EncodeTiledFn fn = nullptr;
+    static std::atomic<EncodeTiledFn> cached{nullptr};   // host threads may race here: every one stores the same address
+    EncodeTiledFn fn = cached.load(std::memory_order_acquire);
     if (fn == nullptr) {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
+            q == cudaDriverEntryPointSuccess) {
             fn = reinterpret_cast<EncodeTiledFn>(p);
+            cached.store(fn, std::memory_order_release);
+        }
     }
     return fn;
 }

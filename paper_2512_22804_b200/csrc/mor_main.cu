@@ -33,6 +33,9 @@
 #include <cuda_fp16.h>
 #include <float.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "mor_internal.h"
 
 namespace mor {
@@ -1308,20 +1311,23 @@ template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
 cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
 {
     auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE, SCAN>;
-    static bool configured[64] = {};   // per instantiation and device
-    static int sm_count[64] = {};
+    static std::atomic<int> sm_count[64];   // per instantiation and device; 0 = not set up yet
+    static std::mutex setup;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!configured[dev]) {
+    int sms = sm_count[dev].load(std::memory_order_acquire);
+    if (sms == 0) {
+        std::lock_guard<std::mutex> lock(setup);         // host threads may make their first call together
         e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        if (sms <= 0) return cudaErrorInvalidDevice;
+        sm_count[dev].store(sms, std::memory_order_release);
     }
-    const uint32_t resident = 2u * (uint32_t)sm_count[dev];
+    const uint32_t resident = 2u * (uint32_t)sms;
     const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
     return launch_dependent(kfn, dim3(grid), dim3(kMainThreads), (size_t)kSmemBytes, s, p, partials);
 }
