@@ -457,6 +457,42 @@ def test_error_histogram_counts_one_per_tensor_and_call():
     assert hist.cpu().numpy().tolist() == want2.tolist()
 
 
+def test_two_host_threads_on_two_streams():
+    """Calls from two host threads, each with its own stream, tensors, outputs and workspace, may overlap on the
+    host and on the GPU; every result equals the single-threaded one."""
+    import threading
+
+    import torch
+
+    cases = [(wl.gradient_like(700, 1024, seed=91), recipe((1, 128), THREE)),
+             (wl.weight_like(900, 768, seed=92), recipe((128, 128), TWO))]
+    xs = [parity.to_device(b) for b, _ in cases]
+    want = [mb.analyze_quantize(x, r, block_stats=True) for x, (_, r) in zip(xs, cases)]
+    torch.cuda.synchronize()
+    plans = [mb.BatchPlan([x], [r], block_stats=True) for x, (_, r) in zip(xs, cases)]
+    streams = [torch.cuda.Stream() for _ in cases]
+    errors = []
+
+    def work(i):
+        try:
+            for _ in range(50):
+                plans[i].run(streams[i])
+            streams[i].synchronize()
+        except Exception as e:      # noqa: BLE001
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for p, w in zip(plans, want):
+        o = p.outs[0]
+        assert o.tensor_stats_dict() == w.tensor_stats_dict() and o.tensor_stats_dict()["status"] == 0
+        assert torch.equal(o.codes, w.codes) and torch.equal(o.sel, w.sel) and torch.equal(o.block_stats, w.block_stats)
+
+
 def test_step_captured_as_cuda_graph_replays_identically():
     """BatchPlan.capture(): the memset and the three kernels as one CUDA graph; two replays, each checked
     against the oracle after the outputs were overwritten."""
