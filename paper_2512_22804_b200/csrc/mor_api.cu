@@ -223,7 +223,7 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
     r.tile_begin = it.tile_begin;
     r.criterion = d.criterion; r.scale_mode = d.scale_mode; r.n_formats = d.n_formats;
-    r.flags = d.flags; r.threshold = d.threshold;
+    r.flags = d.flags | (it.prepass ? kFlagAmaxFinal : 0u); r.threshold = d.threshold;
 }
 
 inline bool same_variant(const MainVariant& a, const MainVariant& b)

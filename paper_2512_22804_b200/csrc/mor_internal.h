@@ -69,6 +69,10 @@ struct TensorRec {
     float threshold;
 };
 
+// Internal bit of TensorRec::flags (the public MOR_FLAG_* bits are the low ones): the amax pre-pass ran for this
+// tensor, so its amax slot is final and the main kernel need not gather the tensor amax.
+constexpr uint32_t kFlagAmaxFinal = 0x80000000u;
+
 struct BatchParams {
     int n;
     uint32_t tile_end[kMaxBatch]; // exclusive prefix of tiles within this launch

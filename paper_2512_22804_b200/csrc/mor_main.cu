@@ -987,8 +987,10 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
             // patterns order like the values)
-            const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
-            raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
+            if (!(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot) {
+                const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
+                raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
+            }
         } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
             key = scan_words(w);
             uint32_t tile_amax = 0u;
@@ -1022,7 +1024,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = scan_words_finite(w);
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here
-            raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead);
+            raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead && !(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot);
         } else {
             key = scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
@@ -1211,7 +1213,7 @@ __device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control&
                 }
                 if (dir == 0) {                             // no pre-pass ran: gather the tensor amax for the summaries
                     const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
-                    raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
+                    raise_amax(R.amax_slot, wamax, lane == 0 && !dead && R.amax == R.amax_slot);
                 }
             }
             const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
