@@ -520,6 +520,7 @@ int orc_fake_quant(const orc_cfg_t* cfg, const uint16_t* x, const uint8_t* sel, 
 
 /* Element-level helpers exported for the pins. */
 float orc_scale_value(float x, float scale) { return scale_value(x, scale); }
+uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
 double orc_rel_err_e4m3(float y) { return rel_err(y, orc_decode_e4m3(orc_encode_e4m3(y))); }
 double orc_rel_err_e5m2(float y) { return rel_err(y, orc_decode_e5m2(orc_encode_e5m2(y))); }
 int orc_sizeof_cfg(void) { return (int)sizeof(orc_cfg_t); }

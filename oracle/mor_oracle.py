@@ -19,6 +19,10 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "mor_oracle.c")
 _LIB = os.path.join(_HERE, "libmor_oracle.so")
+# The pins are themselves tested by running them against deliberately wrong copies of the C file
+# (tests/test_oracle_planted_mistakes.py); such a run names the source and the library to use here.
+if os.environ.get("MOR_ORACLE_SRC") and os.environ.get("MOR_ORACLE_LIB"):
+    _SRC, _LIB = os.environ["MOR_ORACLE_SRC"], os.environ["MOR_ORACLE_LIB"]
 
 FMT_E4M3, FMT_E5M2, FMT_BF16 = 0, 1, 2
 CRIT_TENSOR_MEAN_REL, CRIT_BLOCK_VS_E5M2, CRIT_BLOCK_MEAN_REL = 0, 1, 2
@@ -101,6 +105,8 @@ def lib():
         L.orc_fake_quant.argtypes = [C.POINTER(Cfg), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
         L.orc_scale_value.restype = C.c_float
         L.orc_scale_value.argtypes = [C.c_float, C.c_float]
+        L.orc_f32_to_bf16.restype = C.c_uint16
+        L.orc_f32_to_bf16.argtypes = [C.c_float]
         for n in ("orc_rel_err_e4m3", "orc_rel_err_e5m2"):
             getattr(L, n).restype = C.c_double
             getattr(L, n).argtypes = [C.c_float]
@@ -141,6 +147,11 @@ def block_scale(b_amax: float, m_g: int, scale_mode: int = SCALE_GAM):
 
 def scale_value(x: float, scale: float) -> float:
     return lib().orc_scale_value(x, scale)
+
+
+def f32_to_bf16(f: float) -> int:
+    """BF16 bits of a binary32 value, round to nearest even (the last step of fake quantisation)."""
+    return lib().orc_f32_to_bf16(f)
 
 
 def rel_err_e4m3(y: float) -> float:

@@ -261,6 +261,13 @@ def test_block_mean_rel_criterion():
     means = r.blocks["sum_rel_e4m3"] / r.blocks["nnz"]
     assert means[0] < 0.045 < means[1]
     assert list(r.sel) == [orc.FMT_E4M3, orc.FMT_BF16]
+    # Eq. 2 on a block is strict as well: one exact element (2.0 -> 448) and one flushed element give a block
+    # mean of exactly 0.5, which a threshold of 0.5 rejects and the next larger threshold accepts
+    two = bf16(np.array([[2.0, 2.0 ** -20]]))
+    r = orc.run(two, (1, 128), TWO, orc.CRIT_BLOCK_MEAN_REL, threshold=0.5)
+    assert r.blocks["sum_rel_e4m3"][0] == 1.0 and list(r.sel) == [orc.FMT_BF16]
+    r = orc.run(two, (1, 128), TWO, orc.CRIT_BLOCK_MEAN_REL, threshold=0.5000001)
+    assert list(r.sel) == [orc.FMT_E4M3]
 
 
 def test_ragged_edges_behave_like_absent_elements():
