@@ -23,6 +23,13 @@
 #include <stddef.h>
 #include <stdint.h>
 
+/* The library is built with hidden symbol visibility; only the entry points below are exported. */
+#if defined(__GNUC__)
+#define MOR_API __attribute__((visibility("default")))
+#else
+#define MOR_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -182,16 +189,16 @@ typedef struct mor_outputs {
 } mor_outputs_t;
 
 /* Bytes of DEVICE scratch the calls below need for these `n` descriptors (one partial result per
- * 128 x 128 tile, block keys handed from the amax pre-pass to the main kernel, one amax slot and
- * one counter per tensor, one status word).  Only shapes and block shapes are read.  Returns 0 on
+ * 128 x 128 tile, block keys handed from the amax pre-pass to the main kernel, one amax slot per
+ * tensor, one status word).  Only shapes and block shapes are read.  Returns 0 on
  * a NULL or negative argument.  The scratch needs no initialisation and 256-byte alignment. */
-size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n);
+MOR_API size_t mor_workspace_bytes(const mor_tensor_desc_t* host_descs, int n);
 
 /* Section 3, Algorithm 2 on one tensor: block amax, GAM scale, cast to E4M3 (and E5M2),
  * relative-error sums, per-block or per-tensor decision; writes codes, scales, selection,
  * optional BF16 copies and statistics.  Launches: tensor amax (unless supplied), the fused
  * main kernel, a small finalise kernel. */
-mor_status_t mor_analyze_quantize(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+MOR_API mor_status_t mor_analyze_quantize(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                   void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* The same analysis for `n` tensors with one set of launches per block shape.
@@ -201,7 +208,7 @@ mor_status_t mor_analyze_quantize(const mor_tensor_desc_t* host_desc, const mor_
  * fake-quantised output on the first, are served by one main kernel that reads every tile of the tensor
  * once and converts it along the rows and along the columns; every output equals that of two separate
  * calls. */
-mor_status_t mor_analyze_quantize_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
+MOR_API mor_status_t mor_analyze_quantize_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
                                           int n, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Optional CUDA events (cudaEvent_t passed as void*, created and owned by the caller, NULL to
@@ -216,21 +223,21 @@ typedef struct mor_stage_events {
 } mor_stage_events_t;
 
 /* mor_analyze_quantize_batched plus stage events (host_events may be NULL). */
-mor_status_t mor_analyze_quantize_batched_ex(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
+MOR_API mor_status_t mor_analyze_quantize_batched_ex(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs,
                                              int n, void* workspace, size_t workspace_bytes, void* cuda_stream,
                                              const mor_stage_events_t* host_events);
 
 /* Decisions and statistics only (Eq. 1-4 evaluated, nothing quantised out): reads the
  * tensor, writes `tensor_stats` and, when non-NULL, `block_stats`, `sel`, `scale_e8m0`.
  * Serves threshold calibration and the per-tensor error statistics of Section 4.1.3. */
-mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_block_stats_t* block_stats,
+MOR_API mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_block_stats_t* block_stats,
                               mor_tensor_stats_t* tensor_stats, uint8_t* sel, uint8_t* scale_e8m0,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* The first step of Algorithm 1 alone (the group's largest magnitude), with the whole tensor as the group:
  * writes max|x| over finite elements of tensor i to amax_out[i] (DEVICE, n floats), so
  * that later calls can pass it as group_amax. */
-mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* amax_out,
+MOR_API mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* amax_out,
                             void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* End-to-end variant for data that lives in HOST memory: copies the tensor to the device,
@@ -239,8 +246,8 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
  * In `host_desc` and `host_out` every data pointer is a HOST pointer here (pinned memory
  * makes the copies asynchronous); host_desc->group_amax must be NULL.  `device_staging`
  * is DEVICE scratch of at least mor_host_staging_bytes() bytes. */
-size_t mor_host_staging_bytes(const mor_tensor_desc_t* host_desc);
-mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+MOR_API size_t mor_host_staging_bytes(const mor_tensor_desc_t* host_desc);
+MOR_API mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                        void* device_staging, size_t staging_bytes, void* cuda_stream);
 
 /* No counterpart in the paper: a packaging variant of mor_analyze_quantize for callers that cannot
@@ -255,16 +262,19 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
  *     per block), so the limit is roughly 600 M elements, or 62 M elements for (1,128); larger
  *     tensors are refused with MOR_ERR_STATIC_SCRATCH and nothing is launched.
  *   - The first call on each device looks up the array's device address (with that device
- *     current); make that first call outside any stream capture.
+ *     current) and keeps it for the life of the process; make that first call outside any stream
+ *     capture.  The address belongs to the device that is current at the call, which must be the
+ *     device of `cuda_stream`.  After a cudaDeviceReset() the remembered address is stale: a process
+ *     that resets a device must not use this entry point on it afterwards.
  *   - All calls share the one array, and it keeps what the previous call left in it; the call
  *     clears the part that has to start at zero.  Two calls whose kernels overlap on the GPU
  *     (different streams, no ordering between them) race on it: order them.  */
 #define MOR_STATIC_SCRATCH_BYTES (2 * 1024 * 1024)
-mor_status_t mor_analyze_quantize_static(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
+MOR_API mor_status_t mor_analyze_quantize_static(const mor_tensor_desc_t* host_desc, const mor_outputs_t* host_out,
                                          void* cuda_stream);
 
-const char* mor_status_string(mor_status_t status);
-int mor_version(void);
+MOR_API const char* mor_status_string(mor_status_t status);
+MOR_API int mor_version(void);
 
 #ifdef __cplusplus
 }

@@ -170,15 +170,14 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
 }
 
 struct Layout {
-    size_t amax_off, nonf_off, status_off, partial_off, keys_off, total;
+    size_t amax_off, status_off, partial_off, keys_off, total;
 };
 
 Layout layout_of(int n, uint64_t tiles, uint64_t key_words)
 {
     Layout l;
     l.amax_off = 0;
-    l.nonf_off = (size_t)n * sizeof(float);
-    l.status_off = 2 * (size_t)n * sizeof(float);
+    l.status_off = (size_t)n * sizeof(float);
     l.partial_off = round_up(l.status_off + sizeof(uint32_t), kAlign);
     l.keys_off = l.partial_off + round_up((size_t)tiles * sizeof(Partial), kAlign);
     l.total = l.keys_off + round_up((size_t)key_words * sizeof(uint32_t), kAlign);
@@ -213,7 +212,6 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.hist = it.o.error_histogram;
     r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
-    r.nonfinite_slot = reinterpret_cast<uint32_t*>(ws + l.nonf_off) + it.index;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
     r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
     r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kTileRows : 4u;
@@ -271,6 +269,12 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     if (!aligned(workspace, kAlign)) return MOR_ERR_ALIGNMENT;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     Partial* partials = reinterpret_cast<Partial*>(ws + l.partial_off);
+    // every TMA descriptor is encoded before anything is enqueued: a call that fails here has launched nothing
+    std::vector<CUtensorMap> in_maps((size_t)n), out_maps((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        if (items[i].s.n_tiles == 0) continue;
+        if (!encode_maps(*items[i].d, items[i].o, items[i].v.store, in_maps[i], out_maps[i])) return MOR_ERR_CUDA;
+    }
 
     // 1. Algorithm 1, group amax, for the tensors whose caller did not supply it
     if (ev && !record(ev->amax_begin)) return MOR_ERR_CUDA;
@@ -331,7 +335,8 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
                 bp.tile_end[bp.n++] = t_end;
             } else {
                 fill_rec(items[j], ws, l, bp.t[bp.n]);
-                if (!encode_maps(*items[j].d, items[j].o, v.store, mp.in_map[bp.n], mp.out_map[bp.n])) return MOR_ERR_CUDA;
+                mp.in_map[bp.n] = in_maps[j];
+                mp.out_map[bp.n] = out_maps[j];
                 if (items[j].dual == 2) {
                     // the columns' record shares the tiles and the group amax of the rows' record before it
                     if (items[j].d->group_amax == nullptr) bp.t[bp.n].amax = bp.t[bp.n - 1].amax_slot;
@@ -459,6 +464,17 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
     if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
     if (!aligned(workspace, kAlign) || !aligned(amax_out, 4)) return MOR_ERR_ALIGNMENT;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
+    // only the geometry matters here (pointer, shape, pitch, alignment); every descriptor is checked before
+    // anything is enqueued
+    std::vector<Shape> shapes((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        const mor_tensor_desc_t& d = host_descs[i];
+        const mor_status_t st = shape_of(d, shapes[i]);
+        if (st != MOR_OK) return st;
+        if (d.ld < d.cols) return MOR_ERR_INVALID_ARG;
+        if (d.ld % 8 != 0 || !aligned(d.x, 16)) return MOR_ERR_ALIGNMENT;
+        if (d.rows != 0 && d.cols != 0 && d.x == nullptr) return MOR_ERR_INVALID_ARG;
+    }
     if (cudaMemsetAsync(ws, 0, l.partial_off, stream) != cudaSuccess) return MOR_ERR_CUDA;
     BatchParams bp;
     bp.n = 0;
@@ -467,8 +483,7 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         Item it;
         mor_tensor_desc_t d = host_descs[i];
         d.group_amax = nullptr;
-        mor_status_t st = check_desc(d, it.s);
-        if (st != MOR_OK) return st;
+        it.s = shapes[i];
         std::memset(&it.o, 0, sizeof(it.o));
         it.d = &d; it.index = i; it.tile_begin = 0; it.key_begin = 0; it.prepass = false;   // no keys wanted
         if (it.s.n_tiles) {

@@ -50,7 +50,6 @@ struct TensorRec {
     uint32_t* hist;               // optional 12-bin histogram of the tensor-level error (Section 4.1.3)
     const float* amax;            // group amax on the device (workspace slot or the caller's)
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
-    uint32_t* nonfinite_slot;     // workspace: element count of NaN/inf found by the amax pre-pass
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
     uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows

@@ -104,7 +104,7 @@ __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __v
 
 // One 128 x 128 tile per CTA (the tiling of the main kernel); 16-byte loads straight to registers,
 // 16 lanes per 256-byte row piece.  Results: the tensor's amax (Algorithm 1, first step,
-// with the tensor as one group) by atomicMax, the count of NaN/inf elements, and, when the tensor
+// with the tensor as one group) by atomicMax and, when the tensor
 // record has a key array, the key of every row piece of the tile (1x128 partition: that is the
 // block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main
 // kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its elements (the key itself
@@ -244,7 +244,6 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
         // (atomics on one address are served one at a time: read first, most tiles end there)
         unsigned int* slot = reinterpret_cast<unsigned int*>(R.amax_slot);
         if (__ldcg(slot) < ((kk >> 16) << 16)) atomicMax(slot, (kk >> 16) << 16);
-        if (nf) atomicAdd(R.nonfinite_slot, nf);
     }
 }
 
@@ -276,7 +275,6 @@ __global__ void __launch_bounds__(kThreads)
 mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __restrict__ partials)
 {
     __shared__ WarpPart s_wp[kThreads / 32];
-    __shared__ WarpPart s_tot;
     pdl_wait();                                          // the main kernel's partials and outputs are complete
     const TensorRec& R = p.t[blockIdx.x];
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -363,7 +361,6 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
             }
         }
         s_fmt = fmt;
-        (void)s_tot;
     }
     __syncthreads();
     if (KIND != KIND_TENSOR && R.criterion == MOR_CRIT_TENSOR_MEAN_REL && R.sel) {

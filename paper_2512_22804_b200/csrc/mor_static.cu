@@ -5,7 +5,7 @@
 // inside somebody else's runtime that owns all device memory, a real-time loop in which an
 // allocation's implicit device synchronisation is not acceptable, a process whose memory
 // budget was fixed at start-up.  Such a caller still owns its inputs and outputs; only the
-// scratch (an amax slot and a counter, then per 32 KiB tile of input one 40-byte partial result and
+// scratch (an amax slot and a status word, then per 32 KiB tile of input one 40-byte partial result and
 // the block keys that the amax pre-pass hands to the main kernel) comes from here.
 #include <mutex>
 

@@ -31,6 +31,17 @@ def test_every_declared_entry_point_is_exported(lib):
         assert getattr(lib, n) is not None
 
 
+def test_nothing_but_the_declared_entry_points_is_exported(lib):
+    """The dynamic symbol table holds the mor_* functions of the header and nothing else of this library's
+    own code (the CUDA runtime that is linked in statically may add names of its own)."""
+    import subprocess
+
+    out = subprocess.run(["nm", "-D", "--defined-only", mb.LIB_PATH], capture_output=True, text=True, check=True).stdout
+    names = [line.split()[-1] for line in out.splitlines() if line.strip()]
+    ours = [n for n in names if not n.startswith(("cuda", "__cuda", "_init", "_fini", "__bss_start", "_edata", "_end"))]
+    assert sorted(ours) == declared_functions(), ours
+
+
 def test_version_and_status_strings(lib):
     assert mb.mor_version() >= 100
     seen = {mb.mor_status_string(s) for s in range(0, 8)}
@@ -103,6 +114,35 @@ def test_misaligned_workspace_is_rejected(lib):
     need = mb.mor_workspace_bytes([d])
     assert mb.mor_analyze_quantize(d, out_struct(), 0x10010, need) == mb.MOR_ERR_ALIGNMENT
     assert mb.mor_analyze_quantize(d, out_struct(), 0x10000, need - 1) == mb.MOR_ERR_WORKSPACE
+
+
+def test_group_amax_checks_every_descriptor_before_it_launches(lib):
+    """A bad descriptor anywhere in the list is reported although the first ones are fine; only the geometry is
+    looked at (formats, criterion and threshold play no part in an amax)."""
+    import ctypes as C
+
+    good, bad = desc(), desc(ld=260)
+    arr = (mb.mor_tensor_desc_t * 2)(good, bad)
+    assert lib.mor_group_amax(arr, 2, C.c_void_p(0x6000), C.c_void_p(0x10000), 1 << 20, None) == mb.MOR_ERR_ALIGNMENT
+    odd = desc()
+    odd.n_formats = 9                                                        # not looked at by this entry point
+    odd.rows = -1
+    arr = (mb.mor_tensor_desc_t * 1)(odd)
+    assert lib.mor_group_amax(arr, 1, C.c_void_p(0x6000), C.c_void_p(0x10000), 1 << 20, None) == mb.MOR_ERR_INVALID_ARG
+
+
+def test_static_scratch_refuses_tensors_beyond_its_limit(lib):
+    """The size check of mor_analyze_quantize_static comes before any CUDA call, so it can be exercised
+    without a device: nothing is looked up, nothing is launched."""
+    r = mb.Recipe((128, 128), (0, 2))
+    rows = cols = 128 * 200                                              # 40,000 tiles * 56 B > 2 MiB
+    d = mb.make_desc(0x10000, rows, cols, cols, r)
+    assert mb.mor_workspace_bytes([d]) > mb.MOR_STATIC_SCRATCH_BYTES
+    o = mb.mor_outputs_t()
+    o.codes, o.codes_ld, o.tensor_stats, o.scale_e8m0, o.sel = 0x20000, cols, 0x30000, 0x40000, 0x50000
+    st = mb.mor_analyze_quantize_static(d, o, 0)
+    assert st == mb.MOR_ERR_STATIC_SCRATCH
+    assert "built-in" in mb.mor_status_string(st)
 
 
 def test_null_descriptors(lib):

@@ -170,6 +170,22 @@ def test_fake_quant_output(block):
         parity.run_and_compare(g, r, pad_to=1008, block_stats=False, fake_quant=True, group_amax_supplied=True)
 
 
+def test_fake_quant_where_the_last_rounding_is_a_tie():
+    """FP32-amax scaling with a block amax of 133 * 2^p makes the scale fl32(64/19) * 2^-p; elements cast to the
+    E4M3 value 15 * 2^j then de-scale to 285 * 2^(j-6), exactly half way between two BF16 numbers, so the
+    round-to-nearest-even of the BF16 conversion decides the output bits for over a hundred elements here."""
+    from tests.test_oracle_fake_quant import midpoint_tensor
+
+    x = midpoint_tensor(rows=256, seed=96)
+    r = recipe((1, 128), TWO, scale_mode=mb.MOR_SCALE_FP32_AMAX)
+    ref = orc.run(x, (1, 128), list(TWO), r.criterion, r.threshold, r.scale_mode)
+    v = wl.bf16_bits_to_float(x).astype(np.float32) * ref.scale_f32.reshape(-1, 1).astype(np.float32)
+    near15 = np.abs(np.abs(v) / np.exp2(np.floor(np.log2(np.maximum(np.abs(v), 1e-30)))) - 1.875) <= 0.0625
+    assert near15.sum() > 1000
+    parity.run_and_compare(x, r, fake_quant=True)
+    parity.run_and_compare(np.tile(x, (1, 2)), recipe((128, 128), TWO, scale_mode=mb.MOR_SCALE_E8M0), fake_quant=True)
+
+
 # ------------------------------------------------------------ per-channel partition (one block per row)
 
 @pytest.mark.parametrize("shape", [(256, 512), (130, 1000), (1, 128), (300, 72), (5, 2049)])
@@ -280,8 +296,10 @@ def test_supplied_group_amax_on_ragged_gradient_data(block):
 
 @pytest.mark.parametrize("amax_bits", [0x3F80, 0x4049, 0x3C23, 0x4B12, 0x0090, 0x7F00, 0x2D5A])
 def test_every_bf16_pattern_through_the_cast(amax_bits):
-    """All 65,536 BF16 patterns under several scales, per-tensor partition with the group amax
-    supplied (so values above it exercise saturation); NaN/inf patterns included."""
+    """All 65,536 BF16 patterns under several scales (the supplied group amax fixes the shared mantissa; block
+    amaxes always come from the data, so finite values never exceed the format's range after scaling and the
+    saturating side of the cast is reached by the +-inf patterns only, whose codes the kernel sets explicitly);
+    NaN/inf patterns included."""
     import torch
 
     bits = np.arange(65536, dtype=np.uint32).astype(np.uint16).reshape(512, 128)
@@ -296,6 +314,38 @@ def test_every_bf16_pattern_through_the_cast(amax_bits):
             ga = torch.tensor([amax], dtype=torch.float32, device="cuda")
             out = mb.analyze_quantize(parity.to_device(b), r, group_amax=ga, block_stats=True, scale_f32=True)
             parity.compare(b, r, out, ref)
+
+
+# ------------------------------------------------------------ row-sharded use, data steps on the GPU
+
+@pytest.mark.parametrize("crit,block", [(mb.MOR_CRIT_BLOCK_VS_E5M2, (128, 128)), (mb.MOR_CRIT_BLOCK_VS_E5M2, (1, 128)),
+                                        (mb.MOR_CRIT_TENSOR_MEAN_REL, (128, 128))])
+def test_row_sharded_entry_with_its_default_cuda_steps(crit, block):
+    """``sharded.analyze_quantize_row_sharded`` with the CUDA functions it uses by default (no process group: one
+    rank holds all rows), against the oracle's run over the tensor; then two halves run one after the other with
+    the tensor-wide amax, which must give the same codes as the whole."""
+    import torch
+
+    from paper_2512_22804_b200 import sharded
+
+    full = wl.activation_like(512, 384, seed=81)
+    full[300:, :] = wl.gradient_like(212, 384, seed=82)
+    r = recipe(block, TWO, crit)
+    ref = orc.run(full, block, list(TWO), crit, 0.045)
+    got = sharded.analyze_quantize_row_sharded(parity.to_device(full), r, device=torch.device("cuda"))
+    torch.cuda.synchronize()
+    assert got.group_amax == ref.tensor["group_amax"]
+    parity.compare(full, r, got.outputs, ref)
+    assert got.tensor["tensor_format"] == ref.tensor["tensor_format"] and got.tensor["nnz"] == ref.tensor["nnz"]
+    # the halves, each given the amax of the whole tensor as a rank of a sharded run would have it
+    codes = []
+    for half in (full[:256], full[256:]):
+        _, out = sharded._cuda_analyze(parity.to_device(half), r, ref.tensor["group_amax"])
+        torch.cuda.synchronize()
+        codes.append(out.codes_view().cpu().numpy())
+    ex = parity.exempt_blocks(ref, r)
+    if not ex.any() and crit != mb.MOR_CRIT_TENSOR_MEAN_REL:
+        np.testing.assert_array_equal(np.concatenate(codes), ref.codes)
 
 
 # ------------------------------------------------------------ API behaviour
