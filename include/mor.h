@@ -156,8 +156,10 @@ typedef struct mor_outputs {
                                transposed, [cols, codes_ld] with codes_ld >= roundup(rows,16),
                                so that every block is contiguous).  E4M3 codes
                                everywhere except in blocks that selected E5M2; blocks that
-                               selected BF16 still hold their E4M3 codes.  Bytes in columns
-                               cols..codes_ld-1 of each row are left untouched               */
+                               selected BF16 still hold their E4M3 codes.  The tile store works
+                               on 16-byte pieces of a row: the bytes of a row from column cols
+                               up to the next multiple of 16 are overwritten (with the code of
+                               zero); bytes from there to codes_ld-1 are left untouched       */
     int64_t  codes_ld;      /* bytes between row starts; >= roundup(cols,16); multiple of 16 */
     uint8_t* scale_e8m0;    /* [n_blocks] biased binary32 exponent of the selected format's
                                scale.  The scale is bits((e << 23) | group_mantissa); the

@@ -226,7 +226,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
 
 inline bool same_variant(const MainVariant& a, const MainVariant& b)
 {
-    return a.kind == b.kind && a.yard == b.yard && a.three == b.three && a.store == b.store && a.scan == b.scan;
+    return a.kind == b.kind && a.yard == b.yard && a.three == b.three && a.store == b.store && a.scan == b.scan &&
+           a.extra == b.extra;
 }
 
 // The launch sequence shared by every entry point.
@@ -269,7 +270,13 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     if (!aligned(workspace, kAlign)) return MOR_ERR_ALIGNMENT;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     Partial* partials = reinterpret_cast<Partial*>(ws + l.partial_off);
-    // every TMA descriptor is encoded before anything is enqueued: a call that fails here has launched nothing
+    // every TMA descriptor is encoded before anything is enqueued: a call that fails here has launched nothing.
+    // The encoder is a driver entry point and wants a current context; a host thread that has made no runtime
+    // call yet has none, so the thread's device is made current first (a no-op for every later call).
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaSetDevice(dev) != cudaSuccess) return MOR_ERR_CUDA;
+    }
     std::vector<CUtensorMap> in_maps((size_t)n), out_maps((size_t)n);
     for (int i = 0; i < n; ++i) {
         if (items[i].s.n_tiles == 0) continue;
@@ -381,6 +388,7 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.three = d->n_formats == 3;
     it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
     it.v.store = store;
+    it.v.extra = store && (o.bf16_fallback != nullptr || o.fake_quant != nullptr);
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
     // Nor is it needed where the scale has no shared mantissa (E8M0 and FP32-amax modes): those need the block

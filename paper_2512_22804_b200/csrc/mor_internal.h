@@ -96,6 +96,7 @@ struct MainVariant {
     bool three;      // three-way recipe: keep E5M2 codes and the non-zero minimum (Eq. 4)
     bool store;      // write codes (false for mor_select_stats)
     bool scan;       // the kernel scans the data for amax / smallest non-zero itself (no keys from the pre-pass)
+    bool extra;      // some tensor of the launch wants a BF16 copy of rejected blocks or the fake-quantised output
 };
 
 // Programmatic dependent launch: a kernel launched with launch_dependent() may become resident while the

@@ -1,1384 +1,28 @@
-// The fused main kernel of the MoR analyse-and-quantise pass for sm_100a.
-//
-// Per 128 x 128 tile: block amax and GAM scale (Algorithm 1), cast to E4M3 and E5M2,
-// relative-error sums (Eq. 1-3), range statistics (Eq. 4), per-block decision (Algorithm 2),
-// codes, scale bytes, selection bytes and a per-tile partial for the tensor-wide aggregate.
-//
-// Structure: persistent CTAs (two per SM), ten warps each.
-//   load warp      sleeps on a hardware barrier until the compute warps have copied a stage of the
-//                  two-stage ring of 32 KiB buffers to registers, then one thread starts the TMA
-//                  tile load (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) of the
-//                  tile that uses the stage next; an mbarrier per stage tells when it has landed;
-//   compute warps  8 warps, two threads per tile row (per tile column with 128x1 blocks).  A thread
-//                  copies its 64 elements from the stage to registers, takes the block's amax and
-//                  smallest non-zero from the key that the amax pre-pass left for the block and
-//                  that arrived with the tile (or scans its registers for them where the caller
-//                  supplied the group amax and no pre-pass ran), derives the scale, converts and
-//                  accumulates the error terms from the registers, and writes its codes to a
-//                  16 KiB staging buffer;
-//   store warp     sleeps on a hardware barrier until the staging buffer is complete, issues the
-//                  TMA tile store of the codes (clipped at the tensor's edge by the hardware),
-//                  adds up the threads' sums in a fixed order, and writes the tile's partial and,
-//                  for 128x128 and 64x64 blocks, the blocks' decisions and metadata.
-// Every wait on an mbarrier is bounded; a wait that runs out sets a status word that the
-// finalise kernel copies into mor_tensor_stats_t.status.  From then on the CTA's threads skip
-// the work and the waits but keep every barrier arrival, so that nobody is left waiting.
-//
-// Arithmetic that must be exact: amax (integer compare of BF16 bit patterns), the scale (IEEE
-// binary32 division, looked up by the 7 mantissa bits of the BF16 amax from a table that each
-// CTA fills with that same division), the scaled value (one IEEE binary32 multiply) and the FP8
-// codes (cvt.rn.satfinite).  The error ratio uses an approximate reciprocal; it only feeds
-// sums that are compared with a tolerance.
-#include <cuda_bf16.h>
-#include <cuda_fp16.h>
-#include <float.h>
-
-#include <atomic>
-#include <mutex>
-
+// Dispatch of the fused main kernel by partition kind; the kernel itself is in mor_main.cuh and is
+// instantiated kind by kind in the mor_main_*.cu files (separate files so that they compile side by side).
 #include "mor_internal.h"
 
 namespace mor {
-namespace {
 
-constexpr int kStages = 2;
-constexpr int kInBytes = kTileRows * kTileCols * 2;      // 32768
-constexpr int kOutBytes = kTileRows * kTileCols;         // 16384
-constexpr int kComputeWarps = kThreads / 32;             // 8
-constexpr int kLoadWarp = kComputeWarps;                 // warp 8; warp 9 is the store warp
-constexpr int kBarCompute = 1;                           // hardware barrier of the compute threads
-constexpr int kBarOutFull = 2;                           // + staging buffer index: compute threads arrive, store warp waits
-constexpr int kBarStageFree = 4;                         // + stage index: compute threads arrive, load warp waits
-constexpr uint32_t kBf16Inf = 0x7F80u;
-constexpr long long kWaitCycles = 400000000ll;           // a wait on an mbarrier gives up after about 0.2 s
-constexpr uint32_t kSelNone = 3u;                        // entry of a tile row outside the tensor
-
-// What the load warp tells the other warps about the tile in a stage.
-struct __align__(16) TileMeta {
-    int32_t ti;            // tensor index within the launch
-    int32_t vrows, vcols;  // rows / columns of the tile inside the tensor (1..128)
-    uint32_t blk_base;     // ROW128: index of the block of the tile's first row
-    uint32_t local;        // tile index within the tensor
-    int32_t row0, col0;    // first row / column of the tile
-    uint32_t pad;
-};
-
-// What a compute thread hands to the store warp: its (ROW128: its block's) sums and counts.
-struct __align__(16) Entry {
-    float e43, e52;
-    uint32_t nnz_nonf;     // non-zeros | non-finites << 16
-    uint32_t sel_min;      // selection (kSelNone: not a block) | (smallest non-zero bits - 1) << 16
-};
-
-struct Control {
-    unsigned long long full[kStages];                   // input ring: the tile has landed
-    unsigned long long out_empty[2];                    // code staging + entries have been consumed
-    unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
-    unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
-    TileMeta meta[kStages];
-    uint32_t keys[kStages][kTileRows];                   // block keys of the tile from the pre-pass (arrive with the tile)
-    Entry entry[2][kThreads];
-    // 128x128 and 64x64 blocks (a tile holds one block, or four: index q = 2 * (row >= 64) + (column >= 64))
-    uint32_t wmax[2][2][2 * kComputeWarps];              // per tile parity, per pass: warp (and column half) amax | inverted min
-    uint32_t tile_scale[2][4][2];                        // scale bits (E4M3, E5M2) of the tile's blocks
-    uint32_t tile_key[2][4];                             // amax bits << 16 | 0xFFFF - (min - 1)
-    uint32_t dec_sel[2][4];
-    uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
-    uint32_t issued;                                     // tile loads issued so far by this CTA
-    volatile uint32_t abort;
-};
-
-constexpr int kSmemBytes = 1024 + kStages * kInBytes + 2 * kOutBytes + (int)sizeof(Control);
-
-// ------------------------------------------------------------------ PTX helpers ----
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(void* bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(void* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
-{
-    uint32_t done;
-    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
-// Poll with a pause between tries (the pause keeps a waiting warp from taking issue slots away
-// from the warps that compute); gives up after kWaitCycles.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const volatile uint32_t* abort_flag)
-{
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i) {
-            __nanosleep(64);
-            if (mbar_test(bar, parity)) return true;
-        }
-        if (abort_flag != nullptr && *abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) return false;
-    }
-}
-// Bounded wait for the phase with the given parity; false when the limit ran out or (with a flag
-// given) another thread of the CTA has given up already.
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, const volatile uint32_t* abort_flag)
-{
-    const uint32_t a = smem_addr(bar);
-    if (mbar_test(a, parity)) return true;
-    return mbar_wait_slow(a, parity, abort_flag);
-}
-__device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, void* bar)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
-}
-// plain bulk copy global -> shared (16-byte aligned, size a multiple of 16), completing on the same mbarrier
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, void* bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, int x, int y, const void* src)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(smem_addr(src)) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-// barrier over the compute threads that also ORs a predicate
-__device__ __forceinline__ bool compute_bar_or(bool v)
-{
-    uint32_t r;
-    asm volatile("{ .reg .pred p, q; setp.ne.u32 p, %1, 0; barrier.cta.red.or.pred q, %2, %3, p; selp.u32 %0, 1, 0, q; }"
-                 : "=r"(r) : "r"((uint32_t)v), "n"(kBarCompute), "n"(kThreads) : "memory");
-    return r != 0;
-}
-// Producer / consumer hand-off on hardware barriers: the 256 compute threads announce, the 32
-// threads of the load warp (a stage is free) or of the store warp (a staging buffer is complete)
-// sleep until all have.  A thread asleep on a hardware barrier takes no issue slots.
-__device__ __forceinline__ void stage_free_arrive(uint32_t s)
-{
-    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(kBarStageFree + s), "n"(kThreads + 32) : "memory");
-}
-__device__ __forceinline__ void stage_free_sync(uint32_t s)
-{
-    asm volatile("barrier.cta.sync %0, %1;" ::"r"(kBarStageFree + s), "n"(kThreads + 32) : "memory");
-}
-__device__ __forceinline__ void out_full_arrive(uint32_t b)
-{
-    asm volatile("barrier.cta.arrive %0, %1;" ::"r"(kBarOutFull + b), "n"(kThreads + 32) : "memory");
-}
-__device__ __forceinline__ void out_full_sync(uint32_t b)
-{
-    asm volatile("barrier.cta.sync %0, %1;" ::"r"(kBarOutFull + b), "n"(kThreads + 32) : "memory");
-}
-
-__device__ __forceinline__ uint4 lds128(uint32_t a)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t a, uint4 v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void sts64(uint32_t a, uint2 v)
-{
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
-}
-
-// {hi, lo} -> two FP8 codes, `lo` in the low byte (round to nearest even, saturate to the largest finite)
-__device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
-{
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ uint32_t cvt_e5m2x2(float hi, float lo)
-{
-    uint16_t r;
-    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-// two FP8 codes -> f16x2 (exact: every E4M3 and E5M2 value is a binary16 number)
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t c)
-{
-    uint32_t r;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(static_cast<uint16_t>(c)));
-    return r;
-}
-__device__ __forceinline__ uint32_t e5m2x2_to_f16x2(uint32_t c)
-{
-    uint32_t r;
-    asm("cvt.rn.f16x2.e5m2x2 %0, %1;" : "=r"(r) : "h"(static_cast<uint16_t>(c)));
-    return r;
-}
-// (q.lo - ylo, q.hi - yhi) with q binary16 and y binary32, each one binary32 operation; exact
-// here because q is the FP8 neighbour of y
-__device__ __forceinline__ void diff_f16x2_f32(uint32_t q, float ylo, float yhi, float& dlo, float& dhi)
-{
-    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; sub.f32.f16 %0, l, %3; sub.f32.f16 %1, h, %4; }"
-        : "=f"(dlo), "=f"(dhi) : "r"(q), "f"(ylo), "f"(yhi));
-}
-// the two BF16 halves of a word as binary32, by the mixed-precision subtract x - 0 (keeps -0)
-__device__ __forceinline__ void unpack_bf16x2(uint32_t w, float& lo, float& hi)
-{
-    asm("{ .reg .b16 l, h; mov.b32 {l, h}, %2; sub.f32.bf16 %0, l, %3; sub.f32.bf16 %1, h, %3; }"
-        : "=f"(lo), "=f"(hi) : "r"(w), "f"(0.0f));
-}
-__device__ __forceinline__ float rcp_ftz(float a)
-{
-    float r;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
-    return r;
-}
-__device__ __forceinline__ float rcp_approx(float a)
-{
-    float r;
-    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(a));
-    return r;
-}
-__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi)
-{
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-// two IEEE binary32 multiplies / fused multiply-adds in one instruction (each lane rounds to nearest even)
-__device__ __forceinline__ unsigned long long mul_f32x2(unsigned long long a, unsigned long long b)
-{
-    unsigned long long r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c)
-{
-    unsigned long long r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-
-// ------------------------------------------------------------------ Algorithm 1 ----
-
-// Algorithm 1's binary32 scaling factor 448 / amax by one IEEE division; a quotient above the largest
-// finite binary32 is replaced by it
-__device__ __forceinline__ uint32_t ideal_scale_bits_div(float amax)
-{
-    return __float_as_uint(fminf(__fdiv_rn(448.0f, amax), FLT_MAX));
-}
-
-// The same for an amax that is a finite non-zero BF16 value, given as its 15 magnitude bits:
-// 448 / (2^e * (1 + m/128)) = (448 / (1 + m/128)) * 2^-e, and scaling by a power of two is exact
-// as long as the result stays a normal binary32 (it always does at the small end; at the large end,
-// and for subnormal amax, the exponent test finds the overflow).
-__device__ __forceinline__ uint32_t ideal_scale_bits_tab(uint32_t a, const uint32_t* rtab)
-{
-    const int32_t e = (int32_t)(a >> 7);
-    const uint32_t t = rtab[a & 127u];
-    const int32_t ef = (int32_t)(t >> 23) + 127 - e;
-    return ef > 254 ? 0x7F7FFFFFu : t + (uint32_t)((127 - e) * (1 << 23));
-}
-
-// Algorithm 1, group part: mantissa of 448 / g_amax (0 for an all-zero tensor, and for the
-// scale modes that have no shared mantissa)
-__device__ __forceinline__ uint32_t group_mantissa(float g_amax, int scale_mode)
-{
-    if (scale_mode != MOR_SCALE_GAM || !(g_amax > 0.0f)) return 0u;
-    return ideal_scale_bits_div(g_amax) & 0x7FFFFFu;
-}
-
-// Algorithm 1, block part: exponent of 448 / b_amax, lowered by one when the group mantissa
-// exceeds the block's; the scale is the shared mantissa joined to that exponent.  The E5M2
-// scale is 7 binades higher (57344 = 448 * 2^7), capped at exponent field 254.
-__device__ __forceinline__ void block_scale(uint32_t amax_bits, uint32_t m_g, int scale_mode, const uint32_t* rtab,
-                                            uint32_t& s4_bits, uint32_t& s5_bits)
-{
-    uint32_t e = 127u, m = (scale_mode == MOR_SCALE_FP32_AMAX) ? 0u : m_g;
-    if (amax_bits != 0u) {
-        const uint32_t sb = ideal_scale_bits_tab(amax_bits, rtab);
-        const uint32_t m_b = sb & 0x7FFFFFu;
-        e = sb >> 23;
-        if (scale_mode == MOR_SCALE_FP32_AMAX) m = m_b;
-        else if (m_g > m_b) e -= 1u;
-    }
-    const uint32_t e5 = min(e + 7u, 254u);
-    s4_bits = (e << 23) | m;
-    s5_bits = (e5 << 23) | m;
-}
-
-__device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
-{
-    return minm1_bits == 0xFFFFu ? __uint_as_float(0x7F800000u) : __uint_as_float((minm1_bits + 1u) << 16);
-}
-
-// ------------------------------------------------------------------ scan ----
-
-// Block statistics of a thread's 64 elements in one pass over packed BF16 pairs, returned as
-// one word: amax bits << 16 | 0xFFFF - (smallest non-zero bits - 1), so that both combine with
-// a packed 16-bit maximum.
-//   amax  per-halfword max of the |x| bit patterns.  NaN and inf compare above every finite
-//         pattern, which is how a non-finite input is noticed.
-//   min   per-halfword min of (|x| bits - 1) mod 2^16: zeros wrap to 0xFFFF and drop out.
-__device__ __forceinline__ uint32_t scan_words(const uint32_t (&w)[32])
-{
-    uint32_t mx[2] = {0u, 0u}, mn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-        const uint32_t a0 = w[i] & 0x7FFF7FFFu, a1 = w[i + 1] & 0x7FFF7FFFu, a2 = w[i + 2] & 0x7FFF7FFFu, a3 = w[i + 3] & 0x7FFF7FFFu;
-        mx[0] = __vimax3_u16x2(mx[0], a0, a1);
-        mx[1] = __vimax3_u16x2(mx[1], a2, a3);
-        mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
-        mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
-        mn[2] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn[2]);
-        mn[3] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn[3]);
-    }
-    const uint32_t mxx = __vimax3_u16x2(mx[0], mx[1], mx[1]);
-    const uint32_t mnn = __vimin3_u16x2(__vimin3_u16x2(mn[0], mn[1], mn[2]), mn[3], mn[3]);
-    const uint32_t amax = max(mxx & 0xFFFFu, mxx >> 16), minm1 = min(mnn & 0xFFFFu, mnn >> 16);
-    return (amax << 16) | (0xFFFFu - minm1);
-}
-
-// the same over finite elements only (used once a non-finite element has been seen).  A real
-// call, with the words passed by value in registers: inlined, the compiler turns this rare path
-// into predicated instructions that every tile would pay for.
-__device__ __forceinline__ void scan_finite4(uint4 v, uint32_t& m, uint32_t& n)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
-        if (lo < kBf16Inf) { m = max(m, lo); n = min(n, (lo - 1u) & 0xFFFFu); }
-        if (hi < kBf16Inf) { m = max(m, hi); n = min(n, (hi - 1u) & 0xFFFFu); }
-    }
-}
-__device__ __noinline__ uint32_t scan_finite_call(uint4 a, uint4 b, uint4 c, uint4 d, uint4 e, uint4 f, uint4 g, uint4 h)
-{
-    uint32_t m = 0u, n = 0xFFFFu;
-    scan_finite4(a, m, n); scan_finite4(b, m, n); scan_finite4(c, m, n); scan_finite4(d, m, n);
-    scan_finite4(e, m, n); scan_finite4(f, m, n); scan_finite4(g, m, n); scan_finite4(h, m, n);
-    return (m << 16) | (0xFFFFu - n);
-}
-__device__ __forceinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
-{
-#define MOR_W4(j) make_uint4(w[4 * (j)], w[4 * (j) + 1], w[4 * (j) + 2], w[4 * (j) + 3])
-    return scan_finite_call(MOR_W4(0), MOR_W4(1), MOR_W4(2), MOR_W4(3), MOR_W4(4), MOR_W4(5), MOR_W4(6), MOR_W4(7));
-#undef MOR_W4
-}
-
-__device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
-
-// Raise the tensor amax slot to the BF16 magnitude `bits` (non-negative binary32 patterns order like the
-// values).  Atomics on one address are served one at a time, so the slot is read first: after the first
-// tiles of a tensor almost every call ends there.
-__device__ __forceinline__ void raise_amax(float* slot, uint32_t bits, bool active)
-{
-    if (!active || bits == 0u) return;
-    unsigned int* p = reinterpret_cast<unsigned int*>(slot);
-    if (__ldcg(p) < (bits << 16)) atomicMax(p, bits << 16);
-}
-
-// ------------------------------------------------------------------ conversion ----
-
-// Fast path for one BF16 pair: two E4M3 codes (and two E5M2 codes) with their terms of
-// Eq. 1-3.   y = fl32(x * scale); c = RNE-saturating cast; q = value of c;
-// term = |y - q| / |y|, formed as |y - q| * |rcp(y + 2^-126)| (the sum inside a fused
-// multiply-add).  The caller guarantees that the block holds no NaN/inf and that every non-zero
-// |y| is at least 2^-100, so the added constant changes a term by less than 2^-26 relative, and a
-// zero element gives 0 * 2^126.  The same reciprocal counts the non-zeros: y * rcp is 1 for a
-// non-zero element (within 2^-22) and 0 for a zero.
-template <bool YARD>
-__device__ __forceinline__ void convert_pair_fast(uint32_t w, unsigned long long s4x2, unsigned long long s5x2,
-                                                  unsigned long long tiny2, float& a43, float& a52,
-                                                  unsigned long long& cnt2, uint32_t& c4, uint32_t& c5)
-{
-    float xlo, xhi;
-    unpack_bf16x2(w, xlo, xhi);
-    const unsigned long long x2 = pack_f32x2(xlo, xhi);
-    const unsigned long long y2 = mul_f32x2(x2, s4x2);
-    float ylo, yhi, ulo, uhi;
-    unpack_f32x2(y2, ylo, yhi);
-    unpack_f32x2(fma_f32x2(x2, s4x2, tiny2), ulo, uhi);
-    const float rlo = rcp_ftz(ulo), rhi = rcp_ftz(uhi);
-    cnt2 = fma_f32x2(y2, pack_f32x2(rlo, rhi), cnt2);
-    c4 = cvt_e4m3x2(yhi, ylo);
-    float dlo, dhi;
-    diff_f16x2_f32(e4m3x2_to_f16x2(c4), ylo, yhi, dlo, dhi);
-    a43 = fmaf(fabsf(dlo), fabsf(rlo), a43);
-    a43 = fmaf(fabsf(dhi), fabsf(rhi), a43);
-    if (YARD) {
-        float zlo, zhi, elo, ehi;
-        unpack_f32x2(mul_f32x2(x2, s5x2), zlo, zhi);
-        c5 = cvt_e5m2x2(zhi, zlo);
-        diff_f16x2_f32(e5m2x2_to_f16x2(c5), zlo, zhi, elo, ehi);
-        // |z - q'| / |z| = |z - q'| * (1/|y|) * (scale4/scale5); the power-of-two ratio is applied once per block
-        a52 = fmaf(fabsf(elo), fabsf(rlo), a52);
-        a52 = fmaf(fabsf(ehi), fabsf(rhi), a52);
-    } else {
-        c5 = 0;
-    }
-}
-
-struct CarefulAcc {
-    float a43, a52;
-    uint32_t nnz, nbig, nonfinite;
-};
-
-// Careful path for one BF16 pair: handles NaN/inf elements (stated reading: ignored by
-// every count and sum, NaN -> 0x7F, +-inf -> +-largest finite) and non-zero elements whose
-// scaled value leaves binary32's normal range (flushed by both formats: term 1, added by
-// the caller from the counts nnz - nbig).
-template <bool YARD>
-__device__ __forceinline__ void convert_pair_careful(uint32_t w, float s4, float s5, CarefulAcc& A, uint32_t& c4, uint32_t& c5)
-{
-    const uint32_t blo = w << 16, bhi = w & 0xFFFF0000u;
-    const uint32_t alo = blo & 0x7FFFFFFFu, ahi = bhi & 0x7FFFFFFFu;
-    const float xlo = __uint_as_float(blo), xhi = __uint_as_float(bhi);
-    const bool uselo = alo < 0x7F800000u, usehi = ahi < 0x7F800000u;
-    A.nonfinite += (uselo ? 0u : 1u) + (usehi ? 0u : 1u);
-    A.nnz += ((alo != 0u && uselo) ? 1u : 0u) + ((ahi != 0u && usehi) ? 1u : 0u);
-
-    const float ylo = __fmul_rn(xlo, s4), yhi = __fmul_rn(xhi, s4);
-    c4 = cvt_e4m3x2(yhi, ylo);
-    float dlo, dhi;
-    diff_f16x2_f32(e4m3x2_to_f16x2(c4), ylo, yhi, dlo, dhi);
-    const float aylo = fabsf(ylo), ayhi = fabsf(yhi);
-    const bool biglo = (aylo >= FLT_MIN) && uselo, bighi = (ayhi >= FLT_MIN) && usehi;
-    const float rlo = rcp_approx(aylo), rhi = rcp_approx(ayhi);
-    if (biglo) { A.a43 = fmaf(fabsf(dlo), rlo, A.a43); A.nbig++; }
-    if (bighi) { A.a43 = fmaf(fabsf(dhi), rhi, A.a43); A.nbig++; }
-
-    if (YARD) {
-        const float zlo = __fmul_rn(xlo, s5), zhi = __fmul_rn(xhi, s5);
-        c5 = cvt_e5m2x2(zhi, zlo);
-        float elo, ehi;
-        diff_f16x2_f32(e5m2x2_to_f16x2(c5), zlo, zhi, elo, ehi);
-        if (biglo) A.a52 = fmaf(fabsf(elo), rlo, A.a52);
-        if (bighi) A.a52 = fmaf(fabsf(ehi), rhi, A.a52);
-    } else {
-        c5 = 0;
-    }
-    if (!uselo) {
-        const bool nan = (alo & 0x007F0000u) != 0u;
-        const uint32_t sg = (blo >> 24) & 0x80u;
-        c4 = (c4 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Eu));
-        c5 = (c5 & 0xFF00u) | (nan ? 0x7Fu : (sg | 0x7Bu));
-    }
-    if (!usehi) {
-        const bool nan = (ahi & 0x007F0000u) != 0u;
-        const uint32_t sg = (bhi >> 24) & 0x80u;
-        c4 = (c4 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Eu)) << 8);
-        c5 = (c5 & 0x00FFu) | ((nan ? 0x7Fu : (sg | 0x7Bu)) << 8);
-    }
-}
-
-// A thread's 64 elements, held as 8 chunks of 4 words; chunk j belongs at byte offset
-// (j ^ swz) * 8 of the thread's 64 code bytes.  The E4M3 codes go to the staging buffer; a block
-// that ends up in E5M2 has them replaced afterwards (emit_e5m2_codes).
-// Results: e43 = the thread's sum of E4M3 terms, complete; e52 = its sum of E5M2 terms, complete;
-// nnz; nonfinite.
-template <bool YARD, bool CAREFUL, bool STORE>
-__device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s4b, uint32_t s5b,
-                                              float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite)
-{
-    const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
-    float a43[4] = {0.0f, 0.0f, 0.0f, 0.0f}, a52[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-    unsigned long long cnt2[2] = {0ull, 0ull};
-    CarefulAcc A;
-    A.a43 = A.a52 = 0.0f;
-    A.nnz = A.nbig = A.nonfinite = 0u;
-    const unsigned long long s4x2 = pack_f32x2(s4, s4), s5x2 = pack_f32x2(s5, s5), tiny2 = pack_f32x2(FLT_MIN, FLT_MIN);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        uint32_t a[4], b[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (CAREFUL) convert_pair_careful<YARD>(w[4 * j + i], s4, s5, A, a[i], b[i]);
-            else convert_pair_fast<YARD>(w[4 * j + i], s4x2, s5x2, tiny2, a43[i], a52[i], cnt2[i & 1], a[i], b[i]);
-        }
-        if (STORE) sts64(out_addr ^ (j << 3), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
-    }
-    // scale4 / scale5 = 2^(e4 - e5)
-    const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);
-    if (CAREFUL) {
-        const float tiny = (float)(A.nnz - A.nbig);
-        nnz = A.nnz;
-        nonfinite = A.nonfinite;
-        e43 = A.a43 + tiny;
-        e52 = YARD ? A.a52 * ratio + tiny : 0.0f;
-    } else {
-        float c0, c1, c2, c3;
-        unpack_f32x2(cnt2[0], c0, c1);
-        unpack_f32x2(cnt2[1], c2, c3);
-        nnz = (uint32_t)__float2int_rn((c0 + c1) + (c2 + c3));
-        nonfinite = 0u;
-        e43 = (a43[0] + a43[1]) + (a43[2] + a43[3]);
-        e52 = YARD ? ((a52[0] + a52[1]) + (a52[2] + a52[3])) * ratio : 0.0f;
-    }
-}
-
-// The E5M2 codes of a thread's 64 elements, for a block that selected E5M2 (such a block holds no
-// NaN or inf): z = fl32(x * scale5), RNE-saturating cast, over the E4M3 codes in the staging buffer.
-__device__ __forceinline__ void emit_e5m2_codes(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s5b)
-{
-    const float s5 = __uint_as_float(s5b);
-    const unsigned long long s5x2 = pack_f32x2(s5, s5);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        uint32_t c[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t ww = w[4 * j + i];
-            float zlo, zhi;
-            unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(ww << 16), __uint_as_float(ww & 0xFFFF0000u)), s5x2), zlo, zhi);
-            c[i] = cvt_e5m2x2(zhi, zlo);
-        }
-        sts64(out_addr ^ (j << 3), make_uint2(__byte_perm(c[0], c[1], 0x5410), __byte_perm(c[2], c[3], 0x5410)));
-    }
-}
-
-// Algorithm 2 for one block with the per-block metrics (M_1 = Eq. 3, M_2 = Eq. 4, or
-// Eq. 1-2 on the block alone).
-template <typename T>
-__device__ __forceinline__ uint32_t decide_block(const TensorRec& R, T e43, T e52, uint32_t nnz,
-                                                 uint32_t nonfinite, uint32_t amax_bits, uint32_t minm1_bits,
-                                                 uint32_t n_elems)
-{
-    if (nonfinite) return MOR_FMT_BF16;
-    if (R.criterion == MOR_CRIT_BLOCK_VS_E5M2) {
-        const bool ok = (R.flags & MOR_FLAG_STRICT_TIES) ? (e43 < e52) : (e43 <= e52);
-        if (ok) return MOR_FMT_E4M3;
-        if (R.n_formats == 3) {
-            // max|b| < (57344 * 2^14) * min|b|, exact in binary32 (11 significant bits)
-            float mnv = minnz_value(minm1_bits);
-            if ((R.flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) && nnz < n_elems) mnv = 0.0f;
-            const float amax = __uint_as_float(amax_bits << 16);
-            if (amax < 939524096.0f * mnv) return MOR_FMT_E5M2;
-        }
-        return MOR_FMT_BF16;
-    }
-    if (R.criterion == MOR_CRIT_BLOCK_MEAN_REL) {
-        const double err = nnz ? (double)e43 / (double)nnz : 0.0;
-        return err < (double)R.threshold ? MOR_FMT_E4M3 : MOR_FMT_BF16;
-    }
-    return MOR_FMT_E4M3;   // tensor-level criterion: decided by the finalise kernel
-}
-
-
-// ------------------------------------------------------------------ tile bookkeeping ----
-
-struct TileId {
-    int ti;
-    uint32_t local;
-    int row0, col0, vrows, vcols;
-};
-
-__device__ __forceinline__ TileId locate_tile(const BatchParams& b, uint32_t tile)
-{
-    int ti = 0;
-    uint32_t begin = 0;
-#pragma unroll 1
-    while (ti < b.n - 1 && tile >= b.tile_end[ti]) { begin = b.tile_end[ti]; ++ti; }
-    const TensorRec& R = b.t[ti];
-    TileId t;
-    t.ti = ti;
-    t.local = tile - begin;
-    const uint32_t bi = t.local / R.nbc, bj = t.local - bi * R.nbc;
-    t.row0 = (int)(bi * kTileRows);
-    t.col0 = (int)(bj * kTileCols);
-    const long long rr = R.rows - t.row0, cc = R.cols - t.col0;
-    t.vrows = (int)(rr < kTileRows ? rr : kTileRows);
-    t.vcols = (int)(cc < kTileCols ? cc : kTileCols);
-    return t;
-}
-
-__device__ __forceinline__ void give_up(Control& C, uint32_t* device_status)
-{
-    C.abort = 1u;
-    atomicOr(device_status, 1u);
-}
-
-__device__ __forceinline__ double shfl_xor_f64(double v, int o) { return __shfl_xor_sync(0xFFFFFFFFu, v, o); }
-
-// ------------------------------------------------------------------ load warp ----
-
-// One thread: start the TMA load of the CTA's tile number `it` into its stage (nothing when the CTA
-// has no such tile).  The stage must be free.
-__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it)
-{
-    const uint32_t tile = blockIdx.x + it * gridDim.x;
-    if (tile >= p.total_tiles) return;
-    const uint32_t s = it % kStages;
-    const TileId t = locate_tile(p.b, tile);
-    TileMeta m;
-    m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
-    m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
-    if (p.b.t[t.ti].kind == KIND_COL128) m.blk_base = (uint32_t)(t.row0 / kTileRows) * (uint32_t)p.b.t[t.ti].cols + (uint32_t)t.col0;
-    if (p.b.t[t.ti].kind == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
-    m.pad = 0;
-    C.meta[s] = m;
-    const TensorRec& R = p.b.t[t.ti];
-    const uint32_t key_bytes = R.keys != nullptr ? R.key_stride * 4u : 0u;
-    mbar_arrive_expect_tx(&C.full[s], kInBytes + key_bytes);
-    tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
-    if (key_bytes) {
-        const uint32_t* src = R.kind == KIND_CHANNEL ? R.row_keys + t.row0 : R.keys + (size_t)t.local * R.key_stride;
-        bulk_load(&C.keys[s][0], src, key_bytes, &C.full[s]);
-    }
-    C.issued = it + 1;
-}
-
-__device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in, int lane)
-{
-    if (lane == 0) {
-        for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load(p, C, in, it);
-    }
-#pragma unroll 1
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
-        if (tile >= p.total_tiles) break;
-        stage_free_sync(it % kStages);                  // sleeps until every compute thread has its copy
-        if (lane == 0 && !C.abort) issue_tile_load(p, C, in, it + kStages);
-    }
-    if (lane == 0 && C.abort) {
-        // copies that may still be in flight must land (or be given up on) before the CTA goes
-        const uint32_t issued = C.issued;
-        for (uint32_t k = 0; k < (uint32_t)kStages && k < issued; ++k) {
-            const uint32_t it = issued - 1 - k;
-            mbar_wait(&C.full[it % kStages], (it / kStages) & 1u, nullptr);
-        }
-    }
-}
-
-// ------------------------------------------------------------------ store warp ----
-
-template <int KIND, bool THREE, bool STORE>
-__device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsigned char* out, Partial* __restrict__ partials,
-                                           int lane)
-{
-    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128 || KIND == KIND_DUAL;   // 128 one-line blocks per tile
-    constexpr int kEntries = kLineBlocks ? kTileRows : kThreads;
-    bool stores_pending = false;
-#pragma unroll 1
-    for (uint32_t it = 0;; ++it) {
-        // both directions from one read: two conversions per tile, rows (record ti) then columns (record ti + 1)
-        const uint32_t tile = blockIdx.x + (KIND == KIND_DUAL ? it >> 1 : it) * gridDim.x;
-        if (tile >= p.total_tiles) break;
-        const uint32_t b = it & 1u, n = it >> 1;
-        const bool columns = KIND == KIND_COL128 || (KIND == KIND_DUAL && (it & 1u));
-        TileId t = locate_tile(p.b, tile);              // before the wait: off the critical path
-        if (KIND == KIND_DUAL && columns) t.ti += 1;
-        const TensorRec& R = p.b.t[t.ti];
-        constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
-        // the decision is handed back every tile of a launch with whole-tile blocks, whether this
-        // tensor's compute threads wait for it or not: the barrier's phase then follows the tile count,
-        // also when tensors with and without a BF16 copy share a launch
-        constexpr bool need_dec = kTileBlocks;
-        const bool codes_wait = STORE && kTileBlocks && THREE;
-        out_full_sync(b);                                // sleeps until every compute thread has arrived
-        if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
-            if (STORE && !codes_wait && lane == 0) {
-                // the codes are complete: start the tile store at once, it runs while the sums are formed
-                // (sub-column blocks: the staging tile and the code tensor are transposed)
-                tma_store_tile(&p.out_map[t.ti], columns ? t.row0 : t.col0, columns ? t.col0 : t.row0, out + b * kOutBytes);
-                bulk_commit();
-                stores_pending = true;
-            }
-
-            // the threads' sums in a fixed order: lane-strided in binary32, then a butterfly in double.
-            // With 64x64 blocks a lane's entries belong to one column half (lane & 1) and to the upper
-            // (k < 4) or lower rows: two sets of sums per lane, combined over the lanes of equal parity.
-            constexpr int NR = KIND == KIND_BLK64 ? 2 : 1;
-            float f43[NR], f52[NR];
-            uint32_t nnz[NR], nonf[NR], n4 = 0, n5 = 0, nb = 0, mn = 0xFFFFu;
-#pragma unroll
-            for (int r = 0; r < NR; ++r) { f43[r] = 0.0f; f52[r] = 0.0f; nnz[r] = 0; nonf[r] = 0; }
-#pragma unroll
-            for (int k = 0; k < kEntries / 32; ++k) {
-                const Entry e = C.entry[b][lane + 32 * k];
-                const int r = (NR == 2 && k >= 4) ? 1 : 0;
-                f43[r] += e.e43;
-                f52[r] += e.e52;
-                nnz[r] += e.nnz_nonf & 0xFFFFu;
-                nonf[r] += e.nnz_nonf >> 16;
-                if (kLineBlocks) {
-                    const uint32_t sel = e.sel_min & 0xFFFFu;
-                    n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
-                }
-                mn = min(mn, e.sel_min >> 16);
-            }
-            double s43[NR], s52[NR];
-#pragma unroll
-            for (int r = 0; r < NR; ++r) {
-                s43[r] = (double)f43[r]; s52[r] = (double)f52[r];
-#pragma unroll
-                for (int o = 16; o > (NR == 2 ? 1 : 0); o >>= 1) {
-                    s43[r] += shfl_xor_f64(s43[r], o); s52[r] += shfl_xor_f64(s52[r], o);
-                    if (NR == 2) { nnz[r] += __shfl_xor_sync(0xFFFFFFFFu, nnz[r], o); nonf[r] += __shfl_xor_sync(0xFFFFFFFFu, nonf[r], o); }
-                }
-                if (NR == 1) { nnz[r] = __reduce_add_sync(0xFFFFFFFFu, nnz[r]); nonf[r] = __reduce_add_sync(0xFFFFFFFFu, nonf[r]); }
-            }
-            mn = __reduce_min_sync(0xFFFFFFFFu, mn);
-            if (kLineBlocks) {
-                n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
-                n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
-                nb = __reduce_add_sync(0xFFFFFFFFu, nb);
-            }
-
-            // tile totals (64x64: the four blocks in the order q = 0..3, taken from lanes 0 and 1)
-            double t43 = s43[0], t52 = s52[0];
-            uint32_t tnnz = nnz[0], tnonf = nonf[0];
-            if (NR == 2) {
-                const double a1 = __shfl_sync(0xFFFFFFFFu, s43[0], 1), b1 = __shfl_sync(0xFFFFFFFFu, s52[0], 1);
-                const double a3 = __shfl_sync(0xFFFFFFFFu, s43[NR - 1], 1), b3 = __shfl_sync(0xFFFFFFFFu, s52[NR - 1], 1);
-                t43 = ((s43[0] + a1) + s43[NR - 1]) + a3;
-                t52 = ((s52[0] + b1) + s52[NR - 1]) + b3;
-                tnnz = nnz[0] + nnz[NR - 1]; tnnz += __shfl_xor_sync(0xFFFFFFFFu, tnnz, 1);
-                tnonf = nonf[0] + nonf[NR - 1]; tnonf += __shfl_xor_sync(0xFFFFFFFFu, tnonf, 1);
-            }
-
-            if (kTileBlocks && lane < (NR == 2 ? 2 : 1)) {
-                // Algorithm 2 for the tile's block(s): lane 0 decides block(s) of the left column half, lane 1 of the right
-#pragma unroll
-                for (int r = 0; r < NR; ++r) {
-                    const int q = NR == 2 ? 2 * r + lane : 0;
-                    const int br = NR == 2 ? 64 : 128;
-                    const int vr = min(br, t.vrows - (NR == 2 ? 64 * r : 0)), vc = min(br, t.vcols - (NR == 2 ? 64 * lane : 0));
-                    uint32_t bsel = kSelNone;
-                    if (vr > 0 && vc > 0) {
-                        const uint32_t key = C.tile_key[b][q], s4b = C.tile_scale[b][q][0], s5b = C.tile_scale[b][q][1];
-                        const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
-                        bsel = decide_block(R, s43[r], s52[r], nnz[r], nonf[r], amax_bits, minm1, (uint32_t)(vr * vc));
-                        const uint32_t blk = NR == 2 ? (uint32_t)(t.row0 / 64 + r) * R.nbc_blk + (uint32_t)(t.col0 / 64 + lane) : t.local;
-                        const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
-                        if (R.sel) R.sel[blk] = (uint8_t)bsel;
-                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
-                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
-                        if (R.block_stats) {
-                            mor_block_stats_t bs;
-                            bs.amax = __uint_as_float(amax_bits << 16);
-                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                            bs.nnz = nnz[r]; bs.n_nonfinite = nonf[r];
-                            bs.sum_rel_e4m3 = (float)s43[r]; bs.sum_rel_e5m2 = (float)s52[r];
-                            R.block_stats[blk] = bs;
-                        }
-                    }
-                    if (need_dec) C.dec_sel[b][q] = bsel;
-                    n4 += bsel == MOR_FMT_E4M3; n5 += bsel == MOR_FMT_E5M2; nb += bsel == MOR_FMT_BF16;
-                }
-            }
-            if (NR == 2) {
-                n4 += __shfl_xor_sync(0xFFFFFFFFu, n4, 1); n5 += __shfl_xor_sync(0xFFFFFFFFu, n5, 1); nb += __shfl_xor_sync(0xFFFFFFFFu, nb, 1);
-            }
-            if (need_dec) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&C.dec_full[b]);      // compute threads may be waiting for the decision
-            }
-            if (lane == 0) {
-                Partial P;
-                P.sum43 = t43; P.sum52 = t52; P.nnz = tnnz; P.nonfinite = tnonf;
-                P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
-                partials[R.tile_begin + t.local] = P;
-            }
-            if (codes_wait) {
-                // three formats, 128x128 blocks: the compute threads put the chosen format's codes in place
-                // after the decision
-                bool ok = mbar_wait(&C.codes_full[b], n & 1u, &C.abort);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok && lane == 0) give_up(C, p.device_status);
-                if (ok && lane == 0) {
-                    tma_store_tile(&p.out_map[t.ti], t.col0, t.row0, out + b * kOutBytes);
-                    bulk_commit();
-                    stores_pending = true;
-                }
-            }
-            if (STORE && lane == 0 && stores_pending) bulk_wait_read<0>();   // the staging buffer may be overwritten from here on
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&C.out_empty[b]);
-    }
-    if (lane == 0 && stores_pending) bulk_wait_all();
-}
-
-// ------------------------------------------------------------------ compute warps ----
-
-// copy of every block that stays in BF16, straight from the registers
-__device__ __forceinline__ void write_fallback(const TensorRec& R, const uint32_t (&w)[32], const TileMeta& m, int row, int h, int swz)
-{
-    if (row >= m.vrows) return;
-    uint16_t* dst_row = R.fallback + (long long)(m.row0 + row) * R.ld + m.col0 + h * 64;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int c = (j ^ swz) * 8;                      // first of the chunk's 8 elements within the thread's 64
-        const int left = m.vcols - (h * 64 + c);
-        if (left >= 8) {
-            *reinterpret_cast<uint4*>(dst_row + c) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i < left) dst_row[c + i] = (uint16_t)(w[4 * j + (i >> 1)] >> (16 * (i & 1)));
-        }
-    }
-}
-
-// Fake quantisation of a thread's 64 elements (Section 4: quantise, dequantise, de-scale; BF16 out): the FP8
-// value of format `fmt` divided by the scale in one binary32 division, rounded to BF16; a block that stays
-// in BF16 and NaN/inf elements are copied.  Straight from the registers, like the fallback copy.
-__device__ __noinline__ void fake_quant_chunk(uint4 v, uint32_t fmt, float s, uint32_t (&o)[4])
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t ww = w[i];
-        const float xlo = __uint_as_float(ww << 16), xhi = __uint_as_float(ww & 0xFFFF0000u);
-        const float ylo = __fmul_rn(xlo, s), yhi = __fmul_rn(xhi, s);
-        const uint32_t q = fmt == MOR_FMT_E5M2 ? e5m2x2_to_f16x2(cvt_e5m2x2(yhi, ylo)) : e4m3x2_to_f16x2(cvt_e4m3x2(yhi, ylo));
-        const float2 qf = __half22float2(*reinterpret_cast<const __half2*>(&q));
-        const float tlo = __fdiv_rn(qf.x, s), thi = __fdiv_rn(qf.y, s);
-        uint32_t r;
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(thi), "f"(tlo));
-        if ((ww & 0x7F80u) == 0x7F80u) r = (r & 0xFFFF0000u) | (ww & 0xFFFFu);             // NaN / inf: as they are
-        if ((ww & 0x7F800000u) == 0x7F800000u) r = (r & 0xFFFFu) | (ww & 0xFFFF0000u);
-        o[i] = r;
-    }
-}
-__device__ __forceinline__ void write_fake_quant(const TensorRec& R, const uint32_t (&w)[32], const TileMeta& m, int row, int h, int swz,
-                                                 uint32_t fmt, uint32_t s4b, uint32_t s5b)
-{
-    if (row >= m.vrows) return;
-    const float s = __uint_as_float(fmt == MOR_FMT_E5M2 ? s5b : s4b);
-    uint16_t* dst_row = R.fake_quant + (long long)(m.row0 + row) * R.ld + m.col0 + h * 64;
-#pragma unroll 1
-    for (int j = 0; j < 8; ++j) {
-        const int c = (j ^ swz) * 8;
-        const int left = m.vcols - (h * 64 + c);
-        if (left <= 0) continue;
-        // chunk j of the registers, selected without indexing them dynamically
-        uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
-#pragma unroll
-        for (int k = 1; k < 8; ++k)
-            if (j == k) v = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
-        uint32_t o[4] = {v.x, v.y, v.z, v.w};
-        if (fmt != MOR_FMT_BF16) fake_quant_chunk(v, fmt, s, o);
-        if (left >= 8) {
-            *reinterpret_cast<uint4*>(dst_row + c) = make_uint4(o[0], o[1], o[2], o[3]);
-        } else {
-            for (int i = 0; i < left; ++i) dst_row[c + i] = (uint16_t)(o[i >> 1] >> (16 * (i & 1)));
-        }
-    }
-}
-
-template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
-__device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
-{
-    const int lane = tid & 31, warp = tid >> 5;
-    const int row = tid >> 1, h = tid & 1;
-    // Chunk order: thread (row, h) holds the 16-byte chunk c of its 128 bytes as chunk c ^ swz.  With
-    // this choice the 8 threads of a 128-bit load phase and the 16 threads of a 64-bit store phase
-    // touch distinct banks.
-    // Sub-column blocks read 16-bit pieces down a column; all rows of a column share a bank, so there
-    // the two columns that share a 32-bit word get the same order (they then read the same word) at the
-    // price of a two-way conflict on the stores.
-    const int swz = KIND == KIND_COL128 ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
-    constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;
-    const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
-    const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
-    const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
-    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
-
-    // what changes only with the tensor, kept in registers
-    int cur_ti = -1;
-    uint32_t m_g = 0;            // Algorithm 1, group part
-    int scale_mode = 0;
-    bool has_fallback = false;
-    bool has_fq = false, fq_e4m3 = false;   // fake-quantised output wanted; ... with E4M3 values whatever the block's selection
-    uint32_t tensor_amax_bits = 0;
-    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
-    bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
-#pragma unroll 1
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
-        if (tile >= p.total_tiles) break;
-        const uint32_t s = it % kStages, b = it & 1u, n2 = it >> 1;
-
-        if (!dead) {
-            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
-        }
-        TileMeta m;
-        {
-            const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
-            m.ti = dead ? 0 : (int32_t)q.x; m.vrows = (int32_t)q.y; m.vcols = (int32_t)q.z; m.blk_base = q.w;
-            m.local = 0; m.row0 = 0; m.col0 = 0; m.pad = 0;
-        }
-        uint32_t w[32];
-        if (KIND == KIND_COL128) {
-            // sub-column blocks: this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows
-            // per word, so that everything after this point works on the block as on a row piece
-            const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                uint32_t lo, hi;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
-                w[i] = lo | (hi << 16);
-            }
-        } else {
-            const uint32_t a = in_base + s * kInBytes + in_off;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const uint4 v = lds128(a ^ (j << 4));
-                w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
-            }
-        }
-        const TensorRec& R = p.b.t[m.ti];
-        if (m.ti != cur_ti) {
-            cur_ti = m.ti;
-            scale_mode = R.scale_mode;
-            has_fallback = STORE && R.fallback != nullptr;
-            has_fq = STORE && R.fake_quant != nullptr;
-            fq_e4m3 = KIND == KIND_TENSOR || KIND == KIND_CHANNEL || R.criterion == MOR_CRIT_TENSOR_MEAN_REL;
-            if (!dead) {
-                m_g = group_mantissa(*R.amax, scale_mode);
-                if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
-            }
-        }
-        if (has_fallback || has_fq) {      // the BF16 outputs need the tile's position too
-            const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
-            m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z;
-        }
-        uint32_t key = 0u;
-        if (!SCAN) {
-            // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + ((KIND == KIND_ROW128 || KIND == KIND_CHANNEL) ? (uint32_t)row * 4u : (uint32_t)q * 4u)));
-        }
-        stage_free_arrive(s);                           // this thread's copy of the stage is in registers
-
-        // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
-        bool nonfin = false;
-        if (!SCAN) {
-            nonfin = (key >> 31) != 0u;
-            key &= 0x7FFFFFFFu;
-            if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);   // warp-uniform (a tile-wide key is CTA-uniform already)
-        } else if (kLineBlocks) {
-            key = scan_words(w);
-            key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
-            nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
-            if (nonfin) {
-                key = scan_words_finite(w);
-                key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
-            }
-            // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
-            // patterns order like the values)
-            if (!(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot) {
-                const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
-                raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
-            }
-        } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
-            key = scan_words(w);
-            uint32_t tile_amax = 0u;
-#pragma unroll 1
-            for (int pass = 0; pass < 2; ++pass) {
-                // the warps exchange their keys; with 64x64 blocks a warp has one per column half (lane parity)
-                const uint32_t part = KIND == KIND_BLK64 ? (h ? 0xAAAAAAAAu : 0x55555555u) : 0xFFFFFFFFu;
-                const uint32_t hi = __reduce_max_sync(part, key >> 16), lo = __reduce_max_sync(part, key & 0xFFFFu);
-                if (KIND == KIND_BLK64) { if (lane < 2) C.wmax[b][pass][2 * warp + h] = (hi << 16) | lo; }
-                else if (lane == 0) C.wmax[b][pass][warp] = (hi << 16) | lo;
-                dead = compute_bar_or(dead);                                       // also spreads the word that a wait ran out
-                uint32_t any;                                                      // the largest key of the tile: CTA-uniform
-                if (KIND == KIND_BLK64) {
-                    const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]), k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
-                    const uint4 k2 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][8]), k3 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][12]);
-                    // entries 2 * warp + h: warps 0-3 hold the upper rows, 4-7 the lower
-                    const uint32_t u0 = __vimax3_u16x2(k0.x, k0.z, key_max(k1.x, k1.z)), u1 = __vimax3_u16x2(k0.y, k0.w, key_max(k1.y, k1.w));
-                    const uint32_t l0 = __vimax3_u16x2(k2.x, k2.z, key_max(k3.x, k3.z)), l1 = __vimax3_u16x2(k2.y, k2.w, key_max(k3.y, k3.w));
-                    key = (row >> 6) ? (h ? l1 : l0) : (h ? u1 : u0);
-                    any = key_max(key_max(u0, u1), key_max(l0, l1));
-                } else {
-                    const uint4 k0 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][0]);
-                    const uint4 k1 = *reinterpret_cast<const uint4*>(&C.wmax[b][pass][4]);
-                    key = key_max(key_max(__vimax3_u16x2(k0.x, k0.y, k0.z), k0.w), key_max(__vimax3_u16x2(k1.x, k1.y, k1.z), k1.w));
-                    any = key;
-                }
-                nonfin = pass == 1 || (any >> 16) >= kBf16Inf;                     // CTA-uniform
-                if (dead) { key = 0u; nonfin = false; }
-                tile_amax = any >> 16;
-                if (pass == 1 || !nonfin) break;
-                key = scan_words_finite(w);
-            }
-            // no pre-pass ran: the tensor amax that the summary reports is gathered here
-            raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead && !(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot);
-        } else {
-            key = scan_words(w);
-            nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
-            if (nonfin) key = scan_words_finite(w);
-        }
-        uint32_t amax_bits = key >> 16;
-        const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
-        // per-tensor partition: the block is the tensor, its amax was reduced by the pre-pass
-        if (KIND == KIND_TENSOR) amax_bits = tensor_amax_bits;
-
-        uint32_t s4b, s5b;
-        block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
-
-        // The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_pair_fast).
-        // minm1 covers this thread's block (ROW128), this tile (BLK128), this thread (TENSOR).
-        bool careful = nonfin;
-        if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
-        if (KIND != KIND_BLK128) careful = __any_sync(0xFFFFFFFFu, careful);
-
-        // ---- staging buffer and entries of tile it - 2 must have been consumed ----
-        if (n2 > 0 && !dead) {
-            bool ok = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
-        }
-
-        const uint32_t oa = out_base + b * kOutBytes + out_off;
-        uint32_t sel = MOR_FMT_E4M3;
-        if (!dead) {
-            // ---- cast and error terms ----
-            float e43, e52;
-            uint32_t nnz, nonf;
-            if (careful) convert_words<YARD, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
-            else         convert_words<YARD, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
-
-            if (kLineBlocks) {
-                // ---- block sums, decision, metadata ----
-                e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
-                e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
-                uint32_t nz = nnz | (nonf << 16);
-                nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
-                const bool valid = row < (KIND == KIND_COL128 ? m.vcols : m.vrows);
-                sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
-                if (THREE && STORE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
-                if (h == 0) {
-                    sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
-                           make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
-                    if (valid) {
-                        const uint32_t blk = m.blk_base + (uint32_t)row * (KIND == KIND_COL128 ? 1u : R.nbc);
-                        const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
-                        if (R.sel) R.sel[blk] = (uint8_t)sel;
-                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
-                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
-                        if (R.block_stats) {
-                            mor_block_stats_t bs;
-                            bs.amax = __uint_as_float(amax_bits << 16);
-                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                            bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
-                            R.block_stats[blk] = bs;
-                        }
-                    }
-                }
-                if (has_fallback && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
-                if (has_fq) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
-            } else {
-                sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
-                       make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
-                if ((KIND == KIND_TENSOR || KIND == KIND_CHANNEL) && has_fq)
-                    write_fake_quant(R, w, m, row, h, swz, (uint32_t)MOR_FMT_E4M3, s4b, s5b);
-                if (KIND == KIND_CHANNEL && h == 0 && m.blk_base != 0xFFFFFFFFu && row < m.vrows) {
-                    // per-channel: the row's scale, written by the tile that holds the row's first columns
-                    const uint32_t blk = m.blk_base + (uint32_t)row;
-                    if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(s4b >> 23);
-                    if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(s4b);
-                }
-                if ((KIND == KIND_BLK128 && tid == 0) || (KIND == KIND_BLK64 && (row & 63) == 0)) {
-                    C.tile_scale[b][q][0] = s4b; C.tile_scale[b][q][1] = s5b; C.tile_key[b][q] = key;
-                }
-            }
-            if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
-        }
-        out_full_arrive(b);
-
-        if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
-            const bool need_dec = THREE || has_fallback || has_fq;
-            if (need_dec) {
-                if (!dead) {
-                    bool ok = mbar_wait(&C.dec_full[b], n2 & 1u, &C.abort);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
-                }
-                if (!dead) sel = C.dec_sel[b][q];
-                if (THREE && STORE) {
-                    if (!dead && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&C.codes_full[b]);
-                }
-                if (has_fallback && !dead && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
-                if (has_fq && !dead) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------ both directions from one read ----
-
-// KIND_DUAL: the tensor is wanted with 1x128 blocks and with 128x1 blocks (the two operand layouts of the forward
-// and backward GEMMs).  A tile is loaded once; the compute threads take it from the stage twice, first as rows
-// (record ti, exactly the 1x128 path), then as columns (record ti + 1, exactly the 128x1 path, codes transposed),
-// and hand each direction to the store warp as a tile of its own, so the two staging buffers alternate between
-// the directions.  The stage is released after the second copy to registers.
-template <bool YARD, bool THREE, bool SCAN>
-__device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
-{
-    const int lane = tid & 31;
-    const int row = tid >> 1, h = tid & 1;
-    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
-    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
-    int cur_ti = -1;
-    uint32_t m_g = 0;
-    int scale_mode = 0;
-    bool dead = false;
-#pragma unroll 1
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t tile = blockIdx.x + it * gridDim.x;
-        if (tile >= p.total_tiles) break;
-        const uint32_t s = it % kStages;
-        if (!dead) {
-            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
-        }
-        TileMeta m;
-        {
-            const uint4 q0 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
-            const uint4 q1 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
-            m.ti = dead ? 0 : (int32_t)q0.x; m.vrows = (int32_t)q0.y; m.vcols = (int32_t)q0.z; m.blk_base = q0.w;
-            m.local = q1.x; m.row0 = (int32_t)q1.y; m.col0 = (int32_t)q1.z; m.pad = 0;
-        }
-        if (m.ti != cur_ti) {
-            cur_ti = m.ti;
-            scale_mode = p.b.t[m.ti].scale_mode;
-            if (!dead) m_g = group_mantissa(*p.b.t[m.ti].amax, scale_mode);
-        }
-#pragma unroll 1
-        for (int dir = 0; dir < 2; ++dir) {
-            const TensorRec& R = p.b.t[m.ti + dir];
-            const uint32_t b = (uint32_t)dir, n2 = it;        // conversion number 2 * it + dir
-            const int swz = dir ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
-            uint32_t w[32];
-            uint32_t key = 0u;
-            if (dir == 0) {
-                const uint32_t a = in_base + s * kInBytes + (uint32_t)(row * 256 + h * 128 + (swz << 4));
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint4 v = lds128(a ^ (j << 4));
-                    w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
-                }
-                if (!SCAN) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)row * 4u));
-            } else {
-                // this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows per word
-                const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    uint32_t lo, hi;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
-                    w[i] = lo | (hi << 16);
-                }
-                stage_free_arrive(s);                       // both copies of the stage are in registers
-            }
-
-            // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
-            bool nonfin;
-            if (dir == 0 && !SCAN) {
-                nonfin = __any_sync(0xFFFFFFFFu, (key >> 31) != 0u);
-                key &= 0x7FFFFFFFu;
-            } else {
-                key = scan_words(w);
-                key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
-                nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
-                if (nonfin) {
-                    key = scan_words_finite(w);
-                    key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
-                }
-                if (dir == 0) {                             // no pre-pass ran: gather the tensor amax for the summaries
-                    const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
-                    raise_amax(R.amax_slot, wamax, lane == 0 && !dead && R.amax == R.amax_slot);
-                }
-            }
-            const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
-            uint32_t s4b, s5b;
-            block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
-            bool careful = nonfin;
-            if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
-            careful = __any_sync(0xFFFFFFFFu, careful);
-
-            // ---- staging buffer and entries of the same direction of the tile before must have been consumed ----
-            if (n2 > 0 && !dead) {
-                bool ok = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort);
-                ok = __all_sync(0xFFFFFFFFu, ok);
-                if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
-            }
-            const uint32_t oa = out_base + b * kOutBytes + (uint32_t)(row * 128 + h * 64 + (swz << 3));
-            if (!dead) {
-                float e43, e52;
-                uint32_t nnz, nonf;
-                if (careful) convert_words<YARD, true, true>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
-                else         convert_words<YARD, false, true>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
-                e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
-                e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
-                uint32_t nz = nnz | (nonf << 16);
-                nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
-                const bool valid = row < (dir ? m.vcols : m.vrows);
-                const uint32_t sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(dir ? m.vrows : m.vcols));
-                if (THREE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
-                if (h == 0) {
-                    sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
-                           make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
-                    if (valid) {
-                        const uint32_t blk = dir ? (uint32_t)(m.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)m.col0 + (uint32_t)row
-                                                 : m.blk_base + (uint32_t)row * R.nbc;
-                        const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
-                        if (R.sel) R.sel[blk] = (uint8_t)sel;
-                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
-                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
-                        if (R.block_stats) {
-                            mor_block_stats_t bs;
-                            bs.amax = __uint_as_float(amax_bits << 16);
-                            bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
-                            bs.nnz = nz & 0xFFFFu; bs.n_nonfinite = nz >> 16; bs.sum_rel_e4m3 = e43; bs.sum_rel_e5m2 = e52;
-                            R.block_stats[blk] = bs;
-                        }
-                    }
-                }
-                fence_async_smem();                      // the codes must be visible to the TMA store
-            }
-            out_full_arrive(b);
-        }
-    }
-}
-
-// ------------------------------------------------------------------ kernel ----
-
-template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
-__global__ void __launch_bounds__(kMainThreads, 2)
-mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ partials)
-{
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* base = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
-    unsigned char* in = base;
-    unsigned char* out = base + kStages * kInBytes;
-    Control& C = *reinterpret_cast<Control*>(out + 2 * kOutBytes);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(&C.full[s], 1);
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&C.out_empty[b], 1);
-            mbar_init(&C.dec_full[b], 1);
-            mbar_init(&C.codes_full[b], kComputeWarps);
-        }
-        C.abort = 0u;
-        C.issued = 0u;
-        fence_mbar_init();
-    }
-    // fl32(448 / (1 + m/128)) for the 128 mantissas of a BF16 amax: the division of Algorithm 1,
-    // done here once per CTA with the IEEE divide and looked up per block afterwards
-    if (tid < 128) C.rtab[tid] = __float_as_uint(__fdiv_rn(448.0f, 1.0f + (float)tid * 0.0078125f));
-    __syncthreads();
-    // Up to here nothing was read that an earlier kernel of the stream writes: this CTA may have become resident
-    // while the amax pre-pass was still draining.  From here on its amax and keys are needed.
-    pdl_trigger();
-    pdl_wait();
-
-    if (warp < kComputeWarps) {
-        if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
-        else compute_warps<KIND, YARD, THREE, STORE, SCAN>(p, C, in, out, tid);
-    }
-    else if (warp == kLoadWarp) load_warp(p, C, in, lane);
-    else store_warp<KIND, THREE, STORE>(p, C, out, partials, lane);
-}
-
-template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN>
-cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
-{
-    auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE, SCAN>;
-    static std::atomic<int> sm_count[64];   // per instantiation and device; 0 = not set up yet
-    static std::mutex setup;
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    int sms = sm_count[dev].load(std::memory_order_acquire);
-    if (sms == 0) {
-        std::lock_guard<std::mutex> lock(setup);         // host threads may make their first call together
-        e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        if (sms <= 0) return cudaErrorInvalidDevice;
-        sm_count[dev].store(sms, std::memory_order_release);
-    }
-    const uint32_t resident = 2u * (uint32_t)sms;
-    const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
-    return launch_dependent(kfn, dim3(grid), dim3(kMainThreads), (size_t)kSmemBytes, s, p, partials);
-}
-
-template <int KIND, bool SCAN>
-cudaError_t launch_main_ks(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
-{
-    if (v.three) {
-        return v.store ? launch_main_t<KIND, true, true, true, SCAN>(p, partials, s)
-                       : launch_main_t<KIND, true, true, false, SCAN>(p, partials, s);
-    }
-    if (v.yard) {
-        return v.store ? launch_main_t<KIND, true, false, true, SCAN>(p, partials, s)
-                       : launch_main_t<KIND, true, false, false, SCAN>(p, partials, s);
-    }
-    return v.store ? launch_main_t<KIND, false, false, true, SCAN>(p, partials, s)
-                   : launch_main_t<KIND, false, false, false, SCAN>(p, partials, s);
-}
-
-template <int KIND>
-cudaError_t launch_main_k(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
-{
-    return v.scan ? launch_main_ks<KIND, true>(v, p, partials, s) : launch_main_ks<KIND, false>(v, p, partials, s);
-}
-
-}  // namespace
+cudaError_t launch_main_tensor(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_row128(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_blk128(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_blk64(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_col128(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_channel(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_dual(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
 {
     if (p.total_tiles == 0) return cudaSuccess;
     switch (v.kind) {
-        case KIND_TENSOR: return launch_main_k<KIND_TENSOR>(v, p, partials, s);
-        case KIND_ROW128: return launch_main_k<KIND_ROW128>(v, p, partials, s);
-        case KIND_BLK128: return launch_main_k<KIND_BLK128>(v, p, partials, s);
-        case KIND_BLK64: return launch_main_k<KIND_BLK64>(v, p, partials, s);
-        case KIND_COL128:    // sub-column blocks: the main kernel always scans (the pre-pass leaves no column keys)
-            return v.scan ? launch_main_ks<KIND_COL128, true>(v, p, partials, s) : cudaErrorInvalidValue;
-        case KIND_DUAL:      // rows and columns of the same tensors from one read: codes are always stored
-            if (!v.store) return cudaErrorInvalidValue;
-            if (v.scan) {
-                return v.three ? launch_main_t<KIND_DUAL, true, true, true, true>(p, partials, s)
-                     : v.yard  ? launch_main_t<KIND_DUAL, true, false, true, true>(p, partials, s)
-                               : launch_main_t<KIND_DUAL, false, false, true, true>(p, partials, s);
-            }
-            return v.three ? launch_main_t<KIND_DUAL, true, true, true, false>(p, partials, s)
-                 : v.yard  ? launch_main_t<KIND_DUAL, true, false, true, false>(p, partials, s)
-                           : launch_main_t<KIND_DUAL, false, false, true, false>(p, partials, s);
-        case KIND_CHANNEL:   // the row amax spans tiles: always taken from the pre-pass
-            return v.scan ? cudaErrorInvalidValue : launch_main_ks<KIND_CHANNEL, false>(v, p, partials, s);
+        case KIND_TENSOR: return launch_main_tensor(v, p, partials, s);
+        case KIND_ROW128: return launch_main_row128(v, p, partials, s);
+        case KIND_BLK128: return launch_main_blk128(v, p, partials, s);
+        case KIND_BLK64: return launch_main_blk64(v, p, partials, s);
+        case KIND_COL128: return launch_main_col128(v, p, partials, s);
+        case KIND_CHANNEL: return launch_main_channel(v, p, partials, s);
+        case KIND_DUAL: return launch_main_dual(v, p, partials, s);
     }
     return cudaErrorInvalidValue;
 }

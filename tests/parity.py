@@ -154,13 +154,18 @@ def _guarded(t):
 def guarded_analyze_quantize(x, recipe: mb.Recipe, *, cols=None, group_amax=None, block_stats=True, fake_quant=False):
     """mor_analyze_quantize through the C boundary with every output buffer (codes, scale bytes, selection
     bytes, binary32 scales, block statistics, tensor summary) placed between guard zones and pre-filled with a
-    pattern.  After the call the guard zones and the padding columns of the codes must still hold the pattern:
-    the library writes nowhere outside what the header says it writes."""
+    pattern.  After the call the guard zones must still hold the pattern, and so must the padding columns of the
+    codes beyond the 16-byte piece that holds a row's last code (that piece is written whole, with the code of
+    zero in its unused bytes, as the header states): the library writes nowhere outside what the header says."""
     import torch
 
     d = mb.desc_for(x, recipe, cols, group_amax)
     o = mb.alloc_outputs(d.rows, d.cols, recipe, x.device, block_stats=block_stats, scale_f32=True,
                          fake_quant_like=x if fake_quant else None)
+    if o.codes is not None and o.codes.numel():
+        # two more 16-byte pieces per row than the call needs: they must stay untouched
+        o.codes = torch.empty((o.codes.shape[0], o.codes.shape[1] + 32), dtype=torch.uint8, device=x.device)
+        o.c_struct.codes_ld = o.codes.shape[1]
     bufs = {}
     for name in ("codes", "scale_e8m0", "sel", "scale_f32", "block_stats", "tensor_stats"):
         t = getattr(o, name)
@@ -182,7 +187,9 @@ def guarded_analyze_quantize(x, recipe: mb.Recipe, *, cols=None, group_amax=None
         assert (buf[:GUARD] == PATTERN).all() and (buf[GUARD + nbytes:] == PATTERN).all(), f"write outside {name}"
     if o.codes is not None and o.codes.numel():
         used = d.rows if o.transposed else d.cols
-        assert (o.codes[:, used:] == PATTERN).all(), "padding columns of the codes were written"
+        piece = (used + 15) // 16 * 16
+        assert (o.codes[:, piece:] == PATTERN).all(), "padding columns of the codes were written"
+        assert (o.codes[:, used:piece] == 0).all(), "unused bytes of a row's last 16-byte piece hold the code of zero"
     return o
 
 
