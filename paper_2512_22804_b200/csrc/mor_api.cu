@@ -60,7 +60,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
-    s.key_words = (uint64_t)s.n_tiles * ((s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL) ? (uint64_t)kTileRows : 4u);
+    s.key_words = (uint64_t)s.n_tiles * ((s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL) ? (uint64_t)kRowKeyStride : (uint64_t)kTileKeyStride);
     if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows;      // + one key per row
     return MOR_OK;
 }
@@ -214,8 +214,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
     r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
-    r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kTileRows : 4u;
-    r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kTileRows : nullptr;
+    r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
+    r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kRowKeyStride : nullptr;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
@@ -388,7 +388,8 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.three = d->n_formats == 3;
     it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
     it.v.store = store;
-    it.v.extra = store && (o.bf16_fallback != nullptr || o.fake_quant != nullptr);
+    it.v.extra = (store && (o.bf16_fallback != nullptr || o.fake_quant != nullptr)) || o.block_stats != nullptr ||
+                 d->criterion == MOR_CRIT_BLOCK_MEAN_REL || (d->flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) != 0;
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
     // Nor is it needed where the scale has no shared mantissa (E8M0 and FP32-amax modes): those need the block

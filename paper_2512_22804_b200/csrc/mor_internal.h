@@ -21,6 +21,8 @@ constexpr int kSegsPerTile = 128;
 constexpr int kSegElems = 128;
 constexpr int kThreads = 256;          // amax and finalise kernels; compute threads of the main kernel
 constexpr int kMainThreads = 320;      // 8 compute warps + load warp + store warp
+constexpr int kRowKeyStride = kTileRows + 4;   // 128 block keys + the count of finite non-zero elements of the tile (+ padding to 16 bytes)
+constexpr int kTileKeyStride = 8;              // up to 4 block keys + the count (+ padding)
 constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor maps travel as kernel parameters
 
 enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3, KIND_CHANNEL = 4, KIND_COL128 = 5,
@@ -53,8 +55,9 @@ struct TensorRec {
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
     uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows
-    uint32_t key_stride;          // words per tile in `keys`: 128 (one key per row piece) or 4 (one per tile, or one
-                                  // per 64x64 quadrant in the order top-left, top-right, bottom-left, bottom-right)
+    uint32_t key_stride;          // words per tile in `keys`: kRowKeyStride (one key per row piece, then the tile's
+                                  // non-zero count) or kTileKeyStride (one key per tile, or one per 64x64 quadrant in the
+                                  // order top-left, top-right, bottom-left, bottom-right; word 4: the tile's non-zero count)
     int64_t rows, cols, ld, codes_ld;
     uint32_t nbc;                 // tile columns = ceil(cols / 128)
     uint32_t nbr;                 // tile rows = ceil(rows / 128)
@@ -96,7 +99,9 @@ struct MainVariant {
     bool three;      // three-way recipe: keep E5M2 codes and the non-zero minimum (Eq. 4)
     bool store;      // write codes (false for mor_select_stats)
     bool scan;       // the kernel scans the data for amax / smallest non-zero itself (no keys from the pre-pass)
-    bool extra;      // some tensor of the launch wants a BF16 copy of rejected blocks or the fake-quantised output
+    bool extra;      // some tensor of the launch wants more than codes, scales, selection and the tensor summary: a BF16
+                     // copy of rejected blocks, the fake-quantised output, block statistics, or a decision that needs the
+                     // per-block count of non-zeros (Eq. 1-2 per block; the literal minimum of Eq. 4)
 };
 
 // Programmatic dependent launch: a kernel launched with launch_dependent() may become resident while the

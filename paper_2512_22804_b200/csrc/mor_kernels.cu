@@ -112,7 +112,7 @@ __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __v
 __global__ void __launch_bounds__(kThreads)
 mor_amax_kernel(const __grid_constant__ BatchParams p)
 {
-    __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32];
+    __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32], s_wnz[kThreads / 32];
     __shared__ uint32_t s_qkey[kThreads / 32][4], s_qnf[kThreads / 32][4];   // 64x64 blocks: per warp and quadrant
 
     pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
@@ -149,8 +149,19 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             }
         }
     }
-    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kTileRows;
+    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride;
     uint32_t key[8], all = 0u, nf = 0u;
+    // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once.  The
+    // main kernel takes the tile's count from here and need not count while it converts.
+    uint32_t nz2 = 0u;
+    if (R.keys != nullptr) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            nz2 += __vimin3_u16x2(v[j].x & 0x7FFF7FFFu, 0x00010001u, 0x00010001u) + __vimin3_u16x2(v[j].y & 0x7FFF7FFFu, 0x00010001u, 0x00010001u);
+            nz2 += __vimin3_u16x2(v[j].z & 0x7FFF7FFFu, 0x00010001u, 0x00010001u) + __vimin3_u16x2(v[j].w & 0x7FFF7FFFu, 0x00010001u, 0x00010001u);
+        }
+    }
+    uint32_t nz = (nz2 & 0xFFFFu) + (nz2 >> 16);
     if (per_piece) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) { key[j] = key_of_chunk(v[j]); all = key_max(all, key[j]); }
@@ -187,7 +198,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     if (per_piece) {
         // one key per row piece: combine the 16 lanes that share the piece
         const uint32_t half = (lane & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-        uint32_t* kp = R.keys + (size_t)local * kTileRows + (t >> 4);
+        uint32_t* kp = R.keys + (size_t)local * kRowKeyStride + (t >> 4);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t kk = key[j];
@@ -226,18 +237,21 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     }
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
-    if (lane == 0) { s_wkey[warp] = (hi << 16) | lo; s_wnf[warp] = nf; }
+    nz = __reduce_add_sync(0xFFFFFFFFu, nz);
+    if (lane == 0) { s_wkey[warp] = (hi << 16) | lo; s_wnf[warp] = nf; s_wnz[warp] = nz; }
     __syncthreads();
     if (t == 0) {
         uint32_t kk = s_wkey[0];
-        for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; }
+        for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; nz += s_wnz[i]; }
+        // finite non-zero elements of the tile (NaN and inf are non-zero patterns: taken off)
+        if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (per_piece ? (uint32_t)kTileRows : 4u)] = nz - nf;
         if (R.keys != nullptr && R.kind == KIND_BLK64) {
             for (int q = 0; q < 4; ++q) {
                 uint32_t kq = s_qkey[0][q], nq = s_qnf[0][q];
                 for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, s_qkey[i][q]); nq |= s_qnf[i][q]; }
-                R.keys[(size_t)local * 4 + q] = kq | (nq ? 0x80000000u : 0u);
+                R.keys[(size_t)local * kTileKeyStride + q] = kq | (nq ? 0x80000000u : 0u);
             }
-        } else if (R.keys != nullptr && R.key_stride != (uint32_t)kTileRows) {
+        } else if (R.keys != nullptr && !per_piece) {
             R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
         }
         // non-negative binary32 patterns order like the values
@@ -255,9 +269,9 @@ mor_row_keys_kernel(const __grid_constant__ BatchParams p)
     pdl_trigger();
     const TensorRec& R = p.t[blockIdx.y];
     if (R.kind != KIND_CHANNEL || R.row_keys == nullptr || blockIdx.x >= R.nbr) return;
-    const uint32_t* src = R.keys + ((size_t)blockIdx.x * R.nbc) * kTileRows + threadIdx.x;
+    const uint32_t* src = R.keys + ((size_t)blockIdx.x * R.nbc) * kRowKeyStride + threadIdx.x;
     uint32_t k = 0u, flag = 0u;
-    for (uint32_t j = 0; j < R.nbc; ++j, src += kTileRows) {
+    for (uint32_t j = 0; j < R.nbc; ++j, src += kRowKeyStride) {
         const uint32_t v = *src;
         flag |= v & 0x80000000u;
         k = key_max(k, v & 0x7FFFFFFFu);

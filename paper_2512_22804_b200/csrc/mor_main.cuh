@@ -62,7 +62,7 @@ struct __align__(16) TileMeta {
     uint32_t blk_base;     // ROW128: index of the block of the tile's first row
     uint32_t local;        // tile index within the tensor
     int32_t row0, col0;    // first row / column of the tile
-    uint32_t pad;
+    uint32_t nnz;          // finite non-zero elements of the tile, counted by the pre-pass (prepared tiles only)
 };
 
 // What a compute thread hands to the store warp: its (ROW128: its block's) sums and counts.
@@ -78,7 +78,9 @@ struct Control {
     unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
     unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
     TileMeta meta[kStages];
-    uint32_t keys[kStages][kTileRows];                   // block keys of the tile from the pre-pass (arrive with the tile)
+    uint32_t keys[kStages][kRowKeyStride];               // block keys of the tile from the pre-pass (arrive with the tile)
+    uint32_t prep[kStages][kTileRows];                   // by the load warp, from the keys: scale bits of the row's block (entry = row),
+                                                         // of the quadrant (entry q) or of the tile (entry 0); bit 31: careful path
     Entry entry[2][kThreads];
     // 128x128 and 64x64 blocks (a tile holds one block, or four: index q = 2 * (row >= 64) + (column >= 64))
     uint32_t wmax[2][2][2 * kComputeWarps];              // per tile parity, per pass: warp (and column half) amax | inverted min
@@ -425,9 +427,9 @@ __device__ __forceinline__ void raise_amax(float* slot, uint32_t bits, bool acti
 // term = |y - q| / |y|, formed as |y - q| * |rcp(y + 2^-126)| (the sum inside a fused
 // multiply-add).  The caller guarantees that the block holds no NaN/inf and that every non-zero
 // |y| is at least 2^-100, so the added constant changes a term by less than 2^-26 relative, and a
-// zero element gives 0 * 2^126.  The same reciprocal counts the non-zeros: y * rcp is 1 for a
+// zero element gives 0 * 2^126.  With COUNT the same reciprocal counts the non-zeros: y * rcp is 1 for a
 // non-zero element (within 2^-22) and 0 for a zero.  Pair p of the quad adds into a43[p], a52[p], cnt2[p].
-template <bool YARD>
+template <bool YARD, bool COUNT>
 __device__ __forceinline__ void convert_quad_fast(uint32_t w0, uint32_t w1, unsigned long long s4x2,
                                                   unsigned long long tiny2, float (&a43)[2], float (&a52)[2],
                                                   unsigned long long (&cnt2)[2], uint32_t& c4)
@@ -443,8 +445,10 @@ __device__ __forceinline__ void convert_quad_fast(uint32_t w0, uint32_t w1, unsi
     unpack_f32x2(fma_f32x2(xa, s4x2, tiny2), u0, u1);
     unpack_f32x2(fma_f32x2(xb, s4x2, tiny2), u2, u3);
     const float r0 = rcp_ftz(u0), r1 = rcp_ftz(u1), r2 = rcp_ftz(u2), r3 = rcp_ftz(u3);
-    cnt2[0] = fma_f32x2(ya, pack_f32x2(r0, r1), cnt2[0]);
-    cnt2[1] = fma_f32x2(yb, pack_f32x2(r2, r3), cnt2[1]);
+    if (COUNT) {
+        cnt2[0] = fma_f32x2(ya, pack_f32x2(r0, r1), cnt2[0]);
+        cnt2[1] = fma_f32x2(yb, pack_f32x2(r2, r3), cnt2[1]);
+    }
     uint32_t qa, qb;
     cast4_e4m3(y0, y1, y2, y3, c4, qa, qb);
     float d0, d1, d2, d3;
@@ -543,7 +547,7 @@ __device__ __forceinline__ void conv_init(ConvAcc& c)
 // NCH chunks of 4 words (8 elements each) of a thread's 64 elements; chunk j0 + j belongs at byte offset
 // ((j0 + j) ^ swz) * 8 of the thread's 64 code bytes (out_addr has the swizzle folded in).  The E4M3 codes go to
 // the staging buffer; a block that ends up in E5M2 has them replaced afterwards (emit_e5m2_codes).
-template <bool YARD, bool CAREFUL, bool STORE, int NCH>
+template <bool YARD, bool CAREFUL, bool STORE, int NCH, bool COUNT = true>
 __device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uint32_t out_addr, int j0, uint32_t s4b, uint32_t s5b, ConvAcc& c)
 {
     const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
@@ -559,29 +563,33 @@ __device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uin
             uint32_t c4[2];
 #pragma unroll
             for (int k = 0; k < 2; ++k)
-                convert_quad_fast<YARD>(w[4 * j + 2 * k], w[4 * j + 2 * k + 1], s4x2, tiny2, c.q43[k], c.q52[k], c.cnt2, c4[k]);
+                convert_quad_fast<YARD, COUNT>(w[4 * j + 2 * k], w[4 * j + 2 * k + 1], s4x2, tiny2, c.q43[k], c.q52[k], c.cnt2, c4[k]);
             if (STORE) sts64(out_addr ^ ((j0 + j) << 3), make_uint2(c4[0], c4[1]));
         }
     }
 }
 
 // Results: e43 = the thread's sum of E4M3 terms, complete; e52 = its sum of E5M2 terms, complete; nnz; nonfinite.
-template <bool YARD, bool CAREFUL>
+// (Without COUNT the fast path reports no non-zeros: the caller has the tile's count from the pre-pass.)
+template <bool YARD, bool CAREFUL, bool COUNT = true>
 __device__ __forceinline__ void conv_finish(const ConvAcc& c, uint32_t s4b, uint32_t s5b, float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite)
 {
     if (CAREFUL) {
         // scale4 / scale5 = 2^(e4 - e5)
         const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);
         const float tiny = (float)(c.A.nnz - c.A.nbig);
-        nnz = c.A.nnz;
+        nnz = COUNT ? c.A.nnz : 0u;
         nonfinite = c.A.nonfinite;
         e43 = c.A.a43 + tiny;
         e52 = YARD ? c.A.a52 * ratio + tiny : 0.0f;
     } else {
-        float c0, c1, c2, c3;
-        unpack_f32x2(c.cnt2[0], c0, c1);
-        unpack_f32x2(c.cnt2[1], c2, c3);
-        nnz = (uint32_t)__float2int_rn((c0 + c1) + (c2 + c3));
+        nnz = 0u;
+        if (COUNT) {
+            float c0, c1, c2, c3;
+            unpack_f32x2(c.cnt2[0], c0, c1);
+            unpack_f32x2(c.cnt2[1], c2, c3);
+            nnz = (uint32_t)__float2int_rn((c0 + c1) + (c2 + c3));
+        }
         nonfinite = 0u;
         e43 = (c.q43[0][0] + c.q43[0][1]) + (c.q43[1][0] + c.q43[1][1]);
         e52 = YARD ? ((c.q52[0][0] + c.q52[0][1]) + (c.q52[1][0] + c.q52[1][1])) * 0.0078125f : 0.0f;
@@ -589,14 +597,14 @@ __device__ __forceinline__ void conv_finish(const ConvAcc& c, uint32_t s4b, uint
 }
 
 // A thread's 64 elements, held as 8 chunks of 4 words, in one go.
-template <bool YARD, bool CAREFUL, bool STORE>
+template <bool YARD, bool CAREFUL, bool STORE, bool COUNT = true>
 __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t out_addr, uint32_t s4b, uint32_t s5b,
                                               float& e43, float& e52, uint32_t& nnz, uint32_t& nonfinite)
 {
     ConvAcc c;
     conv_init(c);
-    convert_chunks<YARD, CAREFUL, STORE, 8>(w, out_addr, 0, s4b, s5b, c);
-    conv_finish<YARD, CAREFUL>(c, s4b, s5b, e43, e52, nnz, nonfinite);
+    convert_chunks<YARD, CAREFUL, STORE, 8, COUNT>(w, out_addr, 0, s4b, s5b, c);
+    conv_finish<YARD, CAREFUL, COUNT>(c, s4b, s5b, e43, e52, nnz, nonfinite);
 }
 
 // The E5M2 codes of a thread's 64 elements, for a block that selected E5M2 (such a block holds no
@@ -690,42 +698,103 @@ __device__ __forceinline__ double shfl_xor_f64(double v, int o) { return __shfl_
 
 // ------------------------------------------------------------------ load warp ----
 
-// One thread: start the TMA load of the CTA's tile number `it` into its stage (nothing when the CTA
-// has no such tile).  The stage must be free.
-__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it)
+// The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_quad_fast), no NaN/inf, and an
+// E5M2 exponent that is not capped at 254 (the fast path takes scale5 = 128 scale4).
+__device__ __forceinline__ bool needs_careful(bool nonfin, uint32_t minm1, uint32_t s4b)
+{
+    bool careful = nonfin || (s4b >> 23) > 247u;
+    if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
+    return careful;
+}
+
+// The load warp.  For the CTA's tile number `it`: lane 0 starts the TMA load into the tile's stage (the stage must be
+// free) and the bulk copy of the tile's keys.  With PREP (the pre-pass left keys: nothing has to be scanned) the warp
+// also turns the keys into what the compute threads need -- per row, quadrant or tile the scale of Algorithm 1 and
+// whether the careful path is needed -- so that 256 threads need not each derive them.  The stage's barrier takes two
+// arrivals: one with the byte count when the copies start, one when the tile's facts are in shared memory.
+template <int KIND, bool PREP>
+__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it, int lane,
+                                                int& cur_ti, uint32_t& m_g, int& scale_mode, uint32_t& tensor_amax_bits)
 {
     const uint32_t tile = blockIdx.x + it * gridDim.x;
     if (tile >= p.total_tiles) return;
     const uint32_t s = it % kStages;
     const TileId t = locate_tile(p.b, tile);
-    TileMeta m;
-    m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
-    m.blk_base = (uint32_t)t.row0 * p.b.t[t.ti].nbc + (uint32_t)(t.col0 / kTileCols);
-    if (p.b.t[t.ti].kind == KIND_COL128) m.blk_base = (uint32_t)(t.row0 / kTileRows) * (uint32_t)p.b.t[t.ti].cols + (uint32_t)t.col0;
-    if (p.b.t[t.ti].kind == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
-    m.pad = 0;
-    C.meta[s] = m;
     const TensorRec& R = p.b.t[t.ti];
-    const uint32_t key_bytes = R.keys != nullptr ? R.key_stride * 4u : 0u;
-    mbar_arrive_expect_tx(&C.full[s], kInBytes + key_bytes);
-    tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
-    if (key_bytes) {
-        const uint32_t* src = R.kind == KIND_CHANNEL ? R.row_keys + t.row0 : R.keys + (size_t)t.local * R.key_stride;
-        bulk_load(&C.keys[s][0], src, key_bytes, &C.full[s]);
+    const uint32_t key_bytes = R.keys == nullptr ? 0u : (KIND == KIND_CHANNEL ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
+    const uint32_t* key_src = KIND == KIND_CHANNEL ? R.row_keys + t.row0 : R.keys + (size_t)t.local * R.key_stride;
+    if (lane == 0) {
+        mbar_arrive_expect_tx(&C.full[s], kInBytes + key_bytes);
+        tma_load_tile(in + s * kInBytes, &p.in_map[t.ti], t.col0, t.row0, &C.full[s]);
+        if (key_bytes) bulk_load(&C.keys[s][0], key_src, key_bytes, &C.full[s]);
     }
-    C.issued = it + 1;
+    uint32_t tile_nnz = 0u;
+    if (PREP) {
+        if (t.ti != cur_ti) {
+            cur_ti = t.ti;
+            scale_mode = R.scale_mode;
+            m_g = group_mantissa(*R.amax, scale_mode);
+            if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
+        }
+        tile_nnz = R.keys[(size_t)t.local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)];
+        if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL) {
+            uint32_t key[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) key[k] = key_src[lane + 32 * k];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const bool nonfin = (key[k] >> 31) != 0u;
+                const uint32_t kk = key[k] & 0x7FFFFFFFu;
+                uint32_t s4b, s5b;
+                block_scale(kk >> 16, m_g, scale_mode, C.rtab, s4b, s5b);
+                // the careful path is taken by a warp as a whole: rows 16 w .. 16 w + 15, i.e. this half of the lanes
+                const uint32_t any = __ballot_sync(0xFFFFFFFFu, needs_careful(nonfin, 0xFFFFu - (kk & 0xFFFFu), s4b));
+                const bool careful = ((lane < 16 ? any : any >> 16) & 0xFFFFu) != 0u;
+                C.prep[s][lane + 32 * k] = s4b | (careful ? 0x80000000u : 0u);
+            }
+        } else {
+            // one key per tile, or one per quadrant (lanes 0..3; the other lanes repeat lane 0's work)
+            const uint32_t q = KIND == KIND_BLK64 ? (uint32_t)(lane & 3) : 0u;
+            const uint32_t key = key_src[q];
+            const bool nonfin = (key >> 31) != 0u;
+            const uint32_t kk = key & 0x7FFFFFFFu;
+            uint32_t s4b, s5b;
+            block_scale(KIND == KIND_TENSOR ? tensor_amax_bits : kk >> 16, m_g, scale_mode, C.rtab, s4b, s5b);
+            bool careful = needs_careful(nonfin, 0xFFFFu - (kk & 0xFFFFu), s4b);
+            // 64x64: a warp covers both column halves of its rows, and takes the careful path as a whole
+            if (KIND == KIND_BLK64) {
+                const int other = __shfl_xor_sync(0xFFFFFFFFu, (int)careful, 1);   // (every lane takes part: no short-circuit)
+                careful = careful || other != 0;
+            }
+            if (lane < (KIND == KIND_BLK64 ? 4 : 1)) C.prep[s][lane] = s4b | (careful ? 0x80000000u : 0u);
+        }
+    }
+    if (lane == 0) {
+        TileMeta m;
+        m.ti = t.ti; m.local = t.local; m.row0 = t.row0; m.col0 = t.col0; m.vrows = t.vrows; m.vcols = t.vcols;
+        m.blk_base = (uint32_t)t.row0 * R.nbc + (uint32_t)(t.col0 / kTileCols);
+        if (KIND == KIND_COL128) m.blk_base = (uint32_t)(t.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)t.col0;
+        if (KIND == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
+        m.nnz = tile_nnz;
+        C.meta[s] = m;
+        C.issued = it + 1;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&C.full[s]);             // the tile's facts are in place (release)
 }
 
+template <int KIND, bool PREP>
 __device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in, int lane)
 {
-    if (lane == 0) {
-        for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load(p, C, in, it);
-    }
+    int cur_ti = -1, scale_mode = 0;
+    uint32_t m_g = 0u, tensor_amax_bits = 0u;
+    for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load<KIND, PREP>(p, C, in, it, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
         stage_free_sync(it % kStages);                  // sleeps until every compute thread has its copy
-        if (lane == 0 && !C.abort) issue_tile_load(p, C, in, it + kStages);
+        if (!__any_sync(0xFFFFFFFFu, C.abort != 0u))
+            issue_tile_load<KIND, PREP>(p, C, in, it + kStages, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
     }
     if (lane == 0 && C.abort) {
         // copies that may still be in flight must land (or be given up on) before the CTA goes
@@ -979,8 +1048,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     int scale_mode = 0;
     bool has_fallback = false;
     bool has_fq = false, fq_e4m3 = false;   // fake-quantised output wanted; ... with E4M3 values whatever the block's selection
-    uint32_t tensor_amax_bits = 0;
-    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]);
+    const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]), prep_base = smem_addr(&C.prep[0][0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
@@ -996,8 +1064,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         {
             const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
             m.ti = dead ? 0 : (int32_t)q.x; m.vrows = (int32_t)q.y; m.vcols = (int32_t)q.z; m.blk_base = q.w;
-            m.local = 0; m.row0 = 0; m.col0 = 0; m.pad = 0;
+            m.local = 0; m.row0 = 0; m.col0 = 0; m.nnz = 0;
         }
+        // What the thread has to find out itself.  With keys from the pre-pass (no SCAN) the load warp has prepared the
+        // block's scale; the key itself (amax, smallest non-zero) is then needed only for Eq. 4 and for statistics,
+        // and the non-zeros are counted per thread only where a per-block count is wanted (EXTRA) -- otherwise the
+        // tile's count comes from the pre-pass and travels in thread 0's entry.
+        constexpr bool kNeedKey = SCAN || THREE || EXTRA;
+        constexpr bool kCount = SCAN || EXTRA;
         // Two ways through a tile.  Streaming (keys from the pre-pass, no second use of the data): the scale is known
         // before any element is read, so the thread converts its 64 elements in two halves straight from the stage,
         // 16 registers of data at a time, and hands the stage back after the second half's loads.  Otherwise the 64
@@ -1030,34 +1104,33 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
         }
         const TensorRec& R = p.b.t[m.ti];
-        if (m.ti != cur_ti) {
+        if ((SCAN || EXTRA) && m.ti != cur_ti) {
             cur_ti = m.ti;
-            scale_mode = R.scale_mode;
-            has_fallback = EXTRA && R.fallback != nullptr;
-            has_fq = EXTRA && R.fake_quant != nullptr;
+            has_fallback = EXTRA && STORE && R.fallback != nullptr;
+            has_fq = EXTRA && STORE && R.fake_quant != nullptr;
             fq_e4m3 = KIND == KIND_TENSOR || KIND == KIND_CHANNEL || R.criterion == MOR_CRIT_TENSOR_MEAN_REL;
-            if (!dead) {
-                m_g = group_mantissa(*R.amax, scale_mode);
-                if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
+            if (SCAN) {
+                scale_mode = R.scale_mode;
+                if (!dead) m_g = group_mantissa(*R.amax, scale_mode);
             }
         }
-        if (EXTRA && (has_fallback || has_fq)) {      // the BF16 outputs need the tile's position too
+        if (EXTRA || (!kCount && tid == 0)) {          // the tile's position (BF16 outputs) and its non-zero count
             const uint4 q = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
-            m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z;
+            m.local = q.x; m.row0 = (int32_t)q.y; m.col0 = (int32_t)q.z; m.nnz = q.w;
         }
-        uint32_t key = 0u;
+        uint32_t key = 0u, prep = 0u;
         if (!SCAN) {
-            // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + ((KIND == KIND_ROW128 || KIND == KIND_CHANNEL) ? (uint32_t)row * 4u : (uint32_t)q * 4u)));
+            // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero; the load warp made the scale
+            const uint32_t e = (KIND == KIND_ROW128 || KIND == KIND_CHANNEL) ? (uint32_t)row * 4u : (uint32_t)q * 4u;
+            if (kNeedKey) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kRowKeyStride * 4) + e));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(prep) : "r"(prep_base + s * (uint32_t)(kTileRows * 4) + e));
         }
         if (!kStream) stage_free_arrive(s);             // this thread's copy of the stage is in registers
 
         // ---- block amax and smallest non-zero (Algorithm 1; Eq. 4) ----
         bool nonfin = false;
         if (!SCAN) {
-            nonfin = (key >> 31) != 0u;
-            key &= 0x7FFFFFFFu;
-            if (KIND != KIND_BLK128) nonfin = __any_sync(0xFFFFFFFFu, nonfin);   // warp-uniform (a tile-wide key is CTA-uniform already)
+            key &= 0x7FFFFFFFu;                         // (the flag for NaN/inf is part of the prepared word)
         } else if (kLineBlocks) {
             key = scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
@@ -1113,18 +1186,20 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         }
         uint32_t amax_bits = key >> 16;
         const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
-        // per-tensor partition: the block is the tensor, its amax was reduced by the pre-pass
-        if (KIND == KIND_TENSOR) amax_bits = tensor_amax_bits;
 
         uint32_t s4b, s5b;
-        block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
-
-        // The fast path needs every non-zero |x * scale| to be at least 2^-100 (see convert_pair_fast).
-        // minm1 covers this thread's block (ROW128), this tile (BLK128), this thread (TENSOR).
-        bool careful = nonfin;
-        if (minm1 != 0xFFFFu) careful = careful || !(__fmul_rn(minnz_value(minm1), __uint_as_float(s4b)) >= 7.888609052210118e-31f);
-        careful = careful || (s4b >> 23) > 247u;        // E5M2 exponent capped at 254: the fast path takes scale5 = 128 scale4
-        if (KIND != KIND_BLK128) careful = __any_sync(0xFFFFFFFFu, careful);
+        bool careful;
+        if (!SCAN) {
+            // prepared by the load warp: the scale of Algorithm 1 and, warp-uniform, whether the careful path is needed
+            s4b = prep & 0x7FFFFFFFu;
+            s5b = (min((s4b >> 23) + 7u, 254u) << 23) | (s4b & 0x7FFFFFu);
+            careful = (prep >> 31) != 0u;
+        } else {
+            block_scale(amax_bits, m_g, scale_mode, C.rtab, s4b, s5b);
+            // minm1 covers this thread's block (1x128), this tile (128x128), this quadrant (64x64)
+            careful = needs_careful(nonfin, minm1, s4b);
+            if (KIND != KIND_BLK128) careful = __any_sync(0xFFFFFFFFu, careful);
+        }
 
         // ---- staging buffer and entries of tile it - 2 must have been consumed ----
         if (n2 > 0 && !dead) {
@@ -1153,9 +1228,9 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
                         if (half == 1) stage_free_arrive(s);
-                        convert_chunks<YARD, true, STORE, 4>(wh, oa, 4 * half, s4b, s5b, acc);
+                        convert_chunks<YARD, true, STORE, 4, kCount>(wh, oa, 4 * half, s4b, s5b, acc);
                     }
-                    conv_finish<YARD, true>(acc, s4b, s5b, e43, e52, nnz, nonf);
+                    conv_finish<YARD, true, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 } else {
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
@@ -1166,15 +1241,16 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
                         if (half == 1) stage_free_arrive(s);
-                        convert_chunks<YARD, false, STORE, 4>(wh, oa, 4 * half, s4b, s5b, acc);
+                        convert_chunks<YARD, false, STORE, 4, kCount>(wh, oa, 4 * half, s4b, s5b, acc);
                     }
-                    conv_finish<YARD, false>(acc, s4b, s5b, e43, e52, nnz, nonf);
+                    conv_finish<YARD, false, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 }
             } else if (careful) {
-                convert_words<YARD, true, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
+                convert_words<YARD, true, STORE, kCount>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
             } else {
-                convert_words<YARD, false, STORE>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
+                convert_words<YARD, false, STORE, kCount>(w, oa, s4b, s5b, e43, e52, nnz, nonf);
             }
+            if (!kCount && tid == 0) nnz = m.nnz;       // the tile's count from the pre-pass, handed on in this thread's entry
 
             if (kLineBlocks) {
                 // ---- block sums, decision, metadata ----
@@ -1280,7 +1356,7 @@ __device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control&
             const uint4 q0 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
             const uint4 q1 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta) + 16u);
             m.ti = dead ? 0 : (int32_t)q0.x; m.vrows = (int32_t)q0.y; m.vcols = (int32_t)q0.z; m.blk_base = q0.w;
-            m.local = q1.x; m.row0 = (int32_t)q1.y; m.col0 = (int32_t)q1.z; m.pad = 0;
+            m.local = q1.x; m.row0 = (int32_t)q1.y; m.col0 = (int32_t)q1.z; m.nnz = q1.w;
         }
         if (m.ti != cur_ti) {
             cur_ti = m.ti;
@@ -1301,7 +1377,7 @@ __device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control&
                     const uint4 v = lds128(a ^ (j << 4));
                     w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
                 }
-                if (!SCAN) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)row * 4u));
+                if (!SCAN) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kRowKeyStride * 4) + (uint32_t)row * 4u));
             } else {
                 // this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows per word
                 const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
@@ -1400,7 +1476,7 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) mbar_init(&C.full[s], 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(&C.full[s], 2);   // copies started (with the byte count) + tile facts written
         for (int b = 0; b < 2; ++b) {
             mbar_init(&C.out_empty[b], 1);
             mbar_init(&C.dec_full[b], 1);
@@ -1423,14 +1499,13 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
         if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
         else compute_warps<KIND, YARD, THREE, STORE, SCAN, EXTRA>(p, C, in, out, tid);
     }
-    else if (warp == kLoadWarp) load_warp(p, C, in, lane);
+    else if (warp == kLoadWarp) load_warp<KIND, !SCAN && KIND != KIND_DUAL && KIND != KIND_COL128>(p, C, in, lane);
     else store_warp<KIND, THREE, STORE, EXTRA>(p, C, out, partials, lane);
 }
 
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN, bool EXTRA>
 cudaError_t launch_main_t(const MainParams& p, Partial* partials, cudaStream_t s)
 {
-    static_assert(STORE || !EXTRA, "the BF16 outputs come with the codes");
     auto kfn = mor_main_kernel<KIND, YARD, THREE, STORE, SCAN, EXTRA>;
     static std::atomic<int> sm_count[64];   // per instantiation and device; 0 = not set up yet
     static std::mutex setup;
@@ -1458,10 +1533,12 @@ template <int KIND, bool SCAN>
 cudaError_t launch_main_ks(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
 {
 #define MOR_LAUNCH(Y, T, S, E) launch_main_t<KIND, Y, T, S, SCAN, E>(p, partials, s)
-    if (!v.store && v.extra) return cudaErrorInvalidValue;
-    if (v.three) return v.store ? (v.extra ? MOR_LAUNCH(true, true, true, true) : MOR_LAUNCH(true, true, true, false)) : MOR_LAUNCH(true, true, false, false);
-    if (v.yard) return v.store ? (v.extra ? MOR_LAUNCH(true, false, true, true) : MOR_LAUNCH(true, false, true, false)) : MOR_LAUNCH(true, false, false, false);
-    return v.store ? (v.extra ? MOR_LAUNCH(false, false, true, true) : MOR_LAUNCH(false, false, true, false)) : MOR_LAUNCH(false, false, false, false);
+#define MOR_LAUNCH_SE(Y, T) (v.store ? (v.extra ? MOR_LAUNCH(Y, T, true, true) : MOR_LAUNCH(Y, T, true, false)) \
+                                     : (v.extra ? MOR_LAUNCH(Y, T, false, true) : MOR_LAUNCH(Y, T, false, false)))
+    if (v.three) return MOR_LAUNCH_SE(true, true);
+    if (v.yard) return MOR_LAUNCH_SE(true, false);
+    return MOR_LAUNCH_SE(false, false);
+#undef MOR_LAUNCH_SE
 #undef MOR_LAUNCH
 }
 

@@ -213,6 +213,11 @@ def run_and_compare(bits: np.ndarray, recipe: mb.Recipe, *, cols=None, block_sta
         ga = torch.tensor([ref.tensor["group_amax"]], dtype=torch.float32, device="cuda")
     out = guarded_analyze_quantize(x, recipe, cols=cols, group_amax=ga, block_stats=block_stats, fake_quant=fake_quant)
     rep = compare(host, recipe, out, ref, cols=cols)
+    if block_stats and not fake_quant:
+        # the same call without the optional outputs runs the plain instantiation of the kernel (no per-thread
+        # counts, no keys in the compute threads): same bar
+        plain = guarded_analyze_quantize(x, recipe, cols=cols, group_amax=ga, block_stats=False, fake_quant=False)
+        compare(host, recipe, plain, ref, cols=cols)
     if fake_quant:
         # the fake-quantised tensor, bit for bit, outside blocks whose decision is within the tolerance band;
         # padding columns must stay untouched (zero-initialised output)
