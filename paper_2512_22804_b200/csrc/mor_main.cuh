@@ -192,6 +192,12 @@ __device__ __forceinline__ uint4 lds128(uint32_t a)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
 }
+__device__ __forceinline__ uint2 lds64(uint32_t a)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ void sts128(uint32_t a, uint4 v)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -432,7 +438,7 @@ __device__ __forceinline__ void raise_amax(float* slot, uint32_t bits, bool acti
 template <bool YARD, bool COUNT>
 __device__ __forceinline__ void convert_quad_fast(uint32_t w0, uint32_t w1, unsigned long long s4x2,
                                                   unsigned long long tiny2, float (&a43)[2], float (&a52)[2],
-                                                  unsigned long long (&cnt2)[2], uint32_t& c4)
+                                                  unsigned long long (&cnt2)[2], uint32_t& c4, uint32_t& c5)
 {
     float x0, x1, x2, x3;
     unpack_bf16x2(w0, x0, x1);
@@ -465,8 +471,7 @@ __device__ __forceinline__ void convert_quad_fast(uint32_t w0, uint32_t w1, unsi
         float z0, z1, z2, z3;
         unpack_f32x2(mul_f32x2(ya, k128), z0, z1);
         unpack_f32x2(mul_f32x2(yb, k128), z2, z3);
-        uint32_t c5;                                   // not kept: a block that selects E5M2 has its codes made afterwards
-        cast4_e5m2(z0, z1, z2, z3, c5, qa, qb);
+        cast4_e5m2(z0, z1, z2, z3, c5, qa, qb);           // (the codes are kept only where the caller stashes them)
         diff_f16x2_f32(qa, z0, z1, d0, d1);
         diff_f16x2_f32(qb, z2, z3, d2, d3);
         // |z - q'| / |z| = |z - q'| * (1/|y|) / 128; the factor is applied once per block
@@ -474,6 +479,8 @@ __device__ __forceinline__ void convert_quad_fast(uint32_t w0, uint32_t w1, unsi
         a52[0] = fmaf(fabsf(d1), fabsf(r1), a52[0]);
         a52[1] = fmaf(fabsf(d2), fabsf(r2), a52[1]);
         a52[1] = fmaf(fabsf(d3), fabsf(r3), a52[1]);
+    } else {
+        c5 = 0u;
     }
 }
 
@@ -547,8 +554,11 @@ __device__ __forceinline__ void conv_init(ConvAcc& c)
 // NCH chunks of 4 words (8 elements each) of a thread's 64 elements; chunk j0 + j belongs at byte offset
 // ((j0 + j) ^ swz) * 8 of the thread's 64 code bytes (out_addr has the swizzle folded in).  The E4M3 codes go to
 // the staging buffer; a block that ends up in E5M2 has them replaced afterwards (emit_e5m2_codes).
-template <bool YARD, bool CAREFUL, bool STORE, int NCH, bool COUNT = true>
-__device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uint32_t out_addr, int j0, uint32_t s4b, uint32_t s5b, ConvAcc& c)
+// With STASH the E5M2 codes are kept as well: chunk j0 + j's eight codes go to stash_addr ^ ((j0 + j) << 4), which
+// is the place of the chunk's own (already consumed) input in the stage.
+template <bool YARD, bool CAREFUL, bool STORE, int NCH, bool COUNT = true, bool STASH = false>
+__device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uint32_t out_addr, int j0, uint32_t s4b, uint32_t s5b, ConvAcc& c,
+                                               uint32_t stash_addr = 0u)
 {
     const float s4 = __uint_as_float(s4b), s5 = __uint_as_float(s5b);
     const unsigned long long s4x2 = pack_f32x2(s4, s4), tiny2 = pack_f32x2(FLT_MIN, FLT_MIN);
@@ -559,12 +569,14 @@ __device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uin
 #pragma unroll
             for (int i = 0; i < 4; ++i) convert_pair_careful<YARD>(w[4 * j + i], s4, s5, c.A, a[i], b[i]);
             if (STORE) sts64(out_addr ^ ((j0 + j) << 3), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
+            if (STASH) sts64(stash_addr ^ ((j0 + j) << 4), make_uint2(__byte_perm(b[0], b[1], 0x5410), __byte_perm(b[2], b[3], 0x5410)));
         } else {
-            uint32_t c4[2];
+            uint32_t c4[2], c5[2];
 #pragma unroll
             for (int k = 0; k < 2; ++k)
-                convert_quad_fast<YARD, COUNT>(w[4 * j + 2 * k], w[4 * j + 2 * k + 1], s4x2, tiny2, c.q43[k], c.q52[k], c.cnt2, c4[k]);
+                convert_quad_fast<YARD, COUNT>(w[4 * j + 2 * k], w[4 * j + 2 * k + 1], s4x2, tiny2, c.q43[k], c.q52[k], c.cnt2, c4[k], c5[k]);
             if (STORE) sts64(out_addr ^ ((j0 + j) << 3), make_uint2(c4[0], c4[1]));
+            if (STASH) sts64(stash_addr ^ ((j0 + j) << 4), make_uint2(c5[0], c5[1]));
         }
     }
 }
@@ -605,6 +617,13 @@ __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t 
     conv_init(c);
     convert_chunks<YARD, CAREFUL, STORE, 8, COUNT>(w, out_addr, 0, s4b, s5b, c);
     conv_finish<YARD, CAREFUL, COUNT>(c, s4b, s5b, e43, e52, nnz, nonfinite);
+}
+
+// A block selected E5M2: the thread's 64 stashed E5M2 codes replace its E4M3 codes in the staging buffer.
+__device__ __forceinline__ void copy_stash(uint32_t stash_addr, uint32_t out_addr)
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sts64(out_addr ^ (j << 3), lds64(stash_addr ^ (j << 4)));
 }
 
 // The E5M2 codes of a thread's 64 elements, for a block that selected E5M2 (such a block holds no
@@ -1072,7 +1091,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         // tile's count comes from the pre-pass and travels in thread 0's entry.
         constexpr bool kNeedKey = SCAN || THREE || EXTRA;
         constexpr bool kCount = SCAN || EXTRA;
-        // Two ways through a tile.  Streaming (keys from the pre-pass, no second use of the data): the scale is known
+        // Two ways through a tile.  Streaming (keys from the pre-pass, no BF16 output): the scale is known
         // before any element is read, so the thread converts its 64 elements in two halves straight from the stage,
         // 16 registers of data at a time, and hands the stage back after the second half's loads.  Otherwise the 64
         // elements are copied to registers first (the stage goes back at once) and serve the scan, the conversion
@@ -1080,8 +1099,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
 #ifdef MOR_NO_STREAM
         constexpr bool kStream = false;
 #else
-        constexpr bool kStream = !SCAN && !THREE && !EXTRA && KIND != KIND_COL128;
+        constexpr bool kStream = !SCAN && !EXTRA && KIND != KIND_COL128;
 #endif
+        // Three formats: the E5M2 codes of every element are kept in the thread's part of the stage until the block's
+        // decision is known (a copy then puts them in place); the stage goes back after that.
+        constexpr bool kStash = kStream && THREE && STORE;
         uint32_t w[32];
         if (kStream) {
         } else if (KIND == KIND_COL128) {
@@ -1227,8 +1249,8 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                             const uint4 v = lds128(a ^ ((4 * half + j) << 4));
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
-                        if (half == 1) stage_free_arrive(s);
-                        convert_chunks<YARD, true, STORE, 4, kCount>(wh, oa, 4 * half, s4b, s5b, acc);
+                        if (half == 1 && !kStash) stage_free_arrive(s);
+                        convert_chunks<YARD, true, STORE, 4, kCount, kStash>(wh, oa, 4 * half, s4b, s5b, acc, a);
                     }
                     conv_finish<YARD, true, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 } else {
@@ -1240,8 +1262,8 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                             const uint4 v = lds128(a ^ ((4 * half + j) << 4));
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
-                        if (half == 1) stage_free_arrive(s);
-                        convert_chunks<YARD, false, STORE, 4, kCount>(wh, oa, 4 * half, s4b, s5b, acc);
+                        if (half == 1 && !kStash) stage_free_arrive(s);
+                        convert_chunks<YARD, false, STORE, 4, kCount, kStash>(wh, oa, 4 * half, s4b, s5b, acc, a);
                     }
                     conv_finish<YARD, false, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 }
@@ -1260,7 +1282,13 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
                 const bool valid = row < (KIND == KIND_COL128 ? m.vcols : m.vrows);
                 sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
-                if (THREE && STORE && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
+                if (kStash) {
+                    if (sel == MOR_FMT_E5M2) copy_stash(in_base + s * kInBytes + in_off, oa);
+                    fence_async_smem();                  // the stage is written by the next TMA load: order the stash accesses before it
+                    stage_free_arrive(s);
+                } else if (THREE && STORE && sel == MOR_FMT_E5M2) {
+                    emit_e5m2_codes(w, oa, s5b);
+                }
                 if (h == 0) {
                     sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
                            make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
@@ -1297,7 +1325,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 }
             }
             if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
-        } else if (kStream) {
+        } else if (kStream && !(kStash && !kLineBlocks)) {
             stage_free_arrive(s);                       // given up: the arrival that the conversion would have made
         }
         out_full_arrive(b);
@@ -1312,8 +1340,13 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 }
                 if (!dead) sel = C.dec_sel[b][q];
                 if (THREE && STORE) {
-                    if (!dead && sel == MOR_FMT_E5M2) emit_e5m2_codes(w, oa, s5b);
+                    if (kStash) {
+                        if (!dead && sel == MOR_FMT_E5M2) copy_stash(in_base + s * kInBytes + in_off, oa);
+                    } else if (!dead && sel == MOR_FMT_E5M2) {
+                        emit_e5m2_codes(w, oa, s5b);
+                    }
                     fence_async_smem();
+                    if (kStash) stage_free_arrive(s);     // after the fence: the stash accesses come before the next TMA load
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&C.codes_full[b]);
                 }
