@@ -169,6 +169,9 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
     return true;
 }
 
+std::atomic<uint32_t> g_test_skip_tile{0xFFFFFFFFu};
+std::atomic<long long> g_test_wait_cycles{kDefaultWaitCycles};
+
 struct Layout {
     size_t amax_off, status_off, partial_off, keys_off, total;
 };
@@ -319,6 +322,8 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     std::vector<char> done(n, 0);
     MainParams mp;
     mp.device_status = reinterpret_cast<uint32_t*>(ws + l.status_off);
+    mp.test_skip_tile = g_test_skip_tile.load(std::memory_order_relaxed);
+    mp.wait_cycles = g_test_wait_cycles.load(std::memory_order_relaxed);
     for (int i = 0; i < n; ++i) {
         if (done[i]) continue;
         const MainVariant v = items[i].v;
@@ -602,6 +607,12 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
                                    cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(host_out->tensor_stats, o.tensor_stats, sizeof(mor_tensor_stats_t), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     return ok ? MOR_OK : MOR_ERR_CUDA;
+}
+
+void mor_test_skip_tile_load(uint32_t tile, long long wait_cycles)
+{
+    g_test_skip_tile.store(tile, std::memory_order_relaxed);
+    g_test_wait_cycles.store(tile == 0xFFFFFFFFu || wait_cycles <= 0 ? kDefaultWaitCycles : wait_cycles, std::memory_order_relaxed);
 }
 
 const char* mor_status_string(mor_status_t status)

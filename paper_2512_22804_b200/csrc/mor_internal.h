@@ -9,6 +9,11 @@
 
 #include "mor.h"
 
+// Test hook, exported but not part of mor.h: the next launches of the main kernel leave out the TMA load of tile
+// `tile` (numbered within each launch) and give up waiting after `wait_cycles` clock cycles; every such call then
+// reports MOR_ERR_TIMEOUT in mor_tensor_stats_t.status.  tile = 0xFFFFFFFF switches the hook off again.
+extern "C" MOR_API void mor_test_skip_tile_load(uint32_t tile, long long wait_cycles);
+
 namespace mor {
 
 // The main kernel works on tiles of 128 rows x 128 columns (32 KiB of BF16), whatever the
@@ -89,7 +94,11 @@ struct alignas(64) MainParams {
     BatchParams b;
     uint32_t total_tiles;
     uint32_t* device_status;
+    long long wait_cycles;        // a wait on an mbarrier gives up after this many clock cycles (kDefaultWaitCycles: about 0.2 s)
+    uint32_t test_skip_tile;      // test hook: the load of this tile of the launch is never started (0xFFFFFFFF: none)
 };
+
+constexpr long long kDefaultWaitCycles = 400000000ll;
 
 static_assert(sizeof(MainParams) <= 32764, "kernel parameters are limited to 32764 bytes");
 
