@@ -236,6 +236,13 @@ MOR_API mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_bl
                               mor_tensor_stats_t* tensor_stats, uint8_t* sel, uint8_t* scale_e8m0,
                               void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* mor_select_stats for `n` tensors in one call (tensors sharing a partition and recipe share kernel launches,
+ * 16 per launch).  host_outs[i].codes, .codes_ld, .bf16_fallback and .fake_quant are ignored; tensor_stats is
+ * required, block_stats / sel / scale_e8m0 / scale_f32 / error_histogram are optional as in mor_analyze_quantize.
+ * Same workspace as mor_analyze_quantize_batched for the same descriptors. */
+MOR_API mor_status_t mor_select_stats_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs, int n,
+                                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The first step of Algorithm 1 alone (the group's largest magnitude), with the whole tensor as the group:
  * writes max|x| over finite elements of tensor i to amax_out[i] (DEVICE, n floats), so
  * that later calls can pass it as group_amax. */

@@ -6,7 +6,7 @@ library has not been built, the first call raises.
 
 Low level (one-to-one with ``include/mor.h``):
     mor_workspace_bytes, mor_analyze_quantize, mor_analyze_quantize_batched,
-    mor_analyze_quantize_batched_ex, mor_select_stats, mor_group_amax, mor_host_staging_bytes, mor_analyze_quantize_host,
+    mor_analyze_quantize_batched_ex, mor_select_stats, mor_select_stats_batched, mor_group_amax, mor_host_staging_bytes, mor_analyze_quantize_host,
     mor_status_string, mor_version
 
 Helpers that allocate outputs with torch and fill the descriptors:
@@ -104,6 +104,8 @@ def load():
         L.mor_analyze_quantize_batched_ex.restype = C.c_int
         L.mor_analyze_quantize_batched_ex.argtypes = [pd, po, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p,
                                                       C.POINTER(mor_stage_events_t)]
+        L.mor_select_stats_batched.restype = C.c_int
+        L.mor_select_stats_batched.argtypes = [pd, po, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]
         L.mor_select_stats.restype = C.c_int
         L.mor_select_stats.argtypes = [pd, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.mor_group_amax.restype = C.c_int
@@ -123,7 +125,7 @@ def load():
 
 
 EXPORTS = ["mor_workspace_bytes", "mor_analyze_quantize", "mor_analyze_quantize_batched",
-           "mor_analyze_quantize_batched_ex", "mor_select_stats",
+           "mor_analyze_quantize_batched_ex", "mor_select_stats", "mor_select_stats_batched",
            "mor_group_amax", "mor_host_staging_bytes", "mor_analyze_quantize_host",
            "mor_analyze_quantize_static", "mor_status_string", "mor_version"]
 
@@ -173,6 +175,12 @@ def mor_select_stats(desc: mor_tensor_desc_t, block_stats_ptr: int, tensor_stats
                      scale_ptr: int, workspace_ptr: int, workspace_bytes: int, stream_ptr: int = 0) -> int:
     return load().mor_select_stats(C.byref(desc), block_stats_ptr, tensor_stats_ptr, sel_ptr, scale_ptr,
                                    workspace_ptr, workspace_bytes, stream_ptr)
+
+
+def mor_select_stats_batched(descs, outs, workspace_ptr: int, workspace_bytes: int, stream_ptr: int = 0) -> int:
+    darr, n = _desc_array(descs)
+    oarr = outs if isinstance(outs, C.Array) else (mor_outputs_t * len(outs))(*outs)
+    return load().mor_select_stats_batched(darr, oarr, n, workspace_ptr, workspace_bytes, stream_ptr)
 
 
 def mor_group_amax(descs, amax_out_ptr: int, workspace_ptr: int, workspace_bytes: int, stream_ptr: int = 0) -> int:
@@ -375,7 +383,7 @@ class BatchPlan:
     step is a single call of mor_analyze_quantize_batched."""
 
     def __init__(self, xs: Sequence, recipes: Sequence[Recipe], *, group_amax=None, block_stats=False,
-                 fallback=False, fake_quant=False, error_histograms=None):
+                 fallback=False, fake_quant=False, error_histograms=None, stats_only=False):
         """`fallback` and `fake_quant` are one flag for all tensors or one flag per tensor; `error_histograms`
         is one tensor of MOR_ERROR_BINS 32-bit counters per tensor (or None)."""
         assert len(xs) == len(recipes) and len(xs) > 0
@@ -389,7 +397,7 @@ class BatchPlan:
             ga = None if group_amax is None else group_amax[i:i + 1]
             d = desc_for(x, r, None, ga)
             descs.append(d)
-            self.outs.append(alloc_outputs(d.rows, d.cols, r, x.device, block_stats=block_stats,
+            self.outs.append(alloc_outputs(d.rows, d.cols, r, x.device, block_stats=block_stats, codes=not stats_only,
                                            fallback_like=x if fallback[i] else None,
                                            fake_quant_like=x if fake_quant[i] else None,
                                            error_histogram=None if error_histograms is None else error_histograms[i]))
@@ -398,8 +406,14 @@ class BatchPlan:
         self.n = len(descs)
         self.ws = _workspace(mor_workspace_bytes(self.descs), xs[0].device)
         self._fn = load().mor_analyze_quantize_batched_ex
+        self.stats_only = stats_only          # decisions and statistics only (mor_select_stats_batched): no codes
 
     def run(self, stream=None, events: Optional[mor_stage_events_t] = None) -> None:
+        if self.stats_only:
+            st = load().mor_select_stats_batched(self.descs, self.couts, self.n, self.ws.data_ptr(), self.ws.numel(), _stream_ptr(stream))
+            if st != MOR_OK:
+                raise MorError(st, "mor_select_stats_batched")
+            return
         st = self._fn(self.descs, self.couts, self.n, self.ws.data_ptr(), self.ws.numel(), _stream_ptr(stream),
                       None if events is None else C.byref(events))
         if st != MOR_OK:

@@ -468,6 +468,21 @@ mor_status_t mor_select_stats(const mor_tensor_desc_t* host_desc, mor_block_stat
     return run(items, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
+mor_status_t mor_select_stats_batched(const mor_tensor_desc_t* host_descs, const mor_outputs_t* host_outs, int n,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream)
+{
+    if (host_descs == nullptr || host_outs == nullptr || n < 0) return MOR_ERR_INVALID_ARG;
+    if (n == 0) return MOR_OK;
+    std::vector<Item> items((size_t)n);
+    for (int i = 0; i < n; ++i) {
+        mor_outputs_t o = host_outs[i];
+        o.codes = nullptr; o.codes_ld = 0; o.bf16_fallback = nullptr; o.fake_quant = nullptr;
+        mor_status_t st = make_item(&host_descs[i], o, false, i, items[i]);
+        if (st != MOR_OK) return st;
+    }
+    return run(items, workspace, workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
 mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* amax_out,
                             void* workspace, size_t workspace_bytes, void* cuda_stream)
 {

@@ -380,6 +380,29 @@ def test_select_stats_matches_analyze_quantize():
         parity.compare(g, r, s, ref)
 
 
+@pytest.mark.parametrize("stats", [False, True])
+def test_select_stats_batched_matches_the_oracle(stats):
+    """Decisions and statistics for several tensors of mixed partitions in one call, without codes; with and without
+    block statistics (without: the plain instantiation, whose non-zero counts come from the pre-pass); some with
+    the group amax supplied (single read, the kernel scans)."""
+    import torch
+
+    cases = [(wl.gradient_like(300, 1000, seed=54), recipe((1, 128), THREE)),
+             (wl.weight_like(256, 384, seed=55), recipe((128, 128), TWO)),
+             (wl.activation_like(200, 520, seed=56), recipe((64, 64), THREE)),
+             (wl.gaussian_outlier_rows(256, 256, seed=57), recipe((0, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL)),
+             (wl.weight_like(130, 200, seed=58), recipe((128, 1), TWO)),
+             (wl.activation_like(256, 256, seed=59), recipe((1, 128), TWO, scale_mode=mb.MOR_SCALE_E8M0))]
+    xs = [parity.to_device(b) for b, _ in cases]
+    plan = mb.BatchPlan(xs, [r for _, r in cases], block_stats=stats, stats_only=True)
+    plan.run()
+    torch.cuda.synchronize()
+    for (bits, r), o in zip(cases, plan.outs):
+        assert o.codes is None
+        ref = orc.run(bits, parity.oracle_block(r.block, bits.shape[1]), list(r.formats), r.criterion, r.threshold, r.scale_mode, r.flags)
+        parity.compare(bits, r, o, ref)
+
+
 def test_bf16_fallback_copies_only_rejected_blocks():
     import torch
 
