@@ -107,7 +107,6 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
         if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
         // sub-column blocks leave their codes transposed: [cols, codes_ld] with the rows along the contiguous dimension
         if (o.codes_ld < (int64_t)round_up((size_t)(s.kind == KIND_COL128 ? d.rows : d.cols), 16)) return MOR_ERR_INVALID_ARG;
-        if (s.kind == KIND_COL128 && (o.bf16_fallback != nullptr || o.fake_quant != nullptr)) return MOR_ERR_UNSUPPORTED;
         if (o.codes_ld % 16 != 0 || !aligned(o.codes, 16)) return MOR_ERR_ALIGNMENT;
         if (d.scale_mode == MOR_SCALE_FP32_AMAX && o.scale_f32 == nullptr && s.n_blocks) return MOR_ERR_INVALID_ARG;
         if (o.fake_quant && !aligned(o.fake_quant, 16)) return MOR_ERR_ALIGNMENT;

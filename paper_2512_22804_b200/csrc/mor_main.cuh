@@ -415,6 +415,35 @@ __device__ __forceinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
 
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
 
+// The same two scans for a thread that has not copied its elements to registers: the eight 16-byte chunks are read
+// from the stage at a ^ (j << 4) (the conversion reads them a second time afterwards).
+__device__ __forceinline__ uint32_t scan_stage(uint32_t a)
+{
+    uint32_t mx[2] = {0u, 0u}, mn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint4 v = lds128(a ^ (j << 4));
+        const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
+        mx[0] = __vimax3_u16x2(mx[0], a0, a1);
+        mx[1] = __vimax3_u16x2(mx[1], a2, a3);
+        mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
+        mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
+        mn[2] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn[2]);
+        mn[3] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn[3]);
+    }
+    const uint32_t mxx = __vimax3_u16x2(mx[0], mx[1], mx[1]);
+    const uint32_t mnn = __vimin3_u16x2(__vimin3_u16x2(mn[0], mn[1], mn[2]), mn[3], mn[3]);
+    const uint32_t amax = max(mxx & 0xFFFFu, mxx >> 16), minm1 = min(mnn & 0xFFFFu, mnn >> 16);
+    return (amax << 16) | (0xFFFFu - minm1);
+}
+__device__ __noinline__ uint32_t scan_stage_finite(uint32_t a)
+{
+    uint32_t m = 0u, n = 0xFFFFu;
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) scan_finite4(lds128(a ^ (j << 4)), m, n);
+    return (m << 16) | (0xFFFFu - n);
+}
+
 // Raise the tensor amax slot to the BF16 magnitude `bits` (non-negative binary32 patterns order like the
 // values).  Atomics on one address are served one at a time, so the slot is read first: after the first
 // tiles of a tensor almost every call ends there.
@@ -1044,6 +1073,47 @@ __device__ __forceinline__ void write_fake_quant(const TensorRec& R, const uint3
     }
 }
 
+// Sub-column blocks: 64 elements down a column of the row-major tile, two rows per word, chunk by chunk (a chunk
+// is 8 rows): chunk j of the registers holds rows 8 (j ^ swz) .. + 7 (the order in which the code chunks are stored),
+// so one address is formed per chunk and the eight 16-bit loads of a chunk use constant offsets from it.
+__device__ __forceinline__ void load_column(uint32_t a, int swz, uint32_t (&w)[32])
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t cb = a + ((uint32_t)(j ^ swz) << 11);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            uint32_t lo, hi;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(cb + (uint32_t)(2 * k * 256)));
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(cb + (uint32_t)((2 * k + 1) * 256)));
+            w[4 * j + k] = __byte_perm(lo, hi, 0x5410);
+        }
+    }
+}
+
+// The BF16 outputs of a thread that holds a column piece (sub-column blocks): element by element down the column
+// (2-byte stores; the 16 columns of a warp make 32-byte runs).  `fq`: fake quantisation with format `fmt` and scale
+// `s` (BF16-selected blocks and NaN/inf elements are copied); otherwise the plain copy of a rejected block.
+__device__ __noinline__ void write_column(uint16_t* dst, long long ld, const TileMeta& m, int col, int h, int swz,
+                                          const uint32_t (&w)[32], bool fq, uint32_t fmt, float s)
+{
+    if (col >= m.vcols) return;
+    uint16_t* base = dst + (long long)m.row0 * ld + m.col0 + col;
+#pragma unroll 1
+    for (int j = 0; j < 8; ++j) {
+        uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+        for (int k = 1; k < 8; ++k)
+            if (j == k) v = make_uint4(w[4 * k], w[4 * k + 1], w[4 * k + 2], w[4 * k + 3]);
+        uint32_t o[4] = {v.x, v.y, v.z, v.w};
+        if (fq && fmt != MOR_FMT_BF16) fake_quant_chunk(v, fmt, s, o);
+        const int r0 = 64 * h + 8 * (j ^ swz);             // first of the chunk's 8 rows within the tile
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (r0 + i < m.vrows) base[(long long)(r0 + i) * ld] = (uint16_t)(o[i >> 1] >> (16 * (i & 1)));
+    }
+}
+
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN, bool EXTRA>
 __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
 {
@@ -1092,15 +1162,15 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         // tile's count comes from the pre-pass and travels in thread 0's entry.
         constexpr bool kNeedKey = SCAN || THREE || EXTRA;
         constexpr bool kCount = SCAN || EXTRA;
-        // Two ways through a tile.  Streaming (keys from the pre-pass, no BF16 output): the scale is known
-        // before any element is read, so the thread converts its 64 elements in two halves straight from the stage,
-        // 16 registers of data at a time, and hands the stage back after the second half's loads.  Otherwise the 64
-        // elements are copied to registers first (the stage goes back at once) and serve the scan, the conversion
-        // and whatever follows the block's decision (E5M2 codes, BF16 copy, fake quantisation).
+        // Two ways through a tile.  Streaming (no BF16 output): the thread converts its 64 elements in two halves
+        // straight from the stage, 16 registers of data at a time, and hands the stage back after the second half's
+        // loads; where no pre-pass ran it first scans them, also from the stage.  Otherwise the 64 elements are
+        // copied to registers first (the stage goes back at once) and serve the scan, the conversion and whatever
+        // follows the block's decision (BF16 copy, fake quantisation).
 #ifdef MOR_NO_STREAM
         constexpr bool kStream = false;
 #else
-        constexpr bool kStream = !SCAN && !EXTRA && KIND != KIND_COL128;
+        constexpr bool kStream = !EXTRA && KIND != KIND_COL128;
 #endif
         // Three formats: the E5M2 codes of every element are kept in the thread's part of the stage until the block's
         // decision is known (a copy then puts them in place); the stage goes back after that.
@@ -1111,13 +1181,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             // sub-column blocks: this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows
             // per word, so that everything after this point works on the block as on a row piece
             const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                uint32_t lo, hi;
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
-                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
-                w[i] = lo | (hi << 16);
-            }
+            load_column(a, swz, w);
         } else {
             const uint32_t a = in_base + s * kInBytes + in_off;
 #pragma unroll
@@ -1155,11 +1219,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         if (!SCAN) {
             key &= 0x7FFFFFFFu;                         // (the flag for NaN/inf is part of the prepared word)
         } else if (kLineBlocks) {
-            key = scan_words(w);
+            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
             if (nonfin) {
-                key = scan_words_finite(w);
+                key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
                 key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
@@ -1169,7 +1233,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
             }
         } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
-            key = scan_words(w);
+            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
             uint32_t tile_amax = 0u;
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
@@ -1198,14 +1262,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 if (dead) { key = 0u; nonfin = false; }
                 tile_amax = any >> 16;
                 if (pass == 1 || !nonfin) break;
-                key = scan_words_finite(w);
+                key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here
             raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead && !(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot);
         } else {
-            key = scan_words(w);
+            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
-            if (nonfin) key = scan_words_finite(w);
+            if (nonfin) key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
         }
         uint32_t amax_bits = key >> 16;
         const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
@@ -1308,8 +1372,16 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                         }
                     }
                 }
-                if (EXTRA && has_fallback && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
-                if (EXTRA && has_fq) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
+                if (KIND == KIND_COL128) {
+                    if (EXTRA && has_fallback && sel == MOR_FMT_BF16) write_column(R.fallback, R.ld, m, row, h, swz, w, false, sel, 0.0f);
+                    if (EXTRA && has_fq) {
+                        const uint32_t f = fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel;
+                        write_column(R.fake_quant, R.ld, m, row, h, swz, w, true, f, __uint_as_float(f == MOR_FMT_E5M2 ? s5b : s4b));
+                    }
+                } else {
+                    if (EXTRA && has_fallback && sel == MOR_FMT_BF16) write_fallback(R, w, m, row, h, swz);
+                    if (EXTRA && has_fq) write_fake_quant(R, w, m, row, h, swz, fq_e4m3 ? (uint32_t)MOR_FMT_E4M3 : sel, s4b, s5b);
+                }
             } else {
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
@@ -1415,13 +1487,7 @@ __device__ __forceinline__ void compute_warps_dual(const MainParams& p, Control&
             } else {
                 // this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows per word
                 const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    uint32_t lo, hi;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2) * 256)));
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)(((i ^ (swz << 2)) * 2 + 1) * 256)));
-                    w[i] = lo | (hi << 16);
-                }
+                load_column(a, swz, w);
                 stage_free_arrive(s);                       // both copies of the stage are in registers
             }
 

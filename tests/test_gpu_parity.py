@@ -155,7 +155,7 @@ def test_a_pair_with_different_recipes_is_served_separately():
 
 # ------------------------------------------------------------ fake quantisation (Section 4)
 
-@pytest.mark.parametrize("block", KINDS + [(1, 0)])
+@pytest.mark.parametrize("block", KINDS + [(1, 0), (128, 1)])
 def test_fake_quant_output(block):
     g = np.concatenate([wl.gradient_like(150, 1000, seed=58), wl.weight_like(170, 1000, seed=59)])
     g[7, 13] = 0x7FC0
@@ -409,7 +409,7 @@ def test_bf16_fallback_copies_only_rejected_blocks():
     g = np.concatenate([wl.gradient_like(150, 1000, seed=54), wl.weight_like(150, 1000, seed=57)])
     host = np.zeros((300, 1008), dtype=np.uint16); host[:, :1000] = g
     x = parity.to_device(host)
-    for block in [(1, 128), (128, 128), (64, 64)]:
+    for block in [(1, 128), (128, 128), (64, 64), (128, 1)]:
         r = recipe(block, THREE)
         out = mb.analyze_quantize(x, r, cols=1000, fallback=True)
         torch.cuda.synchronize()
