@@ -61,7 +61,8 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
     s.key_words = (uint64_t)s.n_tiles * ((s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL) ? (uint64_t)kRowKeyStride : (uint64_t)kTileKeyStride);
-    if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows;      // + one key per row
+    if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows      // + one key per row
+                                             + (uint64_t)s.n_tiles * kTileRows * 4; // + per tile and row the partial sums of a per-row decision
     return MOR_OK;
 }
 
@@ -86,9 +87,10 @@ mor_status_t check_desc(const mor_tensor_desc_t& d, Shape& s)
         return MOR_ERR_INVALID_ARG;
     }
     if (d.criterion < MOR_CRIT_TENSOR_MEAN_REL || d.criterion > MOR_CRIT_BLOCK_MEAN_REL) return MOR_ERR_INVALID_ARG;
-    // per-channel blocks span many tiles: this build gives them the tensor-level decision only (the recipe the
-    // paper evaluates them with, Section 4.1)
-    if (s.kind == KIND_CHANNEL && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || d.n_formats != 2)) return MOR_ERR_UNSUPPORTED;
+    // per-channel blocks span many tiles: their decision (tensor-level as in Section 4.1, or per row by Eq. 3 or by
+    // Eq. 1-2 on the row) is taken after the main kernel, when the codes are written; a row that chose E5M2 would need
+    // its codes rewritten, so three formats are not offered here
+    if (s.kind == KIND_CHANNEL && d.n_formats != 2) return MOR_ERR_UNSUPPORTED;
     if (d.scale_mode < MOR_SCALE_GAM || d.scale_mode > MOR_SCALE_FP32_AMAX) return MOR_ERR_INVALID_ARG;
     if (!(d.threshold >= 0.0f) || std::isinf(d.threshold)) return MOR_ERR_INVALID_ARG;
     if (d.flags & ~(uint32_t)(MOR_FLAG_STRICT_TIES | MOR_FLAG_RANGE_MIN_INCLUDES_ZERO)) return MOR_ERR_INVALID_ARG;
@@ -101,7 +103,9 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
     if (o.tensor_stats == nullptr) return MOR_ERR_INVALID_ARG;
     if (o.error_histogram && !aligned(o.error_histogram, 4)) return MOR_ERR_ALIGNMENT;
     if (!aligned(o.tensor_stats, 8) || !aligned(o.block_stats, 4) || !aligned(o.scale_f32, 4)) return MOR_ERR_ALIGNMENT;
-    if (s.kind == KIND_CHANNEL && o.block_stats != nullptr) return MOR_ERR_UNSUPPORTED;   // would need sums across tiles
+    // a per-row decision of the per-channel partition is known only after the main kernel: no BF16 outputs that depend on it
+    if (s.kind == KIND_CHANNEL && d.criterion != MOR_CRIT_TENSOR_MEAN_REL && (o.bf16_fallback != nullptr || o.fake_quant != nullptr))
+        return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     if (store) {
         if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
@@ -218,6 +222,8 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
     r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
     r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kRowKeyStride : nullptr;
+    const bool per_row = it.s.kind == KIND_CHANNEL && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || it.o.block_stats != nullptr);
+    r.row_part = per_row && r.row_keys ? reinterpret_cast<float4*>(r.row_keys + (size_t)it.s.nbr * kTileRows) : nullptr;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
@@ -361,7 +367,12 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         if (!flush()) return MOR_ERR_CUDA;
     }
     if (ev && !record(ev->main_end)) return MOR_ERR_CUDA;
-    for (const Chunk& c : chunks) {
+    for (Chunk& c : chunks) {
+        if (c.kind == KIND_CHANNEL) {
+            bool per_row = false;
+            for (int k = 0; k < c.bp.n; ++k) per_row = per_row || c.bp.t[k].row_part != nullptr;
+            if (per_row && launch_row_decide(c.bp, partials, stream) != cudaSuccess) return MOR_ERR_CUDA;
+        }
         if (c.kind != KIND_DUAL) {
             if (launch_finalise(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
             continue;
@@ -393,6 +404,7 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
     it.v.store = store;
     it.v.extra = (store && (o.bf16_fallback != nullptr || o.fake_quant != nullptr)) || o.block_stats != nullptr ||
+                 (it.s.kind == KIND_CHANNEL && d->criterion != MOR_CRIT_TENSOR_MEAN_REL) ||
                  d->criterion == MOR_CRIT_BLOCK_MEAN_REL || (d->flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) != 0;
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data

@@ -60,6 +60,9 @@ struct TensorRec {
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
     uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows
+    float4* row_part;             // KIND_CHANNEL with a per-row decision or per-row statistics: per tile and row of the tile
+                                  // {sum of E4M3 terms, sum of E5M2 terms, bits(non-zeros | non-finites << 16), unused},
+                                  // written by the main kernel, added up along each row by mor_row_decide_kernel
     uint32_t key_stride;          // words per tile in `keys`: kRowKeyStride (one key per row piece, then the tile's
                                   // non-zero count) or kTileKeyStride (one key per tile, or one per 64x64 quadrant in the
                                   // order top-left, top-right, bottom-left, bottom-right; word 4: the tile's non-zero count)
@@ -137,6 +140,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);
+cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s);
 

@@ -279,6 +279,63 @@ mor_row_keys_kernel(const __grid_constant__ BatchParams p)
     R.row_keys[(size_t)blockIdx.x * kTileRows + threadIdx.x] = k | flag;
 }
 
+// Per-channel partition with a per-row decision (Algorithm 2 with one block per row) or per-row statistics: the
+// row's sums are the sums of its tiles' parts, added in tile order in double.  One CTA of 128 threads per (tile row,
+// tensor); writes sel, block statistics and, into the partial of the tile row's first tile, the counts of rows per
+// format, which the finalise kernel adds up.
+__global__ void __launch_bounds__(kTileRows)
+mor_row_decide_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ partials)
+{
+    __shared__ uint32_t s_n4[kTileRows / 32], s_nb[kTileRows / 32];
+    pdl_wait();                                          // the main kernel's row parts are complete
+    const TensorRec& R = p.t[blockIdx.y];
+    if (R.kind != KIND_CHANNEL || R.row_part == nullptr || blockIdx.x >= R.nbr) return;
+    const long long row = (long long)blockIdx.x * kTileRows + threadIdx.x;
+    const bool valid = row < R.rows;
+    double s43 = 0.0, s52 = 0.0;
+    uint32_t nnz = 0u, nonf = 0u;
+    if (valid) {
+        const float4* src = R.row_part + ((size_t)blockIdx.x * R.nbc) * kTileRows + threadIdx.x;
+        for (uint32_t j = 0; j < R.nbc; ++j, src += kTileRows) {
+            const float4 v = *src;
+            const uint32_t nz = __float_as_uint(v.z);
+            s43 += (double)v.x; s52 += (double)v.y; nnz += nz & 0xFFFFu; nonf += nz >> 16;
+        }
+    }
+    uint32_t sel = MOR_FMT_E4M3;
+    if (valid) {
+        if (nonf) sel = MOR_FMT_BF16;
+        else if (R.criterion == MOR_CRIT_BLOCK_VS_E5M2) {
+            const bool ok = (R.flags & MOR_FLAG_STRICT_TIES) ? (s43 < s52) : (s43 <= s52);
+            sel = ok ? MOR_FMT_E4M3 : MOR_FMT_BF16;
+        } else if (R.criterion == MOR_CRIT_BLOCK_MEAN_REL) {
+            const double err = nnz ? s43 / (double)nnz : 0.0;
+            sel = err < (double)R.threshold ? MOR_FMT_E4M3 : MOR_FMT_BF16;
+        }
+        if (R.criterion != MOR_CRIT_TENSOR_MEAN_REL && R.sel) R.sel[row] = (uint8_t)sel;   // (tensor-level: filled by the finalise kernel)
+        if (R.block_stats) {
+            const uint32_t key = R.row_keys[row] & 0x7FFFFFFFu;
+            mor_block_stats_t bs;
+            bs.amax = __uint_as_float((key >> 16) << 16);
+            bs.min_abs_nz = __uint_as_float(0x7F800000u);           // kept for three formats only, which this partition does not take
+            bs.nnz = nnz; bs.n_nonfinite = nonf;
+            bs.sum_rel_e4m3 = (float)s43; bs.sum_rel_e5m2 = (float)s52;
+            R.block_stats[row] = bs;
+        }
+    }
+    if (R.criterion != MOR_CRIT_TENSOR_MEAN_REL) {
+        const uint32_t b4 = __ballot_sync(0xFFFFFFFFu, valid && sel == MOR_FMT_E4M3), bb = __ballot_sync(0xFFFFFFFFu, valid && sel == MOR_FMT_BF16);
+        if ((threadIdx.x & 31) == 0) { s_n4[threadIdx.x >> 5] = __popc(b4); s_nb[threadIdx.x >> 5] = __popc(bb); }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            Partial& P = partials[R.tile_begin + (size_t)blockIdx.x * R.nbc];
+            P.n_e4m3 = s_n4[0] + s_n4[1] + s_n4[2] + s_n4[3];
+            P.n_e5m2 = 0u;
+            P.n_bf16 = s_nb[0] + s_nb[1] + s_nb[2] + s_nb[3];
+        }
+    }
+}
+
 // ----------------------------------------------------------------------- finalise ----
 
 // One CTA per (tensor, slice).  Every slice repeats the reduction over the tensor's tile
@@ -403,6 +460,15 @@ cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s)
     if (nbr == 0) return cudaSuccess;
     mor_row_keys_kernel<<<dim3(nbr, (unsigned)p.n), kTileRows, 0, s>>>(p);
     return cudaGetLastError();
+}
+
+cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, cudaStream_t s)
+{
+    uint32_t nbr = 0;
+    for (int i = 0; i < p.n; ++i)
+        if (p.t[i].kind == KIND_CHANNEL && p.t[i].row_part != nullptr && p.t[i].nbr > nbr) nbr = p.t[i].nbr;
+    if (nbr == 0) return cudaSuccess;
+    return launch_dependent(mor_row_decide_kernel, dim3(nbr, (unsigned)p.n), dim3(kTileRows), 0, s, p, partials);
 }
 
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s)

@@ -1387,6 +1387,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
                 if (EXTRA && (KIND == KIND_TENSOR || KIND == KIND_CHANNEL) && has_fq)
                     write_fake_quant(R, w, m, row, h, swz, (uint32_t)MOR_FMT_E4M3, s4b, s5b);
+                if (EXTRA && KIND == KIND_CHANNEL && R.row_part != nullptr) {
+                    // per-row decision or statistics: this tile's part of the row's sums, for mor_row_decide_kernel
+                    const float r43 = e43 + __shfl_xor_sync(0xFFFFFFFFu, e43, 1), r52 = e52 + __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
+                    uint32_t nz = nnz | (nonf << 16);
+                    nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
+                    if (h == 0 && row < m.vrows)
+                        R.row_part[(size_t)m.local * kTileRows + row] = make_float4(r43, r52, __uint_as_float(nz), 0.0f);
+                }
                 if (KIND == KIND_CHANNEL && h == 0 && m.blk_base != 0xFFFFFFFFu && row < m.vrows) {
                     // per-channel: the row's scale, written by the tile that holds the row's first columns
                     const uint32_t blk = m.blk_base + (uint32_t)row;

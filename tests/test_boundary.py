@@ -80,7 +80,7 @@ def out_struct(codes=0x2000, codes_ld=256, ts=0x3000):
     (desc(formats=(0, 1)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
     (desc(formats=(0, 1, 2), crit=mb.MOR_CRIT_TENSOR_MEAN_REL), out_struct(), mb.MOR_ERR_UNSUPPORTED),
     (desc(formats=(0, 1, 2), block=(0, 0)), out_struct(), mb.MOR_ERR_UNSUPPORTED),
-    (desc(block=(1, 0)), out_struct(), mb.MOR_ERR_UNSUPPORTED),               # per channel: tensor-level criterion only
+    (desc(block=(1, 0), formats=(0, 1, 2)), out_struct(), mb.MOR_ERR_UNSUPPORTED),   # per channel: two formats only
     (desc(rows=512, block=(128, 1)), out_struct(), mb.MOR_ERR_INVALID_ARG),  # transposed codes: codes_ld covers the rows
     (desc(rows=-1), out_struct(), mb.MOR_ERR_INVALID_ARG),
     (desc(ld=128), out_struct(), mb.MOR_ERR_INVALID_ARG),                  # ld < cols

@@ -205,17 +205,46 @@ def test_per_channel_partition_with_the_tensor_level_decision(shape, mode):
                                group_amax_supplied=True)
 
 
-def test_per_channel_partition_supports_the_tensor_level_recipe_only():
+@pytest.mark.parametrize("shape", [(256, 512), (130, 1000), (300, 72), (5, 2049), (257, 1160)])
+@pytest.mark.parametrize("crit", [mb.MOR_CRIT_BLOCK_VS_E5M2, mb.MOR_CRIT_BLOCK_MEAN_REL])
+def test_per_channel_partition_with_a_decision_per_row(shape, crit):
+    """One block per row, decided row by row (Eq. 3 against E5M2, or Eq. 1-2 on the row): the row's sums are added
+    up over its tiles after the main kernel.  Rows that keep E4M3 next to rows that fall back; an all-zero row, a
+    row with a NaN; with and without per-row statistics; every scale mode; strict ties."""
+    rows, cols = shape
+    x = wl.activation_like(rows, cols, n_outlier_cols=min(4, cols), seed=148)
+    x[rows // 2, :] = 0                                            # an all-zero channel
+    wide = wl.gradient_like(rows, cols, seed=149)
+    x[::3, :] = wide[::3, :]                                       # every third row spans many binades
+    if rows > 3:
+        x[3, cols // 2] = 0x7FC0
+    ld = (cols + 7) // 8 * 8 + 8
+    for mode in (mb.MOR_SCALE_GAM, mb.MOR_SCALE_E8M0, mb.MOR_SCALE_FP32_AMAX):
+        for flags in (0, mb.MOR_FLAG_STRICT_TIES):
+            r = recipe((1, 0), TWO, crit, threshold=0.03, scale_mode=mode, flags=flags)
+            rep = parity.run_and_compare(x, r, pad_to=ld, block_stats=True)
+            assert rep.n_blocks == rows and rep.n_exempt <= 1
+    ref = orc.run(x, (1, cols), list(TWO), crit, 0.03)
+    if rows >= 100:
+        assert ref.tensor["n_e4m3"] > 0 and ref.tensor["n_bf16"] > 0
+    parity.run_and_compare(x, recipe((1, 0), TWO, crit, threshold=0.03), pad_to=ld, block_stats=False, group_amax_supplied=True)
+    # per-row statistics also with the tensor-level decision
+    parity.run_and_compare(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), pad_to=ld, block_stats=True)
+
+
+def test_per_channel_partition_refuses_what_it_cannot_give():
+    """Three formats (a row that chose E5M2 would need its codes rewritten after the last tile) and BF16 outputs that
+    depend on a per-row decision are refused."""
     import torch
 
     x = torch.zeros((128, 256), dtype=torch.bfloat16, device="cuda")
-    for bad in (recipe((1, 0), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2), recipe((1, 0), THREE, mb.MOR_CRIT_BLOCK_VS_E5M2)):
-        with pytest.raises(mb.MorError) as e:
-            mb.analyze_quantize(x, bad)
-        assert e.value.status == mb.MOR_ERR_UNSUPPORTED
     with pytest.raises(mb.MorError) as e:
-        mb.analyze_quantize(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), block_stats=True)
+        mb.analyze_quantize(x, recipe((1, 0), THREE, mb.MOR_CRIT_BLOCK_VS_E5M2))
     assert e.value.status == mb.MOR_ERR_UNSUPPORTED
+    for kw in (dict(fallback=True), dict(fake_quant=True)):
+        with pytest.raises(mb.MorError) as e:
+            mb.analyze_quantize(x, recipe((1, 0), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2), **kw)
+        assert e.value.status == mb.MOR_ERR_UNSUPPORTED
 
 
 # ------------------------------------------------------------ ragged, padded, tiny and empty shapes
