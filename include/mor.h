@@ -96,14 +96,16 @@ typedef struct mor_tensor_desc {
     int64_t ld;             /* elements between row starts; >= cols; multiple of 8           */
     int32_t block_rows;     /* partition: (0,0) whole tensor, (1,128) sub-channel rows,      */
     int32_t block_cols;     /*            (128,128) or (64,64) 2-D blocks (Section 4.1.2 runs
-                                           the smaller size as an ablation), (1,0) per channel:
-                                           one block per row (Section 3; the paper's most
-                                           FP8-efficient partition), with the tensor-level
-                                           criterion only; (128,1) sub-column blocks, for the
-                                           operand whose dot-product dimension runs down the
-                                           rows (its codes come out transposed, see codes).
-                                           Edge blocks may overhang: missing elements take part
-                                           in nothing                                        */
+                                           the smaller size as an ablation); per channel (Section 3;
+                                           the paper's most FP8-efficient partition): (1,0) one
+                                           block per row, (0,1) one block per column, whichever is
+                                           the operand's dot-product dimension, two formats only,
+                                           decided for the tensor (Eq. 2) or per channel (Eq. 3, or
+                                           Eq. 1-2 on the channel); (128,1) sub-column blocks.  The
+                                           column partitions (128,1) and (0,1) serve the operand whose
+                                           dot-product dimension runs down the rows: their codes come
+                                           out transposed, see codes.  Edge blocks may overhang:
+                                           missing elements take part in nothing                  */
     int32_t n_formats;      /* 2 or 3                                                        */
     int32_t formats[3];     /* {E4M3,BF16} or {E4M3,E5M2,BF16}, in this order                */
     int32_t criterion;      /* mor_criterion_t; three formats need BLOCK_VS_E5M2             */
@@ -152,7 +154,7 @@ typedef struct mor_tensor_stats {
  * mor_tensor_stats_t.group_mantissa).  All DEVICE pointers.  Block arrays are row-major
  * over the block grid [ceil(rows/block_rows), ceil(cols/block_cols)]. */
 typedef struct mor_outputs {
-    uint8_t* codes;         /* [rows, codes_ld] FP8 codes, 16-byte aligned ((128,1) blocks:
+    uint8_t* codes;         /* [rows, codes_ld] FP8 codes, 16-byte aligned ((128,1) and (0,1) blocks:
                                transposed, [cols, codes_ld] with codes_ld >= roundup(rows,16),
                                so that every block is contiguous).  E4M3 codes
                                everywhere except in blocks that selected E5M2; blocks that
@@ -167,12 +169,11 @@ typedef struct mor_outputs {
     uint8_t* sel;           /* [n_blocks] mor_format_t chosen for the block                  */
     float*   scale_f32;     /* [n_blocks] optional (required for MOR_SCALE_FP32_AMAX): the
                                selected format's scale as a binary32                         */
-    void*    bf16_fallback; /* optional (not with (128,1) blocks, nor is fake_quant),
-                               BF16 [rows, ld] like x: receives a copy of every
+    void*    bf16_fallback; /* optional, BF16 [rows, ld] like x: receives a copy of every
                                block that selected BF16 (other blocks are left untouched).
                                NULL = the fallback is the input itself.  Per-block criteria
                                only                                                          */
-    mor_block_stats_t*  block_stats;  /* [n_blocks] optional; not with the (1,0) partition   */
+    mor_block_stats_t*  block_stats;  /* [n_blocks] optional                                 */
     mor_tensor_stats_t* tensor_stats; /* required                                            */
     void*    fake_quant;    /* optional, BF16 [rows, ld] like x: the tensor after "quantise,
                                dequantise, de-scale" (Section 4, the form the paper trains with).
@@ -180,8 +181,10 @@ typedef struct mor_outputs {
                                by the block's scale (one binary32 division), rounded to BF16;
                                blocks that stay in BF16 and NaN/inf elements are copied.  Where the
                                decision is taken for the whole tensor (tensor-level criterion,
-                               (0,0) and (1,0) partitions) the E4M3 values are written: keep the
-                               input instead when tensor_format says BF16                        */
+                               (0,0) partition) the E4M3 values are written: keep the input
+                               instead when tensor_format says BF16.  Per-channel partitions take
+                               this output and bf16_fallback with the tensor-level criterion only
+                               (a per-channel decision is known after the codes are written)      */
     uint32_t* error_histogram; /* optional, DEVICE, [MOR_ERROR_BINS] counters of the relative-error
                                histogram of Section 4.1.3: the call adds one to the bin that holds the
                                tensor's error of Eq. 1 (tensor_stats.mean_rel_e4m3).  Bin k covers

@@ -223,6 +223,8 @@ def grid_of(rows: int, cols: int, block) -> tuple:
         return (1, 1)
     if tuple(block) == (1, 0):          # per-channel: one block per row
         return (rows, 1)
+    if tuple(block) == (0, 1):          # per-channel along the columns: one block per column
+        return (1, cols)
     return (-(-rows // block[0]), -(-cols // block[1]))
 
 
@@ -289,7 +291,7 @@ def alloc_outputs(rows: int, cols: int, recipe: Recipe, device, *, codes=True, b
 
     g = grid_of(rows, cols, recipe.block)
     nb = g[0] * g[1]
-    transposed = tuple(recipe.block) == (128, 1)
+    transposed = tuple(recipe.block) in ((128, 1), (0, 1))     # column blocks: codes are stored [cols, rows]
     o = Outputs(cols=cols, rows=rows, transposed=transposed)
     ld = ((rows if transposed else cols) + 15) // 16 * 16
     u8 = dict(dtype=torch.uint8, device=device)

@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmor_b200.so")
 SOURCES = ["mor_api.cu", "mor_kernels.cu", "mor_static.cu", "mor_main.cu", "mor_main_tensor.cu", "mor_main_row128.cu",
-           "mor_main_blk128.cu", "mor_main_blk64.cu", "mor_main_col128.cu", "mor_main_channel.cu", "mor_main_dual.cu"]
+           "mor_main_blk128.cu", "mor_main_blk64.cu", "mor_main_col128.cu", "mor_main_channel.cu", "mor_main_dual.cu", "mor_main_colch.cu"]
 OBJ_DIR = os.path.join(HERE, "_build")
 
 

@@ -31,6 +31,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     else if (d.block_rows == 64 && d.block_cols == 64) s.kind = KIND_BLK64;
     else if (d.block_rows == 1 && d.block_cols == 0) s.kind = KIND_CHANNEL;
     else if (d.block_rows == 128 && d.block_cols == 1) s.kind = KIND_COL128;
+    else if (d.block_rows == 0 && d.block_cols == 1) s.kind = KIND_COLCH;
     else return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     const uint64_t nbc = empty ? 0 : (uint64_t)(d.cols + 127) / 128;
@@ -56,11 +57,17 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
     } else if (s.kind == KIND_CHANNEL) {
         s.n_units = empty ? 0u : (uint32_t)d.rows;
         s.n_blocks = s.n_units;
+    } else if (s.kind == KIND_COLCH) {
+        if (d.cols >= (1ll << 31)) return MOR_ERR_UNSUPPORTED;
+        s.n_units = empty ? 0u : (uint32_t)d.cols;
+        s.n_blocks = s.n_units;
     } else {
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
-    s.key_words = (uint64_t)s.n_tiles * ((s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL) ? (uint64_t)kRowKeyStride : (uint64_t)kTileKeyStride);
+    const bool line_keys = s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL || s.kind == KIND_COLCH;
+    s.key_words = (uint64_t)s.n_tiles * (line_keys ? (uint64_t)kRowKeyStride : (uint64_t)kTileKeyStride);
+    if (s.kind == KIND_COLCH) s.key_words += (uint64_t)s.nbc * kTileCols + (uint64_t)s.n_tiles * kTileCols * 4;   // as for rows, below
     if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows      // + one key per row
                                              + (uint64_t)s.n_tiles * kTileRows * 4; // + per tile and row the partial sums of a per-row decision
     return MOR_OK;
@@ -90,7 +97,7 @@ mor_status_t check_desc(const mor_tensor_desc_t& d, Shape& s)
     // per-channel blocks span many tiles: their decision (tensor-level as in Section 4.1, or per row by Eq. 3 or by
     // Eq. 1-2 on the row) is taken after the main kernel, when the codes are written; a row that chose E5M2 would need
     // its codes rewritten, so three formats are not offered here
-    if (s.kind == KIND_CHANNEL && d.n_formats != 2) return MOR_ERR_UNSUPPORTED;
+    if ((s.kind == KIND_CHANNEL || s.kind == KIND_COLCH) && d.n_formats != 2) return MOR_ERR_UNSUPPORTED;
     if (d.scale_mode < MOR_SCALE_GAM || d.scale_mode > MOR_SCALE_FP32_AMAX) return MOR_ERR_INVALID_ARG;
     if (!(d.threshold >= 0.0f) || std::isinf(d.threshold)) return MOR_ERR_INVALID_ARG;
     if (d.flags & ~(uint32_t)(MOR_FLAG_STRICT_TIES | MOR_FLAG_RANGE_MIN_INCLUDES_ZERO)) return MOR_ERR_INVALID_ARG;
@@ -104,13 +111,15 @@ mor_status_t check_out(const mor_tensor_desc_t& d, const Shape& s, const mor_out
     if (o.error_histogram && !aligned(o.error_histogram, 4)) return MOR_ERR_ALIGNMENT;
     if (!aligned(o.tensor_stats, 8) || !aligned(o.block_stats, 4) || !aligned(o.scale_f32, 4)) return MOR_ERR_ALIGNMENT;
     // a per-row decision of the per-channel partition is known only after the main kernel: no BF16 outputs that depend on it
-    if (s.kind == KIND_CHANNEL && d.criterion != MOR_CRIT_TENSOR_MEAN_REL && (o.bf16_fallback != nullptr || o.fake_quant != nullptr))
+    if ((s.kind == KIND_CHANNEL || s.kind == KIND_COLCH) && d.criterion != MOR_CRIT_TENSOR_MEAN_REL &&
+        (o.bf16_fallback != nullptr || o.fake_quant != nullptr))
         return MOR_ERR_UNSUPPORTED;
     const bool empty = d.rows == 0 || d.cols == 0;
     if (store) {
         if (!empty && o.codes == nullptr) return MOR_ERR_INVALID_ARG;
         // sub-column blocks leave their codes transposed: [cols, codes_ld] with the rows along the contiguous dimension
-        if (o.codes_ld < (int64_t)round_up((size_t)(s.kind == KIND_COL128 ? d.rows : d.cols), 16)) return MOR_ERR_INVALID_ARG;
+        const bool transposed = s.kind == KIND_COL128 || s.kind == KIND_COLCH;
+        if (o.codes_ld < (int64_t)round_up((size_t)(transposed ? d.rows : d.cols), 16)) return MOR_ERR_INVALID_ARG;
         if (o.codes_ld % 16 != 0 || !aligned(o.codes, 16)) return MOR_ERR_ALIGNMENT;
         if (d.scale_mode == MOR_SCALE_FP32_AMAX && o.scale_f32 == nullptr && s.n_blocks) return MOR_ERR_INVALID_ARG;
         if (o.fake_quant && !aligned(o.fake_quant, 16)) return MOR_ERR_ALIGNMENT;
@@ -163,7 +172,7 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
     if (store) {
         const cuuint64_t out_stride[1] = {(cuuint64_t)o.codes_ld};
         const cuuint64_t dims_t[2] = {(cuuint64_t)d.rows, (cuuint64_t)d.cols};      // transposed codes of sub-column blocks
-        const bool transposed = d.block_rows == 128 && d.block_cols == 1;
+        const bool transposed = d.block_cols == 1 && (d.block_rows == 128 || d.block_rows == 0);
         if (enc(&out_map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, o.codes, transposed ? dims_t : dims, out_stride, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -220,10 +229,11 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
     r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
-    r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
-    r.row_keys = (it.prepass && it.s.kind == KIND_CHANNEL) ? r.keys + (size_t)it.s.n_tiles * kRowKeyStride : nullptr;
-    const bool per_row = it.s.kind == KIND_CHANNEL && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || it.o.block_stats != nullptr);
-    r.row_part = per_row && r.row_keys ? reinterpret_cast<float4*>(r.row_keys + (size_t)it.s.nbr * kTileRows) : nullptr;
+    const bool lines = it.s.kind == KIND_CHANNEL || it.s.kind == KIND_COLCH;     // blocks are whole rows / whole columns
+    r.key_stride = (it.s.kind == KIND_ROW128 || lines) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
+    r.row_keys = (it.prepass && lines) ? r.keys + (size_t)it.s.n_tiles * kRowKeyStride : nullptr;
+    const bool per_row = lines && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || it.o.block_stats != nullptr);
+    r.row_part = per_row && r.row_keys ? reinterpret_cast<float4*>(r.row_keys + (size_t)(it.s.kind == KIND_COLCH ? it.s.nbc : it.s.nbr) * kTileRows) : nullptr;
     r.rows = d.rows; r.cols = d.cols; r.ld = d.ld; r.codes_ld = it.o.codes_ld;
     r.nbc = it.s.nbc; r.nbr = it.s.nbr; r.n_units = it.s.n_units; r.n_tiles = it.s.n_tiles;
     r.nbc_blk = (uint32_t)((d.cols + 63) / 64); r.kind = it.s.kind;
@@ -302,7 +312,7 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
             if (bp.n == 0) return true;
             bool ok = launch_amax(bp, t_end, stream) == cudaSuccess;
             bool channel = false;
-            for (int k = 0; k < bp.n; ++k) channel = channel || bp.t[k].kind == KIND_CHANNEL;
+            for (int k = 0; k < bp.n; ++k) channel = channel || bp.t[k].kind == KIND_CHANNEL || bp.t[k].kind == KIND_COLCH;
             if (ok && channel) ok = launch_row_keys(bp, stream) == cudaSuccess;
             bp.n = 0; t_end = 0;
             return ok;
@@ -368,10 +378,10 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     }
     if (ev && !record(ev->main_end)) return MOR_ERR_CUDA;
     for (Chunk& c : chunks) {
-        if (c.kind == KIND_CHANNEL) {
+        if (c.kind == KIND_CHANNEL || c.kind == KIND_COLCH) {
             bool per_row = false;
             for (int k = 0; k < c.bp.n; ++k) per_row = per_row || c.bp.t[k].row_part != nullptr;
-            if (per_row && launch_row_decide(c.bp, partials, stream) != cudaSuccess) return MOR_ERR_CUDA;
+            if (per_row && launch_row_decide(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
         }
         if (c.kind != KIND_DUAL) {
             if (launch_finalise(c.bp, partials, c.kind, stream) != cudaSuccess) return MOR_ERR_CUDA;
@@ -404,13 +414,13 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     it.v.yard = it.v.three || d->criterion == MOR_CRIT_BLOCK_VS_E5M2 || o.block_stats != nullptr;
     it.v.store = store;
     it.v.extra = (store && (o.bf16_fallback != nullptr || o.fake_quant != nullptr)) || o.block_stats != nullptr ||
-                 (it.s.kind == KIND_CHANNEL && d->criterion != MOR_CRIT_TENSOR_MEAN_REL) ||
+                 ((it.s.kind == KIND_CHANNEL || it.s.kind == KIND_COLCH) && d->criterion != MOR_CRIT_TENSOR_MEAN_REL) ||
                  d->criterion == MOR_CRIT_BLOCK_MEAN_REL || (d->flags & MOR_FLAG_RANGE_MIN_INCLUDES_ZERO) != 0;
     // a supplied group amax only fixes the shared mantissa, so the pre-pass can be skipped -- except for
     // the per-tensor partition, whose block amax is the tensor amax and has to come from the data
     // Nor is it needed where the scale has no shared mantissa (E8M0 and FP32-amax modes): those need the block
     // amax only, which the main kernel finds in the tile it has just read, so the tensor is read once.
-    const bool whole_rows = it.s.kind == KIND_TENSOR || it.s.kind == KIND_CHANNEL;
+    const bool whole_rows = it.s.kind == KIND_TENSOR || it.s.kind == KIND_CHANNEL || it.s.kind == KIND_COLCH;
     it.prepass = it.s.n_tiles != 0 && (whole_rows || (d->group_amax == nullptr && d->scale_mode == MOR_SCALE_GAM));
     it.v.scan = !it.prepass || it.s.kind == KIND_COL128;       // sub-column blocks: the main kernel always scans
     it.dual = 0;
@@ -584,7 +594,7 @@ mor_status_t mor_analyze_quantize_host(const mor_tensor_desc_t* host_desc, const
     if (host_out->bf16_fallback != nullptr) return MOR_ERR_UNSUPPORTED;   // the fallback is the caller's own host tensor
     if (host_out->fake_quant != nullptr) return MOR_ERR_UNSUPPORTED;
     if (host_out->error_histogram != nullptr) return MOR_ERR_UNSUPPORTED;  // a device array that outlives the call
-    if (host_desc->block_rows == 128 && host_desc->block_cols == 1) return MOR_ERR_UNSUPPORTED;   // transposed codes: device entry points only
+    if (host_desc->block_cols == 1) return MOR_ERR_UNSUPPORTED;   // column blocks leave transposed codes: device entry points only
     if (host_desc->rows < 0 || host_desc->cols < 0 || host_desc->ld < host_desc->cols) return MOR_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int64_t dev_codes_ld = (int64_t)round_up((size_t)host_desc->cols, 16);

@@ -33,7 +33,10 @@ constexpr int kMaxBatch = 16;          // tensors per launch; records and tensor
 enum Kind : int { KIND_TENSOR = 0, KIND_ROW128 = 1, KIND_BLK128 = 2, KIND_BLK64 = 3, KIND_CHANNEL = 4, KIND_COL128 = 5,
                   // main kernel only: 1x128 blocks and 128x1 blocks of the same tensor from one read of each tile; the
                   // launch's records come in pairs (rows, columns) that share their tiles
-                  KIND_DUAL = 6 };
+                  KIND_DUAL = 6,
+                  // per-channel along the columns: one block per column; computed like 128x1 blocks (column pieces,
+                  // transposed codes) with the column's scale taken from keys that span all tile rows
+                  KIND_COLCH = 7 };
 
 // Per-tile partial results, reduced in tile order by the finalise kernel.
 struct Partial {
@@ -59,8 +62,9 @@ struct TensorRec {
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
-    uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows
-    float4* row_part;             // KIND_CHANNEL with a per-row decision or per-row statistics: per tile and row of the tile
+    uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows;
+                                  // KIND_COLCH: one key per column, padded to 128 columns
+    float4* row_part;             // KIND_CHANNEL / KIND_COLCH with a per-line decision or per-line statistics: per tile and row (column) of the tile
                                   // {sum of E4M3 terms, sum of E5M2 terms, bits(non-zeros | non-finites << 16), unused},
                                   // written by the main kernel, added up along each row by mor_row_decide_kernel
     uint32_t key_stride;          // words per tile in `keys`: kRowKeyStride (one key per row piece, then the tile's
@@ -139,8 +143,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 #endif
 
 cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
-cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);
-cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);      // per-channel: keys of whole rows / whole columns
+cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, int kind, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int kind, cudaStream_t s);
 

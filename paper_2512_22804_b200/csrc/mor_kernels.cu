@@ -114,6 +114,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
 {
     __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32], s_wnz[kThreads / 32];
     __shared__ uint32_t s_qkey[kThreads / 32][4], s_qnf[kThreads / 32][4];   // 64x64 blocks: per warp and quadrant
+    __shared__ uint32_t s_cm[kThreads / 32][64], s_cn[kThreads / 32][64], s_cf[kThreads / 32][16];   // per-channel columns
 
     pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -149,7 +150,8 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             }
         }
     }
-    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride;
+    const bool col_piece = R.keys != nullptr && R.kind == KIND_COLCH;      // per-channel columns: one key per column piece of the tile
+    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && !col_piece;
     uint32_t key[8], all = 0u, nf = 0u;
     // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once.  The
     // main kernel takes the tile's count from here and need not count while it converts.
@@ -235,6 +237,57 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             if ((lane & 7) == 0 && lane < 16) { s_qkey[warp][2 * r + (lane >> 3)] = kq[r]; s_qnf[warp][2 * r + (lane >> 3)] = nq[r]; }
         }
     }
+    if (col_piece) {
+        // One key per column of the tile.  This thread holds 8 rows of 8 columns: per column the maximum and the
+        // wrapped minimum over its rows, packed two columns to a word; lanes l and l ^ 16 hold the same columns of
+        // other rows; the warps' results meet in shared memory and 128 threads finish one column each.
+        uint32_t cm[4] = {0u, 0u, 0u, 0u}, cn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu}, cf = 0u;
+        if (!warp_nf) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t a[4] = {v[j].x & 0x7FFF7FFFu, v[j].y & 0x7FFF7FFFu, v[j].z & 0x7FFF7FFFu, v[j].w & 0x7FFF7FFFu};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { cm[i] = __vimax3_u16x2(cm[i], a[i], a[i]); cn[i] = __viaddmin_u16x2(a[i], 0xFFFFFFFFu, cn[i]); }
+            }
+        } else {
+            // NaN or inf somewhere in the warp's data: element by element, finite ones only (rare path)
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t w4[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+                for (int i = 0; i < 4; ++i)
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const uint32_t x = (w4[i] >> (16 * hf)) & 0x7FFFu;
+                        if (x >= kBf16Inf) { cf |= 1u << (2 * i + hf); continue; }
+                        const uint32_t m = (cm[i] >> (16 * hf)) & 0xFFFFu, n = (cn[i] >> (16 * hf)) & 0xFFFFu;
+                        const uint32_t m2 = max(m, x), n2 = min(n, (x - 1u) & 0xFFFFu);
+                        cm[i] = (cm[i] & ~(0xFFFFu << (16 * hf))) | (m2 << (16 * hf));
+                        cn[i] = (cn[i] & ~(0xFFFFu << (16 * hf))) | (n2 << (16 * hf));
+                    }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t om = __shfl_xor_sync(0xFFFFFFFFu, cm[i], 16), on = __shfl_xor_sync(0xFFFFFFFFu, cn[i], 16);
+            cm[i] = __vimax3_u16x2(cm[i], om, om);
+            cn[i] = __vimin3_u16x2(cn[i], on, on);
+        }
+        cf |= __shfl_xor_sync(0xFFFFFFFFu, cf, 16);
+        if (lane < 16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { s_cm[warp][4 * lane + i] = cm[i]; s_cn[warp][4 * lane + i] = cn[i]; }
+            s_cf[warp][lane] = cf;
+        }
+        __syncthreads();
+        if (t < kTileCols) {
+            const int wd = t >> 1, sh = 16 * (t & 1);
+            uint32_t m = 0u, n = 0xFFFFu, f = 0u;
+            for (int wp = 0; wp < kThreads / 32; ++wp) {
+                m = max(m, (s_cm[wp][wd] >> sh) & 0xFFFFu);
+                n = min(n, (s_cn[wp][wd] >> sh) & 0xFFFFu);
+                f |= (s_cf[wp][t >> 3] >> (t & 7)) & 1u;
+            }
+            R.keys[(size_t)local * kRowKeyStride + t] = (m << 16) | (0xFFFFu - n) | (f << 31);
+        }
+    }
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
     nz = __reduce_add_sync(0xFFFFFFFFu, nz);
@@ -244,14 +297,14 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
         uint32_t kk = s_wkey[0];
         for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; nz += s_wnz[i]; }
         // finite non-zero elements of the tile (NaN and inf are non-zero patterns: taken off)
-        if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (per_piece ? (uint32_t)kTileRows : 4u)] = nz - nf;
+        if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)] = nz - nf;
         if (R.keys != nullptr && R.kind == KIND_BLK64) {
             for (int q = 0; q < 4; ++q) {
                 uint32_t kq = s_qkey[0][q], nq = s_qnf[0][q];
                 for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, s_qkey[i][q]); nq |= s_qnf[i][q]; }
                 R.keys[(size_t)local * kTileKeyStride + q] = kq | (nq ? 0x80000000u : 0u);
             }
-        } else if (R.keys != nullptr && !per_piece) {
+        } else if (R.keys != nullptr && !per_piece && !col_piece) {
             R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
         }
         // non-negative binary32 patterns order like the values
@@ -261,17 +314,21 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     }
 }
 
-// Per-channel partition: a block is a whole row, so its key is the combination of the keys of the row's
-// 128-element pieces over all tiles of the tile row.  One CTA of 128 threads per (tile row, tensor).
+// Per-channel partition: a block is a whole row (a whole column), so its key is the combination of the keys of the
+// row's 128-element pieces over all tiles of the tile row (of the column's pieces over all tiles of the tile column).
+// One CTA of 128 threads per (tile row or tile column, tensor).
 __global__ void __launch_bounds__(kTileRows)
 mor_row_keys_kernel(const __grid_constant__ BatchParams p)
 {
     pdl_trigger();
     const TensorRec& R = p.t[blockIdx.y];
-    if (R.kind != KIND_CHANNEL || R.row_keys == nullptr || blockIdx.x >= R.nbr) return;
-    const uint32_t* src = R.keys + ((size_t)blockIdx.x * R.nbc) * kRowKeyStride + threadIdx.x;
+    const bool cols = R.kind == KIND_COLCH;
+    if ((R.kind != KIND_CHANNEL && !cols) || R.row_keys == nullptr || blockIdx.x >= (cols ? R.nbc : R.nbr)) return;
+    const uint32_t n = cols ? R.nbr : R.nbc;
+    const size_t first = cols ? (size_t)blockIdx.x : (size_t)blockIdx.x * R.nbc, stride = cols ? (size_t)R.nbc : 1u;
+    const uint32_t* src = R.keys + first * kRowKeyStride + threadIdx.x;
     uint32_t k = 0u, flag = 0u;
-    for (uint32_t j = 0; j < R.nbc; ++j, src += kRowKeyStride) {
+    for (uint32_t j = 0; j < n; ++j, src += stride * kRowKeyStride) {
         const uint32_t v = *src;
         flag |= v & 0x80000000u;
         k = key_max(k, v & 0x7FFFFFFFu);
@@ -280,23 +337,26 @@ mor_row_keys_kernel(const __grid_constant__ BatchParams p)
 }
 
 // Per-channel partition with a per-row decision (Algorithm 2 with one block per row) or per-row statistics: the
-// row's sums are the sums of its tiles' parts, added in tile order in double.  One CTA of 128 threads per (tile row,
-// tensor); writes sel, block statistics and, into the partial of the tile row's first tile, the counts of rows per
-// format, which the finalise kernel adds up.
+// row's sums are the sums of its tiles' parts, added in tile order in double (likewise for whole columns).  One CTA
+// of 128 threads per (tile row or tile column, tensor); writes sel, block statistics and, into the partial of the
+// line of tiles' first tile, the counts of rows (columns) per format, which the finalise kernel adds up.
 __global__ void __launch_bounds__(kTileRows)
 mor_row_decide_kernel(const __grid_constant__ BatchParams p, Partial* __restrict__ partials)
 {
     __shared__ uint32_t s_n4[kTileRows / 32], s_nb[kTileRows / 32];
     pdl_wait();                                          // the main kernel's row parts are complete
     const TensorRec& R = p.t[blockIdx.y];
-    if (R.kind != KIND_CHANNEL || R.row_part == nullptr || blockIdx.x >= R.nbr) return;
+    const bool cols = R.kind == KIND_COLCH;              // blocks are whole columns: `row` below is a column
+    if ((R.kind != KIND_CHANNEL && !cols) || R.row_part == nullptr || blockIdx.x >= (cols ? R.nbc : R.nbr)) return;
     const long long row = (long long)blockIdx.x * kTileRows + threadIdx.x;
-    const bool valid = row < R.rows;
+    const bool valid = row < (cols ? R.cols : R.rows);
+    const uint32_t n = cols ? R.nbr : R.nbc;
+    const size_t first = cols ? (size_t)blockIdx.x : (size_t)blockIdx.x * R.nbc, stride = cols ? (size_t)R.nbc : 1u;
     double s43 = 0.0, s52 = 0.0;
     uint32_t nnz = 0u, nonf = 0u;
     if (valid) {
-        const float4* src = R.row_part + ((size_t)blockIdx.x * R.nbc) * kTileRows + threadIdx.x;
-        for (uint32_t j = 0; j < R.nbc; ++j, src += kTileRows) {
+        const float4* src = R.row_part + first * kTileRows + threadIdx.x;
+        for (uint32_t j = 0; j < n; ++j, src += stride * kTileRows) {
             const float4 v = *src;
             const uint32_t nz = __float_as_uint(v.z);
             s43 += (double)v.x; s52 += (double)v.y; nnz += nz & 0xFFFFu; nonf += nz >> 16;
@@ -328,7 +388,7 @@ mor_row_decide_kernel(const __grid_constant__ BatchParams p, Partial* __restrict
         if ((threadIdx.x & 31) == 0) { s_n4[threadIdx.x >> 5] = __popc(b4); s_nb[threadIdx.x >> 5] = __popc(bb); }
         __syncthreads();
         if (threadIdx.x == 0) {
-            Partial& P = partials[R.tile_begin + (size_t)blockIdx.x * R.nbc];
+            Partial& P = partials[R.tile_begin + first];
             P.n_e4m3 = s_n4[0] + s_n4[1] + s_n4[2] + s_n4[3];
             P.n_e5m2 = 0u;
             P.n_bf16 = s_nb[0] + s_nb[1] + s_nb[2] + s_nb[3];
@@ -455,18 +515,23 @@ cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s)
 {
     uint32_t nbr = 0;
-    for (int i = 0; i < p.n; ++i)
+    for (int i = 0; i < p.n; ++i) {
         if (p.t[i].kind == KIND_CHANNEL && p.t[i].nbr > nbr) nbr = p.t[i].nbr;
+        if (p.t[i].kind == KIND_COLCH && p.t[i].nbc > nbr) nbr = p.t[i].nbc;
+    }
     if (nbr == 0) return cudaSuccess;
     mor_row_keys_kernel<<<dim3(nbr, (unsigned)p.n), kTileRows, 0, s>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, cudaStream_t s)
+cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, int kind, cudaStream_t s)
 {
     uint32_t nbr = 0;
-    for (int i = 0; i < p.n; ++i)
-        if (p.t[i].kind == KIND_CHANNEL && p.t[i].row_part != nullptr && p.t[i].nbr > nbr) nbr = p.t[i].nbr;
+    for (int i = 0; i < p.n; ++i) {
+        if (p.t[i].kind != kind || p.t[i].row_part == nullptr) continue;
+        const uint32_t lines = kind == KIND_COLCH ? p.t[i].nbc : p.t[i].nbr;
+        if (lines > nbr) nbr = lines;
+    }
     if (nbr == 0) return cudaSuccess;
     return launch_dependent(mor_row_decide_kernel, dim3(nbr, (unsigned)p.n), dim3(kTileRows), 0, s, p, partials);
 }
@@ -487,6 +552,7 @@ cudaError_t launch_finalise(const BatchParams& p, const Partial* partials, int k
         case KIND_BLK64: e = launch_dependent(mor_finalise_kernel<KIND_BLK64>, grid, dim3(kThreads), 0, s, p, partials); break;
         case KIND_CHANNEL: e = launch_dependent(mor_finalise_kernel<KIND_CHANNEL>, grid, dim3(kThreads), 0, s, p, partials); break;
         case KIND_COL128: e = launch_dependent(mor_finalise_kernel<KIND_COL128>, grid, dim3(kThreads), 0, s, p, partials); break;
+        case KIND_COLCH: e = launch_dependent(mor_finalise_kernel<KIND_COLCH>, grid, dim3(kThreads), 0, s, p, partials); break;
         default: return cudaErrorInvalidValue;
     }
     return e;

@@ -11,6 +11,7 @@ cudaError_t launch_main_blk64(const MainVariant& v, const MainParams& p, Partial
 cudaError_t launch_main_col128(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_main_channel(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 cudaError_t launch_main_dual(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
+cudaError_t launch_main_colch(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);
 
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s)
 {
@@ -23,6 +24,7 @@ cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* part
         case KIND_COL128: return launch_main_col128(v, p, partials, s);
         case KIND_CHANNEL: return launch_main_channel(v, p, partials, s);
         case KIND_DUAL: return launch_main_dual(v, p, partials, s);
+        case KIND_COLCH: return launch_main_colch(v, p, partials, s);
     }
     return cudaErrorInvalidValue;
 }

@@ -768,8 +768,9 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     const uint32_t s = it % kStages;
     const TileId t = locate_tile(p.b, tile);
     const TensorRec& R = p.b.t[t.ti];
-    const uint32_t key_bytes = R.keys == nullptr ? 0u : (KIND == KIND_CHANNEL ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
-    const uint32_t* key_src = KIND == KIND_CHANNEL ? R.row_keys + t.row0 : R.keys + (size_t)t.local * R.key_stride;
+    const uint32_t key_bytes = R.keys == nullptr ? 0u : ((KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
+    const uint32_t* key_src = KIND == KIND_CHANNEL ? R.row_keys + t.row0 : KIND == KIND_COLCH ? R.row_keys + t.col0
+                                                   : R.keys + (size_t)t.local * R.key_stride;
     // (test hook: for one chosen tile neither the copies nor their arrival are issued, so that the tile's barrier
     // never completes and the bounded waits of the other warps run out)
     if (lane == 0 && tile != p.test_skip_tile) {
@@ -786,7 +787,7 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
             if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
         }
         tile_nnz = R.keys[(size_t)t.local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)];
-        if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL) {
+        if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_COLCH) {      // one key per row (per column) of the tile
             uint32_t key[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) key[k] = key_src[lane + 32 * k];
@@ -824,6 +825,7 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
         m.blk_base = (uint32_t)t.row0 * R.nbc + (uint32_t)(t.col0 / kTileCols);
         if (KIND == KIND_COL128) m.blk_base = (uint32_t)(t.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)t.col0;
         if (KIND == KIND_CHANNEL) m.blk_base = t.col0 == 0 ? (uint32_t)t.row0 : 0xFFFFFFFFu;   // first tile of its rows: writes the row scales
+        if (KIND == KIND_COLCH) m.blk_base = t.row0 == 0 ? (uint32_t)t.col0 : 0xFFFFFFFFu;     // first tile of its columns: the column scales
         m.nnz = tile_nnz;
         C.meta[s] = m;
         C.issued = it + 1;
@@ -870,7 +872,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         const uint32_t tile = blockIdx.x + (KIND == KIND_DUAL ? it >> 1 : it) * gridDim.x;
         if (tile >= p.total_tiles) break;
         const uint32_t b = it & 1u, n = it >> 1;
-        const bool columns = KIND == KIND_COL128 || (KIND == KIND_DUAL && (it & 1u));
+        const bool columns = KIND == KIND_COL128 || KIND == KIND_COLCH || (KIND == KIND_DUAL && (it & 1u));
         TileId t = locate_tile(p.b, tile);              // before the wait: off the critical path
         if (KIND == KIND_DUAL && columns) t.ti += 1;
         const TensorRec& R = p.b.t[t.ti];
@@ -1125,7 +1127,8 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     // Sub-column blocks read 16-bit pieces down a column; all rows of a column share a bank, so there
     // the two columns that share a 32-bit word get the same order (they then read the same word) at the
     // price of a two-way conflict on the stores.
-    const int swz = KIND == KIND_COL128 ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
+    constexpr bool kColumns = KIND == KIND_COL128 || KIND == KIND_COLCH;   // the thread holds a column piece, codes are stored transposed
+    const int swz = kColumns ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
     constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;
     const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
     const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
@@ -1170,14 +1173,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
 #ifdef MOR_NO_STREAM
         constexpr bool kStream = false;
 #else
-        constexpr bool kStream = !EXTRA && KIND != KIND_COL128;
+        constexpr bool kStream = !EXTRA && !kColumns;
 #endif
         // Three formats: the E5M2 codes of every element are kept in the thread's part of the stage until the block's
         // decision is known (a copy then puts them in place); the stage goes back after that.
         constexpr bool kStash = kStream && THREE && STORE;
         uint32_t w[32];
         if (kStream) {
-        } else if (KIND == KIND_COL128) {
+        } else if (kColumns) {
             // sub-column blocks: this thread takes column `row` of the tile, rows 64 h .. 64 h + 63, two rows
             // per word, so that everything after this point works on the block as on a row piece
             const uint32_t a = in_base + s * kInBytes + (uint32_t)(h * 64 * 256 + row * 2);
@@ -1195,7 +1198,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             cur_ti = m.ti;
             has_fallback = EXTRA && STORE && R.fallback != nullptr;
             has_fq = EXTRA && STORE && R.fake_quant != nullptr;
-            fq_e4m3 = KIND == KIND_TENSOR || KIND == KIND_CHANNEL || R.criterion == MOR_CRIT_TENSOR_MEAN_REL;
+            fq_e4m3 = KIND == KIND_TENSOR || KIND == KIND_CHANNEL || KIND == KIND_COLCH || R.criterion == MOR_CRIT_TENSOR_MEAN_REL;
             if (SCAN) {
                 scale_mode = R.scale_mode;
                 if (!dead) m_g = group_mantissa(*R.amax, scale_mode);
@@ -1208,7 +1211,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         uint32_t key = 0u, prep = 0u;
         if (!SCAN) {
             // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero; the load warp made the scale
-            const uint32_t e = (KIND == KIND_ROW128 || KIND == KIND_CHANNEL) ? (uint32_t)row * 4u : (uint32_t)q * 4u;
+            const uint32_t e = (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)row * 4u : (uint32_t)q * 4u;
             if (kNeedKey) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kRowKeyStride * 4) + e));
             asm volatile("ld.shared.u32 %0, [%1];" : "=r"(prep) : "r"(prep_base + s * (uint32_t)(kTileRows * 4) + e));
         }
@@ -1387,15 +1390,18 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                        make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), kSelNone | (minm1 << 16)));
                 if (EXTRA && (KIND == KIND_TENSOR || KIND == KIND_CHANNEL) && has_fq)
                     write_fake_quant(R, w, m, row, h, swz, (uint32_t)MOR_FMT_E4M3, s4b, s5b);
-                if (EXTRA && KIND == KIND_CHANNEL && R.row_part != nullptr) {
+                if (EXTRA && (KIND == KIND_CHANNEL || KIND == KIND_COLCH) && R.row_part != nullptr) {
                     // per-row decision or statistics: this tile's part of the row's sums, for mor_row_decide_kernel
                     const float r43 = e43 + __shfl_xor_sync(0xFFFFFFFFu, e43, 1), r52 = e52 + __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
                     uint32_t nz = nnz | (nonf << 16);
                     nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
-                    if (h == 0 && row < m.vrows)
+                    if (h == 0 && row < (KIND == KIND_COLCH ? m.vcols : m.vrows))
                         R.row_part[(size_t)m.local * kTileRows + row] = make_float4(r43, r52, __uint_as_float(nz), 0.0f);
                 }
-                if (KIND == KIND_CHANNEL && h == 0 && m.blk_base != 0xFFFFFFFFu && row < m.vrows) {
+                if (EXTRA && KIND == KIND_COLCH && has_fq)
+                    write_column(R.fake_quant, R.ld, m, row, h, swz, w, true, (uint32_t)MOR_FMT_E4M3, __uint_as_float(s4b));
+                if ((KIND == KIND_CHANNEL || KIND == KIND_COLCH) && h == 0 && m.blk_base != 0xFFFFFFFFu &&
+                    row < (KIND == KIND_COLCH ? m.vcols : m.vrows)) {
                     // per-channel: the row's scale, written by the tile that holds the row's first columns
                     const uint32_t blk = m.blk_base + (uint32_t)row;
                     if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(s4b >> 23);
@@ -1607,7 +1613,7 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
         if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
         else compute_warps<KIND, YARD, THREE, STORE, SCAN, EXTRA>(p, C, in, out, tid);
     }
-    else if (warp == kLoadWarp) load_warp<KIND, !SCAN && KIND != KIND_DUAL && KIND != KIND_COL128>(p, C, in, lane);
+    else if (warp == kLoadWarp) load_warp<KIND, !SCAN && KIND != KIND_DUAL && KIND != KIND_COL128>(p, C, in, lane);   // (COLCH: prepared)
     else store_warp<KIND, THREE, STORE, EXTRA>(p, C, out, partials, lane);
 }
 

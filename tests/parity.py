@@ -39,9 +39,14 @@ def recipe_from_case(case) -> mb.Recipe:
                      threshold=case.threshold)
 
 
-def oracle_block(block, cols):
-    """The block shape as the oracle takes it: per-channel rows (1, 0) are blocks of one whole row."""
-    return (1, cols) if tuple(block) == (1, 0) else tuple(block)
+def oracle_block(block, cols, rows=None):
+    """The block shape as the oracle takes it: per-channel rows (1, 0) are blocks of one whole row, per-channel
+    columns (0, 1) blocks of one whole column (``rows`` needed)."""
+    if tuple(block) == (1, 0):
+        return (1, cols)
+    if tuple(block) == (0, 1):
+        return (rows, 1)
+    return tuple(block)
 
 
 def close(a, b, tol=REL_TOL):
@@ -114,7 +119,7 @@ def compare(bits: np.ndarray, recipe: mb.Recipe, out: "mb.Outputs", ref: "orc.Re
         assert (ts["n_e4m3"], ts["n_e5m2"], ts["n_bf16"]) == (ref.tensor["n_e4m3"], ref.tensor["n_e5m2"], ref.tensor["n_bf16"])
 
     if codes is not None and nb:
-        br, bc = oracle_block(recipe.block, cols) if tuple(recipe.block) != (0, 0) else (rows, cols)
+        br, bc = oracle_block(recipe.block, cols, rows) if tuple(recipe.block) != (0, 0) else (rows, cols)
         if ids is None and not ex.any():
             np.testing.assert_array_equal(codes, ref.codes)
         else:
@@ -207,7 +212,7 @@ def run_and_compare(bits: np.ndarray, recipe: mb.Recipe, *, cols=None, block_sta
         cols = bits.shape[1]
     x = to_device(host)
     ga = None
-    ref = orc.run(host, oracle_block(recipe.block, host.shape[1] if cols is None else cols), list(recipe.formats),
+    ref = orc.run(host, oracle_block(recipe.block, host.shape[1] if cols is None else cols, host.shape[0]), list(recipe.formats),
                   recipe.criterion, recipe.threshold, recipe.scale_mode, recipe.flags, cols=cols)
     if group_amax_supplied:
         ga = torch.tensor([ref.tensor["group_amax"]], dtype=torch.float32, device="cuda")
@@ -222,7 +227,7 @@ def run_and_compare(bits: np.ndarray, recipe: mb.Recipe, *, cols=None, block_sta
         # the fake-quantised tensor, bit for bit, outside blocks whose decision is within the tolerance band;
         # padding columns must stay untouched (zero-initialised output)
         c = host.shape[1] if cols is None else cols
-        ob = oracle_block(recipe.block, c)
+        ob = oracle_block(recipe.block, c, host.shape[0])
         want = orc.fake_quant(host, ref, ob, list(recipe.formats), recipe.criterion, recipe.threshold, recipe.scale_mode,
                               recipe.flags, cols=cols)
         got = out.fake_quant.view(torch.int16).cpu().numpy().view(np.uint16)

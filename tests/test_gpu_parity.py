@@ -232,6 +232,39 @@ def test_per_channel_partition_with_a_decision_per_row(shape, crit):
     parity.run_and_compare(x, recipe((1, 0), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), pad_to=ld, block_stats=True)
 
 
+@pytest.mark.parametrize("shape", [(256, 512), (1000, 130), (72, 300), (2049, 5), (1160, 257)])
+@pytest.mark.parametrize("crit", [mb.MOR_CRIT_TENSOR_MEAN_REL, mb.MOR_CRIT_BLOCK_VS_E5M2, mb.MOR_CRIT_BLOCK_MEAN_REL])
+def test_per_channel_partition_along_the_columns(shape, crit):
+    """One block per column (the operand whose dot-product dimension runs down the rows): the column's amax spans the
+    tile rows, codes come out transposed; tensor-level decision or a decision per column; statistics per column;
+    a zero column, a NaN, columns that span many binades; every scale mode; equals the row version of the transpose."""
+    import torch
+
+    rows, cols = shape
+    x = np.ascontiguousarray(wl.activation_like(cols, rows, n_outlier_cols=min(4, rows), seed=150).T)
+    x[:, cols // 2] = 0
+    wide = np.ascontiguousarray(wl.gradient_like(cols, rows, seed=151).T)
+    x[:, ::3] = wide[:, ::3]
+    if cols > 3:
+        x[rows // 2, 3] = 0x7FC0
+    ld = (cols + 7) // 8 * 8 + 8
+    for mode in (mb.MOR_SCALE_GAM, mb.MOR_SCALE_E8M0, mb.MOR_SCALE_FP32_AMAX):
+        r = recipe((0, 1), TWO, crit, threshold=0.03, scale_mode=mode)
+        rep = parity.run_and_compare(x, r, pad_to=ld, block_stats=True)
+        assert rep.n_blocks == cols and rep.n_exempt <= 1
+    parity.run_and_compare(x, recipe((0, 1), TWO, crit, threshold=0.03), pad_to=ld, block_stats=False, group_amax_supplied=True)
+    if crit == mb.MOR_CRIT_TENSOR_MEAN_REL:
+        parity.run_and_compare(x, recipe((0, 1), TWO, crit, threshold=0.03), pad_to=ld, block_stats=False, fake_quant=True)
+    # the same bytes as per-row blocks of the transposed tensor (where both leading dimensions are multiples of 8)
+    if rows % 8 or cols % 8:
+        return
+    a = mb.analyze_quantize(parity.to_device(x), recipe((0, 1), TWO, crit, threshold=0.03))
+    b = mb.analyze_quantize(parity.to_device(np.ascontiguousarray(x.T)), recipe((1, 0), TWO, crit, threshold=0.03))
+    torch.cuda.synchronize()
+    assert torch.equal(a.codes[:, :rows], b.codes[:, :rows])
+    assert torch.equal(a.sel.reshape(-1), b.sel.reshape(-1)) and torch.equal(a.scale_e8m0.reshape(-1), b.scale_e8m0.reshape(-1))
+
+
 def test_per_channel_partition_refuses_what_it_cannot_give():
     """Three formats (a row that chose E5M2 would need its codes rewritten after the last tile) and BF16 outputs that
     depend on a per-row decision are refused."""

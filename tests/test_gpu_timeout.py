@@ -37,6 +37,7 @@ CASES = [
     ("128x1 sub-column blocks", (128, 1), TWO, {}, False),
     ("per tensor", (0, 0), TWO, {}, False),
     ("per channel", (1, 0), TWO, {}, False),
+    ("per channel along the columns, a decision per column with statistics", (0, 1), TWO, dict(block_stats=True), False),
 ]
 
 
@@ -47,7 +48,7 @@ def test_timeout_is_reported_and_the_workspace_recovers(name, block, formats, kw
 
     bits = wl.gradient_like(512, 512, seed=97)                        # 16 tiles, one per thread block
     x = parity.to_device(bits)
-    crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) else mb.MOR_CRIT_BLOCK_VS_E5M2
+    crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) else mb.MOR_CRIT_BLOCK_VS_E5M2     # (0, 1): per column
     r = mb.Recipe(block, formats, crit)
     ga = mb.group_amax([x]) if supplied else None
     torch.cuda.synchronize()
