@@ -30,7 +30,6 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
-import math
 import os
 import statistics
 import subprocess
@@ -276,6 +275,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--profile", default=None, metavar="RECIPE",
+                    help="run only three calls of one recipe on --batch 4096x4096 tensors and exit (the small case that the "
+                         "profiler wraps): 128x128, 1x128, 64x64, 128x1, per-tensor, per-channel, each optionally followed by "
+                         "-supplied (group amax given: single read) or -three (three formats, gradient-like data)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -306,6 +309,23 @@ def main():
     peak, peak_kind = measured_peak()
     T2, T3 = (mb.MOR_FMT_E4M3, mb.MOR_FMT_BF16), (mb.MOR_FMT_E4M3, mb.MOR_FMT_E5M2, mb.MOR_FMT_BF16)
     E3 = mb.MOR_CRIT_BLOCK_VS_E5M2
+
+    if args.profile:
+        name = args.profile
+        three, supplied = name.endswith("-three"), name.endswith("-supplied")
+        base = name.replace("-three", "").replace("-supplied", "")
+        block = {"128x128": (128, 128), "1x128": (1, 128), "64x64": (64, 64), "128x1": (128, 1), "per-tensor": (0, 0), "per-channel": (1, 0)}[base]
+        crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) else E3
+        gen = (lambda i: wl.gradient_like(ROWS, COLS, seed=3 + i)) if three else (lambda i: wl.weight_like(ROWS, COLS, seed=1 + 1000 * i))
+        pxs = [torch.from_numpy(gen(i).view(np.int16)).view(torch.bfloat16).to(dev) for i in range(args.batch)]
+        ga = mb.group_amax(pxs) if supplied else None
+        pplan = mb.BatchPlan(pxs, [mb.Recipe(block, T3 if three else T2, crit, 0.045)] * args.batch, group_amax=ga)
+        for _ in range(3):
+            pplan.run(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": name, "tensors": args.batch, "elements_per_call": ROWS * COLS * args.batch,
+                          "status": [o.tensor_stats_dict()["status"] for o in pplan.outs]}), flush=True)
+        return
 
     # ---- inputs: `batch` distinct tensors per rank, resident in HBM
     B = args.batch
