@@ -428,12 +428,9 @@ def main():
                                     [(g, mb.Recipe((1, 128), T3, E3))], 3, dev, peak, mb))
         configs.append(bench_config("configs[3] 8192x14336 gradient-like, 128x128, three-way (3 copies per call)",
                                     [(g, mb.Recipe((128, 128), T3, E3))], 3, dev, peak, mb))
-        # a grid of 128x128 blocks that really is mixed: per-tile exponent spread drawn between 4 and 24 binades
-        rng = np.random.default_rng(11)
-        mixed = wl.to_bf16_bits(np.repeat(np.repeat(np.exp2(rng.uniform(-12, 0, (32, 32))), 128, 0), 128, 1) *
-                                np.exp2(rng.uniform(-1, 0, (4096, 4096)) * np.repeat(np.repeat(rng.uniform(4, 24, (32, 32)), 128, 0), 128, 1)) *
-                                rng.choice([-1.0, 1.0], (4096, 4096)))
-        configs.append(bench_config("mixed grid: 4096x4096, per-tile spread of 4..24 binades, 128x128, three-way (16 copies per call)",
+        # a grid of 128x128 blocks that really is mixed: per-tile exponent spread drawn between 4 and 36 binades
+        mixed = wl.mixed_grid()
+        configs.append(bench_config("mixed grid: 4096x4096, per-tile spread of 4..36 binades (E4M3, E5M2 and BF16 tiles side by side), 128x128, three-way (16 copies per call)",
                                     [(mixed, mb.Recipe((128, 128), T3, E3))], 16, dev, peak, mb))
         del g, mixed
         cases = wl.config_case(4)

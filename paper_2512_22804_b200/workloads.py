@@ -76,6 +76,18 @@ def gradient_like(rows=8192, cols=14336, mu=-13.0, sd=5.67, lo=-30.0, hi=4.0, p_
     return to_bf16_bits(a)
 
 
+def mixed_grid(rows=4096, cols=4096, tile=128, lo_spread=4.0, hi_spread=36.0, seed=11):
+    """A tensor whose 128x128 tiles differ: one magnitude level per tile drawn from 2**U(-12, 0) and, inside a tile,
+    magnitudes spread uniformly in the exponent over a per-tile number of binades between ``lo_spread`` and
+    ``hi_spread``; random signs.  Narrow tiles suit E4M3, wide ones E5M2 or BF16, side by side."""
+    rng = np.random.default_rng(seed)
+    tr, tc = -(-rows // tile), -(-cols // tile)
+    level = np.repeat(np.repeat(np.exp2(rng.uniform(-12, 0, (tr, tc))), tile, 0), tile, 1)[:rows, :cols]
+    spread = np.repeat(np.repeat(rng.uniform(lo_spread, hi_spread, (tr, tc)), tile, 0), tile, 1)[:rows, :cols]
+    a = level * np.exp2(rng.uniform(-1, 0, (rows, cols)) * spread) * rng.choice([-1.0, 1.0], (rows, cols))
+    return to_bf16_bits(a)
+
+
 @dataclass
 class Case:
     """One tensor plus the recipe it is analysed with."""

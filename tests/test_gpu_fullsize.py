@@ -34,7 +34,7 @@ def test_config1_batched_launch_as_benchmarked():
     host = [wl.weight_like(4096, 4096, seed=1 + 1000 * i) for i in range(B)]
     xs = [parity.to_device(h) for h in host]
     r = mb.Recipe((128, 128), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
-    plan = mb.BatchPlan(xs, [r] * B, block_stats=True)
+    plan = mb.BatchPlan(xs, [r] * B)     # as bench.py builds it: no optional outputs (the plain instantiation)
     plan.run()
     plan.run()                       # the second step must overwrite the first one's results identically
     torch.cuda.synchronize()
@@ -142,3 +142,31 @@ def test_tensor_with_more_than_2_31_elements(block, formats):
     parity.compare(host, r, out, ref, ids=ids)
     assert ts["n_blocks"] == nb == ts["n_e4m3"] + ts["n_e5m2"] + ts["n_bf16"] and ts["status"] == 0
     assert ts["group_amax"] == 3.0 and ts["nnz"] == int(torch.count_nonzero(x).item())
+
+
+def test_mixed_grid_128x128_three_way_full():
+    """A 4096x4096 tensor whose 128x128 tiles differ (E4M3, E5M2 and BF16 blocks side by side), three formats, in
+    bench.py's launch configuration (several copies in one batched call, no optional outputs) and with statistics;
+    the whole tensor against the oracle."""
+    import torch
+
+    bits = wl.mixed_grid()
+    r = mb.Recipe((128, 128), THREE, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+    ref = orc.run(bits, r.block, list(r.formats), r.criterion, r.threshold, n_threads=8)
+    assert min(ref.tensor["n_e4m3"], ref.tensor["n_e5m2"], ref.tensor["n_bf16"]) > 100      # 459 / 388 / 177 tiles
+    xs = [parity.to_device(bits) for _ in range(4)]
+    for stats in (False, True):
+        plan = mb.BatchPlan(xs, [r] * 4, block_stats=stats)
+        plan.run()
+        torch.cuda.synchronize()
+        ex = sum(parity.compare(bits, r, o, ref).n_exempt for o in (plan.outs[0], plan.outs[3]))
+        assert ex <= 4
+        del plan
+    # the same data with 1x128 and 64x64 blocks, sampled
+    for block, nb in (((1, 128), 4096 * 32), ((64, 64), 64 * 64)):
+        rr = mb.Recipe(block, THREE, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+        ids = np.sort(np.random.default_rng(6).choice(nb, 2000, replace=False))
+        sub = orc.run(bits, block, list(THREE), rr.criterion, rr.threshold, ids=ids)
+        out = mb.analyze_quantize(xs[0], rr)
+        torch.cuda.synchronize()
+        assert parity.compare(bits, rr, out, sub, ids=ids).n_exempt <= 4
