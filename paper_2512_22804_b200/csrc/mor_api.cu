@@ -65,7 +65,7 @@ mor_status_t shape_of(const mor_tensor_desc_t& d, Shape& s)
         s.n_units = (uint32_t)segs;
         s.n_blocks = s.kind == KIND_TENSOR ? (empty ? 0 : 1) : segs;
     }
-    const bool line_keys = s.kind == KIND_ROW128 || s.kind == KIND_CHANNEL || s.kind == KIND_COLCH;
+    const bool line_keys = s.kind == KIND_ROW128 || s.kind == KIND_COL128 || s.kind == KIND_CHANNEL || s.kind == KIND_COLCH;
     s.key_words = (uint64_t)s.n_tiles * (line_keys ? (uint64_t)kRowKeyStride : (uint64_t)kTileKeyStride);
     if (s.kind == KIND_COLCH) s.key_words += (uint64_t)s.nbc * kTileCols + (uint64_t)s.n_tiles * kTileCols * 4;   // as for rows, below
     if (s.kind == KIND_CHANNEL) s.key_words += (uint64_t)s.nbr * kTileRows      // + one key per row
@@ -207,6 +207,8 @@ struct Item {
     uint32_t tile_begin;
     uint64_t key_begin;      // first word of the tensor's keys
     bool prepass;            // the amax pre-pass runs for this tensor (and leaves keys)
+    bool has_keys;           // the main kernel finds keys for this tensor (its own pre-pass, or that of the rows' item of its pair)
+    long long col_key_begin; // rows' item of a pair: first word of the columns' item's keys, which its pre-pass fills too (-1: none)
     int dual;                // 1, 2: first (1x128 blocks) and second (128x1 blocks) item of a pair on the same tensor
                              // that the main kernel serves from one read of each tile; 0: not part of a pair
     int index;
@@ -228,9 +230,11 @@ void fill_rec(const Item& it, unsigned char* ws, const Layout& l, TensorRec& r)
     r.amax_slot = reinterpret_cast<float*>(ws + l.amax_off) + it.index;
     r.amax = d.group_amax ? d.group_amax : r.amax_slot;
     r.device_status = reinterpret_cast<const uint32_t*>(ws + l.status_off);
-    r.keys = (it.prepass && it.s.kind != KIND_COL128) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
+    r.keys = it.has_keys ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.key_begin : nullptr;
+    r.col_keys = (it.s.kind == KIND_COL128 || it.s.kind == KIND_COLCH) ? r.keys
+               : (it.prepass && it.col_key_begin >= 0) ? reinterpret_cast<uint32_t*>(ws + l.keys_off) + it.col_key_begin : nullptr;
     const bool lines = it.s.kind == KIND_CHANNEL || it.s.kind == KIND_COLCH;     // blocks are whole rows / whole columns
-    r.key_stride = (it.s.kind == KIND_ROW128 || lines) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
+    r.key_stride = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_COL128 || lines) ? (uint32_t)kRowKeyStride : (uint32_t)kTileKeyStride;
     r.row_keys = (it.prepass && lines) ? r.keys + (size_t)it.s.n_tiles * kRowKeyStride : nullptr;
     const bool per_row = lines && (d.criterion != MOR_CRIT_TENSOR_MEAN_REL || it.o.block_stats != nullptr);
     r.row_part = per_row && r.row_keys ? reinterpret_cast<float4*>(r.row_keys + (size_t)(it.s.kind == KIND_COLCH ? it.s.nbc : it.s.nbr) * kTileRows) : nullptr;
@@ -279,9 +283,12 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
                            a.v.yard == b.v.yard && a.v.three == b.v.three;
         if (!same || !plain) continue;
         a.dual = 1; b.dual = 2;
-        b.prepass = false;                 // the columns are scanned by the main kernel; the tensor amax is the rows' item's
+        b.prepass = false;                 // one pre-pass, the rows' item's, leaves the keys of both and the tensor amax
+        b.has_keys = a.prepass;
+        a.col_key_begin = (long long)b.key_begin;
         a.v.kind = b.v.kind = KIND_DUAL;
         b.v.scan = a.v.scan;
+        a.v.extra = b.v.extra = a.v.extra || b.v.extra;    // (one launch serves both items)
     }
     const Layout l = layout_of(n, tiles, key_words);
     if (workspace == nullptr || workspace_bytes < l.total) return MOR_ERR_WORKSPACE;
@@ -422,7 +429,9 @@ mor_status_t make_item(const mor_tensor_desc_t* d, const mor_outputs_t& o, bool 
     // amax only, which the main kernel finds in the tile it has just read, so the tensor is read once.
     const bool whole_rows = it.s.kind == KIND_TENSOR || it.s.kind == KIND_CHANNEL || it.s.kind == KIND_COLCH;
     it.prepass = it.s.n_tiles != 0 && (whole_rows || (d->group_amax == nullptr && d->scale_mode == MOR_SCALE_GAM));
-    it.v.scan = !it.prepass || it.s.kind == KIND_COL128;       // sub-column blocks: the main kernel always scans
+    it.v.scan = !it.prepass;
+    it.has_keys = it.prepass;
+    it.col_key_begin = -1;
     it.dual = 0;
     return MOR_OK;
 }
@@ -535,7 +544,7 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         d.group_amax = nullptr;
         it.s = shapes[i];
         std::memset(&it.o, 0, sizeof(it.o));
-        it.d = &d; it.index = i; it.tile_begin = 0; it.key_begin = 0; it.prepass = false;   // no keys wanted
+        it.d = &d; it.index = i; it.tile_begin = 0; it.key_begin = 0; it.prepass = false; it.has_keys = false; it.col_key_begin = -1;   // no keys wanted
         if (it.s.n_tiles) {
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);

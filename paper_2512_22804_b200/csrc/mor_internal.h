@@ -62,6 +62,10 @@ struct TensorRec {
     float* amax_slot;             // workspace: tensor amax written by the pre-pass (when it runs)
     const uint32_t* device_status;// workspace: non-zero when a bounded device-side wait expired
     uint32_t* keys;               // workspace: block keys written by the pre-pass (nullptr: none)
+    uint32_t* col_keys;           // workspace: per tile one key per column piece (kRowKeyStride words per tile, the tile's
+                                  // non-zero count after the 128 keys), wanted from the pre-pass.  Blocks along the
+                                  // columns: the same area as `keys`; the rows' record of a rows-and-columns pair: the
+                                  // key area of the columns' record; nullptr: none
     uint32_t* row_keys;           // KIND_CHANNEL: one key per row (the row's amax over all its tiles), padded to 128 rows;
                                   // KIND_COLCH: one key per column, padded to 128 columns
     float4* row_part;             // KIND_CHANNEL / KIND_COLCH with a per-line decision or per-line statistics: per tile and row (column) of the tile

@@ -150,8 +150,8 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
             }
         }
     }
-    const bool col_piece = R.keys != nullptr && R.kind == KIND_COLCH;      // per-channel columns: one key per column piece of the tile
-    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && !col_piece;
+    const bool col_piece = R.col_keys != nullptr;            // blocks along the columns: one key per column piece of the tile
+    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && R.col_keys != R.keys;
     uint32_t key[8], all = 0u, nf = 0u;
     // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once.  The
     // main kernel takes the tile's count from here and need not count while it converts.
@@ -285,7 +285,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
                 n = min(n, (s_cn[wp][wd] >> sh) & 0xFFFFu);
                 f |= (s_cf[wp][t >> 3] >> (t & 7)) & 1u;
             }
-            R.keys[(size_t)local * kRowKeyStride + t] = (m << 16) | (0xFFFFu - n) | (f << 31);
+            R.col_keys[(size_t)local * kRowKeyStride + t] = (m << 16) | (0xFFFFu - n) | (f << 31);
         }
     }
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
@@ -298,6 +298,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
         for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; nz += s_wnz[i]; }
         // finite non-zero elements of the tile (NaN and inf are non-zero patterns: taken off)
         if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)] = nz - nf;
+        if (R.col_keys != nullptr && R.col_keys != R.keys) R.col_keys[(size_t)local * kRowKeyStride + kTileRows] = nz - nf;
         if (R.keys != nullptr && R.kind == KIND_BLK64) {
             for (int q = 0; q < 4; ++q) {
                 uint32_t kq = s_qkey[0][q], nq = s_qnf[0][q];

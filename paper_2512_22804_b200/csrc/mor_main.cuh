@@ -34,6 +34,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <float.h>
+#include <stddef.h>
 
 #include <atomic>
 #include <mutex>
@@ -77,8 +78,8 @@ struct Control {
     unsigned long long dec_full[2];                     // BLK128: the block's decision, when compute threads need it
     unsigned long long codes_full[2];                   // BLK128, three formats: codes in place after the decision
     TileMeta meta[kStages];
-    uint32_t keys[kStages][kRowKeyStride];               // block keys of the tile from the pre-pass (arrive with the tile)
-    uint32_t prep[kStages][kTileRows];                   // by the load warp, from the keys: scale bits of the row's block (entry = row),
+    alignas(16) uint32_t keys[kStages][kRowKeyStride];             // block keys of the tile from the pre-pass (arrive with the tile)
+    alignas(16) uint32_t prep[kStages][kTileRows];              // by the load warp, from the keys: scale bits of the row's block (entry = row),
                                                          // of the quadrant (entry q) or of the tile (entry 0); bit 31: careful path
     Entry entry[2][kThreads];
     // 128x128 and 64x64 blocks (a tile holds one block, or four: index q = 2 * (row >= 64) + (column >= 64))
@@ -87,11 +88,23 @@ struct Control {
     uint32_t tile_key[2][4];                             // amax bits << 16 | 0xFFFF - (min - 1)
     uint32_t dec_sel[2][4];
     uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
+    // blocks along the columns with prepared scales (compute_cols_fast): what the store warp needs per tile besides
+    // the entries -- per column the scale bits (bit 31: the column piece holds NaN or inf), per warp the count of
+    // NaN/inf elements, and the tile's count of finite non-zeros from the pre-pass
+    alignas(16) uint32_t prep2[kStages][kTileCols];      // rows and columns from one read: the columns' prepared scales (prep holds the rows')
+    alignas(16) uint32_t colscale[2][kTileCols];
+    uint32_t colflag[kStages];                           // by the load warp: some column of the tile needs the careful path
+    uint32_t colnonf[2][kComputeWarps];
+    uint32_t colnnz[2];
     uint32_t issued;                                     // tile loads issued so far by this CTA
     volatile uint32_t abort;
 };
 
 constexpr int kSmemBytes = 1024 + kStages * kInBytes + 2 * kOutBytes + (int)sizeof(Control);
+static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM must fit in shared memory");
+static_assert(offsetof(Control, keys) % 16 == 0 && offsetof(Control, prep) % 16 == 0 && offsetof(Control, entry) % 16 == 0 &&
+              offsetof(Control, prep2) % 16 == 0 && offsetof(Control, colscale) % 16 == 0 && offsetof(Control, wmax) % 16 == 0 &&
+              offsetof(Control, meta) % 16 == 0, "16-byte shared-memory accesses");
 
 // ------------------------------------------------------------------ PTX helpers ----
 
@@ -759,7 +772,37 @@ __device__ __forceinline__ bool needs_careful(bool nonfin, uint32_t minm1, uint3
 // also turns the keys into what the compute threads need -- per row, quadrant or tile the scale of Algorithm 1 and
 // whether the careful path is needed -- so that 256 threads need not each derive them.  The stage's barrier takes two
 // arrivals: one with the byte count when the copies start, one when the tile's facts are in shared memory.
-template <int KIND, bool PREP>
+// One key per line (row or column) of the tile -> one prepared word per line: the scale bits of Algorithm 1 and a
+// flag in bit 31.  MODE 0 (rows): the flag says that the line's warp -- lines 16 w .. 16 w + 15, i.e. this half of
+// the lanes -- takes the careful path.  MODE 1 (columns, gathered by 16-bit loads): the same for the CTA as a whole
+// (a warp's elements then come from many columns).  MODE 2 (columns, full-width path): the flag says that the
+// column piece holds NaN or inf (its block then stays in BF16).  Returns whether any line needs the careful path.
+template <int MODE>
+__device__ __forceinline__ bool prepare_lines(const uint32_t* key_src, uint32_t m_g, int scale_mode, const uint32_t* rtab, uint32_t* dst, int lane)
+{
+    uint32_t key[4], sb[4], any[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) key[k] = key_src[lane + 32 * k];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const bool nonfin = (key[k] >> 31) != 0u;
+        const uint32_t kk = key[k] & 0x7FFFFFFFu;
+        uint32_t s5b;
+        block_scale(kk >> 16, m_g, scale_mode, rtab, sb[k], s5b);
+        any[k] = __ballot_sync(0xFFFFFFFFu, needs_careful(nonfin, 0xFFFFu - (kk & 0xFFFFu), sb[k]));
+    }
+    const bool all = (any[0] | any[1] | any[2] | any[3]) != 0u;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        bool flag = ((lane < 16 ? any[k] : any[k] >> 16) & 0xFFFFu) != 0u;
+        if (MODE == 1) flag = all;
+        if (MODE == 2) flag = (key[k] >> 31) != 0u;
+        dst[lane + 32 * k] = sb[k] | (flag ? 0x80000000u : 0u);
+    }
+    return all;
+}
+
+template <int KIND, bool PREP, bool COLFAST>
 __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it, int lane,
                                                 int& cur_ti, uint32_t& m_g, int& scale_mode, uint32_t& tensor_amax_bits)
 {
@@ -768,7 +811,8 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     const uint32_t s = it % kStages;
     const TileId t = locate_tile(p.b, tile);
     const TensorRec& R = p.b.t[t.ti];
-    const uint32_t key_bytes = R.keys == nullptr ? 0u : ((KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
+    // (the full-width column paths need nothing but the prepared words: no copy of the keys)
+    const uint32_t key_bytes = (R.keys == nullptr || COLFAST) ? 0u : ((KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
     const uint32_t* key_src = KIND == KIND_CHANNEL ? R.row_keys + t.row0 : KIND == KIND_COLCH ? R.row_keys + t.col0
                                                    : R.keys + (size_t)t.local * R.key_stride;
     // (test hook: for one chosen tile neither the copies nor their arrival are issued, so that the tile's barrier
@@ -787,20 +831,19 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
             if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
         }
         tile_nnz = R.keys[(size_t)t.local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)];
-        if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_COLCH) {      // one key per row (per column) of the tile
-            uint32_t key[4];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) key[k] = key_src[lane + 32 * k];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const bool nonfin = (key[k] >> 31) != 0u;
-                const uint32_t kk = key[k] & 0x7FFFFFFFu;
-                uint32_t s4b, s5b;
-                block_scale(kk >> 16, m_g, scale_mode, C.rtab, s4b, s5b);
-                // the careful path is taken by a warp as a whole: rows 16 w .. 16 w + 15, i.e. this half of the lanes
-                const uint32_t any = __ballot_sync(0xFFFFFFFFu, needs_careful(nonfin, 0xFFFFu - (kk & 0xFFFFu), s4b));
-                const bool careful = ((lane < 16 ? any : any >> 16) & 0xFFFFu) != 0u;
-                C.prep[s][lane + 32 * k] = s4b | (careful ? 0x80000000u : 0u);
+        if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_DUAL) {          // one key per row of the tile
+            prepare_lines<0>(key_src, m_g, scale_mode, C.rtab, &C.prep[s][0], lane);
+            if (KIND == KIND_DUAL) {
+                // ... and one per column, from the columns' record (same tiles, same group amax)
+                const bool any = prepare_lines<2>(p.b.t[t.ti + 1].keys + (size_t)t.local * kRowKeyStride, m_g, scale_mode, C.rtab, &C.prep2[s][0], lane);
+                if (lane == 0) C.colflag[s] = any ? 1u : 0u;
+            }
+        } else if (KIND == KIND_COL128 || KIND == KIND_COLCH) {                            // one key per column of the tile
+            if (COLFAST) {
+                const bool any = prepare_lines<2>(key_src, m_g, scale_mode, C.rtab, &C.prep[s][0], lane);
+                if (lane == 0) C.colflag[s] = any ? 1u : 0u;
+            } else {
+                prepare_lines<1>(key_src, m_g, scale_mode, C.rtab, &C.prep[s][0], lane);
             }
         } else {
             // one key per tile, or one per quadrant (lanes 0..3; the other lanes repeat lane 0's work)
@@ -834,18 +877,18 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     if (lane == 0) mbar_arrive(&C.full[s]);             // the tile's facts are in place (release)
 }
 
-template <int KIND, bool PREP>
+template <int KIND, bool PREP, bool COLFAST>
 __device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in, int lane)
 {
     int cur_ti = -1, scale_mode = 0;
     uint32_t m_g = 0u, tensor_amax_bits = 0u;
-    for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load<KIND, PREP>(p, C, in, it, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
+    for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
         stage_free_sync(it % kStages);                  // sleeps until every compute thread has its copy
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u))
-            issue_tile_load<KIND, PREP>(p, C, in, it + kStages, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
+            issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it + kStages, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
     }
     if (lane == 0 && C.abort) {
         // copies that may still be in flight must land (or be given up on) before the CTA goes
@@ -859,7 +902,7 @@ __device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsig
 
 // ------------------------------------------------------------------ store warp ----
 
-template <int KIND, bool THREE, bool STORE, bool EXTRA>
+template <int KIND, bool THREE, bool STORE, bool EXTRA, bool COLFAST = false>
 __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsigned char* out, Partial* __restrict__ partials,
                                            int lane)
 {
@@ -892,6 +935,45 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 stores_pending = true;
             }
 
+            if (COLFAST && (KIND != KIND_DUAL || columns)) {
+                // Blocks along the columns, handed over by cols_fast_tile: this lane takes columns 4 lane ..
+                // 4 lane + 3; a column's sums come in four parts (row groups), added in the order of the parts.
+                const uint32_t ea = smem_addr(&C.entry[b][0]) + (uint32_t)lane * 32u;
+                float e43[4] = {0.0f, 0.0f, 0.0f, 0.0f}, e52[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int part = 0; part < 4; ++part) {
+                    const uint4 v0 = lds128(ea + (uint32_t)part * 1024u), v1 = lds128(ea + (uint32_t)part * 1024u + 16u);
+                    e43[0] += __uint_as_float(v0.x); e52[0] += __uint_as_float(v0.y); e43[1] += __uint_as_float(v0.z); e52[1] += __uint_as_float(v0.w);
+                    e43[2] += __uint_as_float(v1.x); e52[2] += __uint_as_float(v1.y); e43[3] += __uint_as_float(v1.z); e52[3] += __uint_as_float(v1.w);
+                }
+                const uint4 sc4 = *reinterpret_cast<const uint4*>(&C.colscale[b][4 * lane]);
+                const uint32_t sc[4] = {sc4.x, sc4.y, sc4.z, sc4.w};
+                uint32_t n4 = 0, n5 = 0, nb = 0;
+                const uint32_t blk0 = (uint32_t)(t.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)t.col0 + 4u * (uint32_t)lane;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (4 * lane + c >= t.vcols) continue;
+                    const uint32_t s4b = sc[c] & 0x7FFFFFFFu;
+                    const uint32_t bsel = decide_block(R, e43[c], e52[c], 0u, sc[c] >> 31, 0u, 0xFFFFu, (uint32_t)t.vrows);
+                    if (R.sel) R.sel[blk0 + c] = (uint8_t)bsel;
+                    if (R.scale_e8m0) R.scale_e8m0[blk0 + c] = (uint8_t)(s4b >> 23);
+                    if (R.scale_f32) R.scale_f32[blk0 + c] = __uint_as_float(s4b);
+                    n4 += bsel == MOR_FMT_E4M3; n5 += bsel == MOR_FMT_E5M2; nb += bsel == MOR_FMT_BF16;
+                }
+                double s43 = (double)((e43[0] + e43[1]) + (e43[2] + e43[3])), s52 = (double)((e52[0] + e52[1]) + (e52[2] + e52[3]));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
+                n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
+                n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
+                nb = __reduce_add_sync(0xFFFFFFFFu, nb);
+                const uint32_t tnonf = __reduce_add_sync(0xFFFFFFFFu, lane < kComputeWarps ? C.colnonf[b][lane] : 0u);
+                if (lane == 0) {
+                    Partial P;
+                    P.sum43 = s43; P.sum52 = s52; P.nnz = C.colnnz[b]; P.nonfinite = tnonf;
+                    P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = 0xFFFFu;
+                    partials[R.tile_begin + t.local] = P;
+                }
+            } else {
             // the threads' sums in a fixed order: lane-strided in binary32, then a butterfly in double.
             // With 64x64 blocks a lane's entries belong to one column half (lane & 1) and to the upper
             // (k < 4) or lower rows: two sets of sums per lane, combined over the lanes of equal parity.
@@ -986,6 +1068,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 P.sum43 = t43; P.sum52 = t52; P.nnz = tnnz; P.nonfinite = tnonf;
                 P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = mn;
                 partials[R.tile_begin + t.local] = P;
+            }
             }
             if (codes_wait) {
                 // three formats, 128x128 blocks: the compute threads put the chosen format's codes in place
@@ -1211,7 +1294,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         uint32_t key = 0u, prep = 0u;
         if (!SCAN) {
             // the pre-pass left the block's (1x128) or the tile's amax and smallest non-zero; the load warp made the scale
-            const uint32_t e = (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)row * 4u : (uint32_t)q * 4u;
+            const uint32_t e = (KIND == KIND_ROW128 || KIND == KIND_COL128 || KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)row * 4u : (uint32_t)q * 4u;
             if (kNeedKey) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(key) : "r"(keys_base + s * (uint32_t)(kRowKeyStride * 4) + e));
             asm volatile("ld.shared.u32 %0, [%1];" : "=r"(prep) : "r"(prep_base + s * (uint32_t)(kTileRows * 4) + e));
         }
@@ -1444,6 +1527,336 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     }
 }
 
+// ------------------------------------------------------------------ blocks along the columns, prepared scales ----
+
+// Four rows of two neighbouring columns (w[i]: the pair's word of row i), each column with its own scale (packed in
+// s2): the fast conversion of convert_quad_fast with the cast pairing rows of one column, so that a column's four
+// codes come out as one word in memory order of the transposed code tile.  Column c of the pair adds into a43[c],
+// a52[c] and leaves its codes in c4[c] (and its E5M2 codes in c5[c]).
+template <bool YARD>
+__device__ __forceinline__ void convert_colpair_fast(const uint32_t (&w)[4], unsigned long long s2, unsigned long long tiny2,
+                                                     float* a43, float* a52, uint32_t* c4, uint32_t* c5)
+{
+    unsigned long long y2[4];
+    float y[4][2], r[4][2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float x0, x1, u0, u1;
+        unpack_bf16x2(w[i], x0, x1);
+        const unsigned long long x2 = pack_f32x2(x0, x1);
+        y2[i] = mul_f32x2(x2, s2);
+        unpack_f32x2(y2[i], y[i][0], y[i][1]);
+        unpack_f32x2(fma_f32x2(x2, s2, tiny2), u0, u1);
+        r[i][0] = rcp_ftz(u0);
+        r[i][1] = rcp_ftz(u1);
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        uint32_t qa, qb;
+        float d0, d1, d2, d3;
+        cast4_e4m3(y[0][c], y[1][c], y[2][c], y[3][c], c4[c], qa, qb);
+        diff_f16x2_f32(qa, y[0][c], y[1][c], d0, d1);
+        diff_f16x2_f32(qb, y[2][c], y[3][c], d2, d3);
+        a43[c] = fmaf(fabsf(d0), fabsf(r[0][c]), a43[c]);
+        a43[c] = fmaf(fabsf(d1), fabsf(r[1][c]), a43[c]);
+        a43[c] = fmaf(fabsf(d2), fabsf(r[2][c]), a43[c]);
+        a43[c] = fmaf(fabsf(d3), fabsf(r[3][c]), a43[c]);
+    }
+    if (YARD) {
+        // (as in convert_quad_fast: the E5M2 scale is 2^7 times the E4M3 scale, so z = 128 y exactly)
+        const unsigned long long k128 = pack_f32x2(128.0f, 128.0f);
+        float z[4][2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) unpack_f32x2(mul_f32x2(y2[i], k128), z[i][0], z[i][1]);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            uint32_t qa, qb;
+            float d0, d1, d2, d3;
+            cast4_e5m2(z[0][c], z[1][c], z[2][c], z[3][c], c5[c], qa, qb);
+            diff_f16x2_f32(qa, z[0][c], z[1][c], d0, d1);
+            diff_f16x2_f32(qb, z[2][c], z[3][c], d2, d3);
+            a52[c] = fmaf(fabsf(d0), fabsf(r[0][c]), a52[c]);
+            a52[c] = fmaf(fabsf(d1), fabsf(r[1][c]), a52[c]);
+            a52[c] = fmaf(fabsf(d2), fabsf(r[2][c]), a52[c]);
+            a52[c] = fmaf(fabsf(d3), fabsf(r[3][c]), a52[c]);
+        }
+    } else {
+        c5[0] = c5[1] = 0u;
+    }
+}
+
+// Careful path for 16 rows of one column (NaN/inf, scaled values below binary32's normal range, capped E5M2
+// exponent): the elements are gathered with 16-bit loads, two rows to a word, and go through
+// convert_pair_careful.  `a`: shared-memory address of the column's first element.  Returns the column's sums
+// and its 16 codes; adds its NaN/inf elements to `nonfinite`.
+template <bool YARD>
+__device__ __noinline__ void convert_col_careful(uint32_t a, uint32_t s4b, uint32_t s5b, float& e43, float& e52, uint4& codes, uint32_t& nonfinite)
+{
+    CarefulAcc A;
+    A.a43 = A.a52 = 0.0f;
+    A.nnz = A.nbig = A.nonfinite = 0u;
+    uint32_t c[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        uint32_t lo, hi, c5;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(a + (uint32_t)(2 * k * 256)));
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(a + (uint32_t)((2 * k + 1) * 256)));
+        convert_pair_careful<YARD>(__byte_perm(lo, hi, 0x5410), __uint_as_float(s4b), __uint_as_float(s5b), A, c[k], c5);
+    }
+    codes = make_uint4(__byte_perm(c[0], c[1], 0x5410), __byte_perm(c[2], c[3], 0x5410),
+                       __byte_perm(c[4], c[5], 0x5410), __byte_perm(c[6], c[7], 0x5410));
+    const float ratio = __uint_as_float((127u - ((s5b >> 23) - (s4b >> 23))) << 23);   // scale4 / scale5
+    const float tiny = (float)(A.nnz - A.nbig);
+    e43 = A.a43 + tiny;
+    e52 = YARD ? A.a52 * ratio + tiny : 0.0f;
+    nonfinite += A.nonfinite;
+}
+
+// 128x1 blocks with keys from the pre-pass, plain outputs, two formats.  The tile is taken in its row-major order
+// with full-width loads instead of a 16-bit gather: a thread owns four neighbouring columns (one 8-byte piece of
+// each row) over 16 rows, i.e. 16 elements of four different blocks, each block with its own prepared scale.  The
+// cast pairs rows of one column, so a column's 16 codes are 16 contiguous bytes of the transposed code tile.
+//   thread (warp wp, lane l):  columns 4 qc .. 4 qc + 3 with qc = (l & 15) + 16 (wp & 1),
+//                              rows 16 g .. 16 g + 15 with g = ((l & 7) + 2 (wp >> 1) + (l >> 4)) & 7.
+// A half-warp's 8-byte loads cover 128 contiguous bytes of a row each (rows differ between lanes, their pitch is a
+// multiple of all banks); the eight lanes of a 16-byte store phase have eight different g, i.e. all banks once.
+// Lanes l and l ^ 16 hold the same columns: they add their sums, and lane l < 16 hands the four columns' sums to
+// the store warp as part wp >> 1 of four (entry area: [part][column] {E4M3 sum, E5M2 sum}); the store warp adds
+// the parts in order, decides the 128 blocks and writes their metadata (store_warp, COLFAST).
+// One tile of that path.  `pw`: the four columns' prepared words; `careful`: the tile takes the careful path;
+// s, b: stage and staging buffer; n2: how many tiles have used staging buffer b before.
+struct ColsFastThread {
+    int lane, wp, qc;
+    uint32_t in_off, out_off;
+    __device__ __forceinline__ ColsFastThread(int tid)
+    {
+        lane = tid & 31; wp = tid >> 5;
+        qc = (lane & 15) + 16 * (wp & 1);
+        const int g = ((lane & 7) + 2 * (wp >> 1) + (lane >> 4)) & 7;
+        in_off = (uint32_t)(g * 16 * 256 + qc * 8);
+        out_off = (uint32_t)(qc * 4 * 128 + g * 16);
+    }
+};
+
+template <bool YARD, bool STORE>
+__device__ __forceinline__ void cols_fast_tile(const MainParams& p, Control& C, const ColsFastThread& T, uint32_t in_base, uint32_t out_base,
+                                               uint4 pw, bool careful, uint32_t tile_nnz, uint32_t s, uint32_t b, uint32_t n2, bool& dead)
+{
+    const int lane = T.lane, wp = T.wp, qc = T.qc;
+    const uint32_t s4b[4] = {pw.x & 0x7FFFFFFFu, pw.y & 0x7FFFFFFFu, pw.z & 0x7FFFFFFFu, pw.w & 0x7FFFFFFFu};
+    // ---- staging buffer and entries of the tile that used them before must have been consumed ----
+    if (n2 > 0 && !dead) {
+        bool ok = mbar_wait(&C.out_empty[b], (n2 - 1) & 1u, &C.abort, p.wait_cycles);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+    }
+    const uint32_t a = in_base + s * kInBytes + T.in_off;
+    const uint32_t oa = out_base + b * kOutBytes + T.out_off;
+    if (!dead) {
+        float e43[4] = {0.0f, 0.0f, 0.0f, 0.0f}, e52[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        uint32_t nonf = 0u;
+        if (!careful) {
+            const unsigned long long tiny2 = pack_f32x2(FLT_MIN, FLT_MIN);
+            const unsigned long long sa = pack_f32x2(__uint_as_float(s4b[0]), __uint_as_float(s4b[1]));
+            const unsigned long long sb = pack_f32x2(__uint_as_float(s4b[2]), __uint_as_float(s4b[3]));
+            uint32_t cw[4][4];                       // [column][group of four rows]
+#pragma unroll
+            for (int grp = 0; grp < 4; ++grp) {
+                uint32_t wa[4], wb[4], c4[4], c5[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint2 v = lds64(a + (uint32_t)((4 * grp + i) * 256));
+                    wa[i] = v.x; wb[i] = v.y;
+                }
+                if (grp == 3) stage_free_arrive(s);
+                convert_colpair_fast<YARD>(wa, sa, tiny2, &e43[0], &e52[0], &c4[0], &c5[0]);
+                convert_colpair_fast<YARD>(wb, sb, tiny2, &e43[2], &e52[2], &c4[2], &c5[2]);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) cw[c][grp] = c4[c];
+            }
+            if (STORE) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) sts128(oa + (uint32_t)(c * 128), make_uint4(cw[c][0], cw[c][1], cw[c][2], cw[c][3]));
+            }
+            if (YARD) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) e52[c] *= 0.0078125f;   // the factor 1/128 of the E5M2 terms, once per column
+            }
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t sc = c == 0 ? s4b[0] : c == 1 ? s4b[1] : c == 2 ? s4b[2] : s4b[3];
+                const uint32_t s5 = (min((sc >> 23) + 7u, 254u) << 23) | (sc & 0x7FFFFFu);
+                float x43, x52;
+                uint4 codes;
+                convert_col_careful<YARD>(a + (uint32_t)(2 * c), sc, s5, x43, x52, codes, nonf);
+                if (STORE) sts128(oa + (uint32_t)(c * 128), codes);
+                if (c == 0) { e43[0] = x43; e52[0] = x52; }
+                if (c == 1) { e43[1] = x43; e52[1] = x52; }
+                if (c == 2) { e43[2] = x43; e52[2] = x52; }
+                if (c == 3) { e43[3] = x43; e52[3] = x52; }
+            }
+            stage_free_arrive(s);
+        }
+        // ---- the sums of lanes l and l ^ 16 (same columns, neighbouring row groups), handed on by lane l < 16 ----
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            e43[c] += __shfl_xor_sync(0xFFFFFFFFu, e43[c], 16);
+            e52[c] += __shfl_xor_sync(0xFFFFFFFFu, e52[c], 16);
+        }
+        nonf = __reduce_add_sync(0xFFFFFFFFu, nonf);
+        if (lane < 16) {
+            const uint32_t ea = smem_addr(&C.entry[b][0]) + (uint32_t)(wp >> 1) * 1024u + (uint32_t)qc * 32u;
+            sts128(ea, make_uint4(__float_as_uint(e43[0]), __float_as_uint(e52[0]), __float_as_uint(e43[1]), __float_as_uint(e52[1])));
+            sts128(ea + 16u, make_uint4(__float_as_uint(e43[2]), __float_as_uint(e52[2]), __float_as_uint(e43[3]), __float_as_uint(e52[3])));
+            if (wp < 2) sts128(smem_addr(&C.colscale[b][0]) + (uint32_t)qc * 16u, pw);      // one thread per four columns
+        }
+        if (lane == 0) C.colnonf[b][wp] = nonf;
+        if (wp == 0 && lane == 0) C.colnnz[b] = tile_nnz;
+        if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
+    } else {
+        stage_free_arrive(s);                       // given up: the arrival that the conversion would have made
+    }
+    out_full_arrive(b);
+}
+
+template <bool YARD, bool STORE>
+__device__ __forceinline__ void compute_cols_fast(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
+{
+    const ColsFastThread T(tid);
+    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out);
+    const uint32_t meta_base = smem_addr(&C.meta[0]), prep_base = smem_addr(&C.prep[0][0]), flag_base = smem_addr(&C.colflag[0]);
+    bool dead = false;
+    const uint32_t n_it = my_tile_count(p);
+#pragma unroll 1
+    for (uint32_t it = 0; it < n_it; ++it) {
+        const uint32_t s = it % kStages;
+        if (!dead) {
+            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort, p.wait_cycles);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { dead = true; if (T.lane == 0) give_up(C, p.device_status); }
+        }
+        // prepared by the load warp: the four columns' scales (bit 31: NaN or inf in the column piece), whether the
+        // tile takes the careful path, and the tile's count of finite non-zeros
+        const uint4 pw = lds128(prep_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)T.qc * 16u);
+        uint32_t careful, tile_nnz = 0u;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(careful) : "r"(flag_base + s * 4u));
+        if (tid == 0) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tile_nnz) : "r"(meta_base + s * (uint32_t)sizeof(TileMeta) + 28u));
+        cols_fast_tile<YARD, STORE>(p, C, T, in_base, out_base, pw, careful != 0u, tile_nnz, s, it & 1u, it >> 1, dead);
+    }
+}
+
+// Rows and columns of the same tensors from one read, keys of both directions from the pre-pass, two formats, plain
+// outputs.  Per tile the rows' conversion streams from the stage exactly as the 1x128 path does (prepared row
+// scales), then the columns' conversion takes the stage as compute_cols_fast does (prepared column scales) and
+// hands it back.  Staging buffer 0 and its entries serve the rows, buffer 1 the columns.
+template <bool YARD>
+__device__ __forceinline__ void compute_dual_fast(const MainParams& p, Control& C, unsigned char* in, unsigned char* out, int tid)
+{
+    const ColsFastThread T(tid);
+    const int lane = tid & 31;
+    const int row = tid >> 1, h = tid & 1;
+    const int swz = (row & 7) ^ (h << 2);
+    const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
+    const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
+    const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
+    const uint32_t meta_base = smem_addr(&C.meta[0]), prep_base = smem_addr(&C.prep[0][0]), prep2_base = smem_addr(&C.prep2[0][0]);
+    const uint32_t flag_base = smem_addr(&C.colflag[0]);
+    bool dead = false;
+    const uint32_t n_it = my_tile_count(p);
+#pragma unroll 1
+    for (uint32_t it = 0; it < n_it; ++it) {
+        const uint32_t s = it % kStages;
+        if (!dead) {
+            bool ok = mbar_wait(&C.full[s], (it / kStages) & 1u, &C.abort, p.wait_cycles);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+        }
+        TileMeta m;
+        {
+            const uint4 q0 = lds128(meta_base + s * (uint32_t)sizeof(TileMeta));
+            m.ti = dead ? 0 : (int32_t)q0.x; m.vrows = (int32_t)q0.y; m.vcols = (int32_t)q0.z; m.blk_base = q0.w;
+        }
+        uint32_t tile_nnz = 0u;
+        if (tid == 0) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tile_nnz) : "r"(meta_base + s * (uint32_t)sizeof(TileMeta) + 28u));
+
+        // ---- rows (record ti): the streaming 1x128 path ----
+        {
+            const TensorRec& R = p.b.t[m.ti];
+            uint32_t prep;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(prep) : "r"(prep_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)row * 4u));
+            const uint32_t s4b = prep & 0x7FFFFFFFu;
+            const uint32_t s5b = (min((s4b >> 23) + 7u, 254u) << 23) | (s4b & 0x7FFFFFu);
+            const bool careful = (prep >> 31) != 0u;
+            if (it > 0 && !dead) {
+                bool ok = mbar_wait(&C.out_empty[0], (it - 1) & 1u, &C.abort, p.wait_cycles);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) { dead = true; if (lane == 0) give_up(C, p.device_status); }
+            }
+            const uint32_t oa = out_base + out_off;
+            if (!dead) {
+                const uint32_t a = in_base + s * kInBytes + in_off;
+                float e43, e52;
+                uint32_t nnz, nonf;
+                ConvAcc acc;
+                conv_init(acc);
+                if (careful) {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t wh[16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 v = lds128(a ^ ((4 * half + j) << 4));
+                            wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
+                        }
+                        convert_chunks<YARD, true, true, 4, false, false>(wh, oa, 4 * half, s4b, s5b, acc, a);
+                    }
+                    conv_finish<YARD, true, false>(acc, s4b, s5b, e43, e52, nnz, nonf);
+                } else {
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t wh[16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 v = lds128(a ^ ((4 * half + j) << 4));
+                            wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
+                        }
+                        convert_chunks<YARD, false, true, 4, false, false>(wh, oa, 4 * half, s4b, s5b, acc, a);
+                    }
+                    conv_finish<YARD, false, false>(acc, s4b, s5b, e43, e52, nnz, nonf);
+                }
+                if (tid == 0) nnz = tile_nnz;            // the tile's count from the pre-pass, handed on in this thread's entry
+                e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
+                e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
+                uint32_t nz = nnz | (nonf << 16);
+                nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
+                const bool valid = row < m.vrows;
+                const uint32_t sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, 0u, 0xFFFFu, (uint32_t)m.vcols);
+                if (h == 0) {
+                    sts128(entry_base + (uint32_t)row * 16u,
+                           make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (0xFFFFu << 16)));
+                    if (valid) {
+                        const uint32_t blk = m.blk_base + (uint32_t)row * R.nbc;
+                        if (R.sel) R.sel[blk] = (uint8_t)sel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(s4b >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(s4b);
+                    }
+                }
+                fence_async_smem();                      // the codes must be visible to the TMA store
+            }
+            out_full_arrive(0);
+        }
+
+        // ---- columns (record ti + 1): the full-width column path; the stage goes back after its loads ----
+        {
+            const uint4 pw = lds128(prep2_base + s * (uint32_t)(kTileCols * 4) + (uint32_t)T.qc * 16u);
+            uint32_t careful;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(careful) : "r"(flag_base + s * 4u));
+            cols_fast_tile<YARD, true>(p, C, T, in_base, out_base, pw, careful != 0u, tile_nnz, s, 1u, it, dead);
+        }
+    }
+}
+
 // ------------------------------------------------------------------ both directions from one read ----
 
 // KIND_DUAL: the tensor is wanted with 1x128 blocks and with 128x1 blocks (the two operand layouts of the forward
@@ -1609,12 +2022,17 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     pdl_trigger();
     pdl_wait();
 
+    // 128x1 blocks (alone, or beside the 1x128 blocks of the same tensor) with keys from the pre-pass, two formats,
+    // plain outputs: the full-width column path
+    constexpr bool kColFast = (KIND == KIND_COL128 || KIND == KIND_DUAL) && !SCAN && !EXTRA && !THREE;
     if (warp < kComputeWarps) {
-        if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
+        if constexpr (KIND == KIND_DUAL && kColFast) compute_dual_fast<YARD>(p, C, in, out, tid);
+        else if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
+        else if constexpr (kColFast) compute_cols_fast<YARD, STORE>(p, C, in, out, tid);
         else compute_warps<KIND, YARD, THREE, STORE, SCAN, EXTRA>(p, C, in, out, tid);
     }
-    else if (warp == kLoadWarp) load_warp<KIND, !SCAN && KIND != KIND_DUAL && KIND != KIND_COL128>(p, C, in, lane);   // (COLCH: prepared)
-    else store_warp<KIND, THREE, STORE, EXTRA>(p, C, out, partials, lane);
+    else if (warp == kLoadWarp) load_warp<KIND, !SCAN && (KIND != KIND_DUAL || kColFast), kColFast>(p, C, in, lane);
+    else store_warp<KIND, THREE, STORE, EXTRA, kColFast>(p, C, out, partials, lane);
 }
 
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN, bool EXTRA>
