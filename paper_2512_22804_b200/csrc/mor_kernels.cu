@@ -109,26 +109,25 @@ __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __v
 // block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main
 // kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its elements (the key itself
 // covers the finite ones only).
-__global__ void __launch_bounds__(kThreads)
-mor_amax_kernel(const __grid_constant__ BatchParams p)
+struct AmaxShared {
+    uint32_t wkey[kThreads / 32], wnf[kThreads / 32], wnz[kThreads / 32];
+    uint32_t qkey[kThreads / 32][4], qnf[kThreads / 32][4];                   // 64x64 blocks: per warp and quadrant
+    uint32_t cm[kThreads / 32][64], cn[kThreads / 32][64], cf[kThreads / 32][16];   // blocks along the columns
+};
+
+// The work of one CTA on its tile.  EDGE: the tile reaches past the tensor's last row or column (its loads are
+// guarded; a tile inside the tensor takes eight plain 16-byte loads).  The two cases are separate instantiations so
+// that the common one carries nothing of the other.
+template <bool EDGE>
+__device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, long long row0, long long col0, AmaxShared& S)
 {
-    __shared__ uint32_t s_wkey[kThreads / 32], s_wnf[kThreads / 32], s_wnz[kThreads / 32];
-    __shared__ uint32_t s_qkey[kThreads / 32][4], s_qnf[kThreads / 32][4];   // 64x64 blocks: per warp and quadrant
-    __shared__ uint32_t s_cm[kThreads / 32][64], s_cn[kThreads / 32][64], s_cf[kThreads / 32][16];   // per-channel columns
-
-    pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    uint32_t local;
-    const TensorRec& R = p.t[find_tensor(p, blockIdx.x, local)];
-    const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
-    const long long row0 = (long long)bi * kTileRows, col0 = (long long)bj * kTileCols;
-
     uint4 v[8];
     const int k = t & 15;
     const long long first = row0 + (t >> 4);
     const uint16_t* src = R.x + first * R.ld + col0 + 8 * k;
     const long long step = 16 * R.ld;
-    if (row0 + kTileRows <= R.rows && col0 + kTileCols <= R.cols) {
+    if (!EDGE) {
         // a tile inside the tensor: eight 16-byte loads, 16 rows apart
 #pragma unroll
         for (int j = 0; j < 8; ++j, src += step) v[j] = *reinterpret_cast<const uint4*>(src);
@@ -234,7 +233,7 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
                 kq[r] = key_max(kq[r], __shfl_xor_sync(0xFFFFFFFFu, kq[r], o));
                 nq[r] |= __shfl_xor_sync(0xFFFFFFFFu, nq[r], o);
             }
-            if ((lane & 7) == 0 && lane < 16) { s_qkey[warp][2 * r + (lane >> 3)] = kq[r]; s_qnf[warp][2 * r + (lane >> 3)] = nq[r]; }
+            if ((lane & 7) == 0 && lane < 16) { S.qkey[warp][2 * r + (lane >> 3)] = kq[r]; S.qnf[warp][2 * r + (lane >> 3)] = nq[r]; }
         }
     }
     if (col_piece) {
@@ -273,17 +272,17 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
         cf |= __shfl_xor_sync(0xFFFFFFFFu, cf, 16);
         if (lane < 16) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { s_cm[warp][4 * lane + i] = cm[i]; s_cn[warp][4 * lane + i] = cn[i]; }
-            s_cf[warp][lane] = cf;
+            for (int i = 0; i < 4; ++i) { S.cm[warp][4 * lane + i] = cm[i]; S.cn[warp][4 * lane + i] = cn[i]; }
+            S.cf[warp][lane] = cf;
         }
         __syncthreads();
         if (t < kTileCols) {
             const int wd = t >> 1, sh = 16 * (t & 1);
             uint32_t m = 0u, n = 0xFFFFu, f = 0u;
             for (int wp = 0; wp < kThreads / 32; ++wp) {
-                m = max(m, (s_cm[wp][wd] >> sh) & 0xFFFFu);
-                n = min(n, (s_cn[wp][wd] >> sh) & 0xFFFFu);
-                f |= (s_cf[wp][t >> 3] >> (t & 7)) & 1u;
+                m = max(m, (S.cm[wp][wd] >> sh) & 0xFFFFu);
+                n = min(n, (S.cn[wp][wd] >> sh) & 0xFFFFu);
+                f |= (S.cf[wp][t >> 3] >> (t & 7)) & 1u;
             }
             R.col_keys[(size_t)local * kRowKeyStride + t] = (m << 16) | (0xFFFFu - n) | (f << 31);
         }
@@ -291,18 +290,18 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
     nz = __reduce_add_sync(0xFFFFFFFFu, nz);
-    if (lane == 0) { s_wkey[warp] = (hi << 16) | lo; s_wnf[warp] = nf; s_wnz[warp] = nz; }
+    if (lane == 0) { S.wkey[warp] = (hi << 16) | lo; S.wnf[warp] = nf; S.wnz[warp] = nz; }
     __syncthreads();
     if (t == 0) {
-        uint32_t kk = s_wkey[0];
-        for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, s_wkey[i]); nf += s_wnf[i]; nz += s_wnz[i]; }
+        uint32_t kk = S.wkey[0];
+        for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, S.wkey[i]); nf += S.wnf[i]; nz += S.wnz[i]; }
         // finite non-zero elements of the tile (NaN and inf are non-zero patterns: taken off)
         if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)] = nz - nf;
         if (R.col_keys != nullptr && R.col_keys != R.keys) R.col_keys[(size_t)local * kRowKeyStride + kTileRows] = nz - nf;
         if (R.keys != nullptr && R.kind == KIND_BLK64) {
             for (int q = 0; q < 4; ++q) {
-                uint32_t kq = s_qkey[0][q], nq = s_qnf[0][q];
-                for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, s_qkey[i][q]); nq |= s_qnf[i][q]; }
+                uint32_t kq = S.qkey[0][q], nq = S.qnf[0][q];
+                for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, S.qkey[i][q]); nq |= S.qnf[i][q]; }
                 R.keys[(size_t)local * kTileKeyStride + q] = kq | (nq ? 0x80000000u : 0u);
             }
         } else if (R.keys != nullptr && !per_piece && !col_piece) {
@@ -313,6 +312,19 @@ mor_amax_kernel(const __grid_constant__ BatchParams p)
         unsigned int* slot = reinterpret_cast<unsigned int*>(R.amax_slot);
         if (__ldcg(slot) < ((kk >> 16) << 16)) atomicMax(slot, (kk >> 16) << 16);
     }
+}
+
+__global__ void __launch_bounds__(kThreads)
+mor_amax_kernel(const __grid_constant__ BatchParams p)
+{
+    __shared__ AmaxShared S;
+    pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
+    uint32_t local;
+    const TensorRec& R = p.t[find_tensor(p, blockIdx.x, local)];
+    const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
+    const long long row0 = (long long)bi * kTileRows, col0 = (long long)bj * kTileCols;
+    if (row0 + kTileRows <= R.rows && col0 + kTileCols <= R.cols) amax_tile<false>(R, local, row0, col0, S);
+    else amax_tile<true>(R, local, row0, col0, S);
 }
 
 // Per-channel partition: a block is a whole row (a whole column), so its key is the combination of the keys of the
