@@ -183,6 +183,8 @@ bool encode_maps(const mor_tensor_desc_t& d, const mor_outputs_t& o, bool store,
 
 std::atomic<uint32_t> g_test_skip_tile{0xFFFFFFFFu};
 std::atomic<long long> g_test_wait_cycles{kDefaultWaitCycles};
+std::atomic<uint32_t> g_test_skip_pre_tile{0xFFFFFFFFu};
+std::atomic<long long> g_test_pre_wait_cycles{kDefaultWaitCycles};
 
 struct Layout {
     size_t amax_off, status_off, partial_off, keys_off, total;
@@ -312,24 +314,31 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
     if (ev && !record(ev->amax_begin)) return MOR_ERR_CUDA;
     if (cudaMemsetAsync(ws, 0, l.partial_off, stream) != cudaSuccess) return MOR_ERR_CUDA;
     {
-        BatchParams bp;
+        MainParams pre;
+        pre.device_status = reinterpret_cast<uint32_t*>(ws + l.status_off);
+        pre.test_skip_tile = g_test_skip_pre_tile.load(std::memory_order_relaxed);
+        pre.wait_cycles = g_test_pre_wait_cycles.load(std::memory_order_relaxed);
+        BatchParams& bp = pre.b;
         bp.n = 0;
         uint32_t t_end = 0;
         auto flush = [&]() -> bool {
             if (bp.n == 0) return true;
-            bool ok = launch_amax(bp, t_end, stream) == cudaSuccess;
+            pre.total_tiles = t_end;
+            bool ok = launch_amax(pre, stream) == cudaSuccess;
             bool channel = false;
             for (int k = 0; k < bp.n; ++k) channel = channel || bp.t[k].kind == KIND_CHANNEL || bp.t[k].kind == KIND_COLCH;
             if (ok && channel) ok = launch_row_keys(bp, stream) == cudaSuccess;
             bp.n = 0; t_end = 0;
             return ok;
         };
-        for (const Item& it : items) {
+        for (int i = 0; i < n; ++i) {
+            const Item& it = items[i];
             // a supplied group amax only fixes the shared mantissa; the per-tensor partition still
             // needs its block amax, which is the tensor amax, from the data (Algorithm 1)
             if (!it.prepass) continue;
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);
+            pre.in_map[bp.n] = in_maps[i];
             t_end += r.n_tiles;
             bp.tile_end[bp.n++] = t_end;
             if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
@@ -534,8 +543,26 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         if (d.ld % 8 != 0 || !aligned(d.x, 16)) return MOR_ERR_ALIGNMENT;
         if (d.rows != 0 && d.cols != 0 && d.x == nullptr) return MOR_ERR_INVALID_ARG;
     }
+    // the pre-pass reads its tiles with TMA: every descriptor is encoded before anything is enqueued (the encoder
+    // wants a current context, see run())
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaSetDevice(dev) != cudaSuccess) return MOR_ERR_CUDA;
+    }
+    std::vector<CUtensorMap> in_maps((size_t)n);
+    {
+        mor_outputs_t none;
+        std::memset(&none, 0, sizeof(none));
+        CUtensorMap unused;
+        for (int i = 0; i < n; ++i)
+            if (shapes[i].n_tiles && !encode_maps(host_descs[i], none, false, in_maps[i], unused)) return MOR_ERR_CUDA;
+    }
     if (cudaMemsetAsync(ws, 0, l.partial_off, stream) != cudaSuccess) return MOR_ERR_CUDA;
-    BatchParams bp;
+    MainParams pre;
+    pre.device_status = reinterpret_cast<uint32_t*>(ws + l.status_off);
+    pre.test_skip_tile = 0xFFFFFFFFu;
+    pre.wait_cycles = kDefaultWaitCycles;
+    BatchParams& bp = pre.b;
     bp.n = 0;
     uint32_t t_end = 0;
     for (int i = 0; i < n; ++i) {
@@ -548,11 +575,13 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         if (it.s.n_tiles) {
             TensorRec& r = bp.t[bp.n];
             fill_rec(it, ws, l, r);
+            pre.in_map[bp.n] = in_maps[i];
             t_end += r.n_tiles;
             bp.tile_end[bp.n++] = t_end;
         }
         if (bp.n == kMaxBatch || (i == n - 1 && bp.n)) {
-            if (launch_amax(bp, t_end, stream) != cudaSuccess) return MOR_ERR_CUDA;
+            pre.total_tiles = t_end;
+            if (launch_amax(pre, stream) != cudaSuccess) return MOR_ERR_CUDA;
             bp.n = 0; t_end = 0;
         }
     }
@@ -658,6 +687,12 @@ void mor_test_skip_tile_load(uint32_t tile, long long wait_cycles)
 {
     g_test_skip_tile.store(tile, std::memory_order_relaxed);
     g_test_wait_cycles.store(tile == 0xFFFFFFFFu || wait_cycles <= 0 ? kDefaultWaitCycles : wait_cycles, std::memory_order_relaxed);
+}
+
+void mor_test_skip_prepass_tile_load(uint32_t tile, long long wait_cycles)
+{
+    g_test_skip_pre_tile.store(tile, std::memory_order_relaxed);
+    g_test_pre_wait_cycles.store(tile == 0xFFFFFFFFu || wait_cycles <= 0 ? kDefaultWaitCycles : wait_cycles, std::memory_order_relaxed);
 }
 
 const char* mor_status_string(mor_status_t status)

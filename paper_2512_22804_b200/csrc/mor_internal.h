@@ -13,6 +13,8 @@
 // `tile` (numbered within each launch) and give up waiting after `wait_cycles` clock cycles; every such call then
 // reports MOR_ERR_TIMEOUT in mor_tensor_stats_t.status.  tile = 0xFFFFFFFF switches the hook off again.
 extern "C" MOR_API void mor_test_skip_tile_load(uint32_t tile, long long wait_cycles);
+// The same for the amax pre-pass (tiles numbered within each of its launches).
+extern "C" MOR_API void mor_test_skip_prepass_tile_load(uint32_t tile, long long wait_cycles);
 
 namespace mor {
 
@@ -146,7 +148,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 }
 #endif
 
-cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s);
+cudaError_t launch_amax(const MainParams& p, cudaStream_t s);   // records, input tensor maps, tile count, status word, wait limit
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);      // per-channel: keys of whole rows / whole columns
 cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, int kind, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);

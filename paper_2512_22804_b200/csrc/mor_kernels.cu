@@ -1,11 +1,16 @@
 // The two small kernels around the fused main kernel (mor_main.cu).
 //
 //   mor_amax_kernel      Algorithm 1, first step: the largest magnitude of the group, the tensor being one group
+//                        (persistent, TMA-fed); it also leaves the block keys and non-zero counts of every tile
 //   mor_finalise_kernel  tensor-wide aggregate of the per-tile partials and the Eq. 2 decision
 #include <cuda_bf16.h>
 #include <float.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "mor_internal.h"
+#include "mor_ptx.cuh"
 
 namespace mor {
 namespace {
@@ -77,15 +82,18 @@ __device__ __forceinline__ float minnz_value(uint32_t minm1_bits)
 
 // Key of 8 elements (four packed BF16 pairs): amax bits << 16 | 0xFFFF - (smallest non-zero bits - 1),
 // so that keys combine with a packed 16-bit maximum.  NaN and inf compare above every finite pattern.
-__device__ __forceinline__ uint32_t key_of_chunk(uint4 v)
+__device__ __forceinline__ uint32_t key_of_masked(uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3)
 {
-    const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
     const uint32_t mx = __vimax3_u16x2(__vimax3_u16x2(a0, a1, a2), a3, a3);
     uint32_t mn = __viaddmin_u16x2(a0, 0xFFFFFFFFu, 0xFFFFFFFFu);
     mn = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn);
     mn = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn);
     mn = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn);
     return (max(mx & 0xFFFFu, mx >> 16) << 16) | (0xFFFFu - min(mn & 0xFFFFu, mn >> 16));
+}
+__device__ __forceinline__ uint32_t key_of_chunk(uint4 v)
+{
+    return key_of_masked(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu, v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu);
 }
 // the same over finite elements only, with the count of the others (a real call: rare path)
 __device__ __noinline__ uint2 key_of_chunk_finite(uint4 v)
@@ -109,69 +117,74 @@ __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __v
 // block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main
 // kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its elements (the key itself
 // covers the finite ones only).
+// What the load warp tells the other warps about the tile in a stage (and, copied into the scratch, the tail warp).
+constexpr uint32_t kModeKeys = 1u;        // the record wants keys (and the tile's count of non-zeros)
+constexpr uint32_t kModePerPiece = 2u;    // ... one per row piece
+constexpr uint32_t kModeColPiece = 4u;    // ... one per column piece
+constexpr uint32_t kModeBlk64 = 8u;       // ... one per 64x64 quadrant
+constexpr uint32_t kModeColsApart = 16u;  // the column keys have an area of their own (rows and columns from one pre-pass)
+struct __align__(16) AmaxMeta {
+    int32_t ti;                // tensor index within the launch
+    uint32_t local;            // tile index within the tensor
+    uint32_t mode;
+    uint32_t key_stride;
+    uint32_t* keys;
+    uint32_t* col_keys;
+};
+static_assert(sizeof(AmaxMeta) == 32, "two 16-byte loads");
+
 struct AmaxShared {
+    AmaxMeta meta;
     uint32_t wkey[kThreads / 32], wnf[kThreads / 32], wnz[kThreads / 32];
     uint32_t qkey[kThreads / 32][4], qnf[kThreads / 32][4];                   // 64x64 blocks: per warp and quadrant
     uint32_t cm[kThreads / 32][64], cn[kThreads / 32][64], cf[kThreads / 32][16];   // blocks along the columns
 };
 
-// The work of one CTA on its tile.  EDGE: the tile reaches past the tensor's last row or column (its loads are
-// guarded; a tile inside the tensor takes eight plain 16-byte loads).  The two cases are separate instantiations so
-// that the common one carries nothing of the other.
-template <bool EDGE>
-__device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, long long row0, long long col0, AmaxShared& S)
+// Hand-off between the 256 compute threads and the tail warp on hardware barriers (a thread asleep there takes no
+// issue slots): "scratch b is complete" (compute threads announce, the tail warp sleeps) and "scratch b has been
+// read" (the tail warp announces, compute threads wait -- normally long past).
+__device__ __forceinline__ void scratch_full_arrive(uint32_t b) { asm volatile("barrier.cta.arrive %0, %1;" ::"r"(2u + b), "n"(kThreads + 32) : "memory"); }
+__device__ __forceinline__ void scratch_full_sync(uint32_t b) { asm volatile("barrier.cta.sync %0, %1;" ::"r"(2u + b), "n"(kThreads + 32) : "memory"); }
+__device__ __forceinline__ void scratch_free_arrive(uint32_t b) { asm volatile("barrier.cta.arrive %0, %1;" ::"r"(4u + b), "n"(kThreads + 32) : "memory"); }
+__device__ __forceinline__ void scratch_free_sync(uint32_t b) { asm volatile("barrier.cta.sync %0, %1;" ::"r"(4u + b), "n"(kThreads + 32) : "memory"); }
+
+// The work of a compute thread on one tile whose data it holds in registers: thread t has the 16-byte chunk
+// (t & 15) of rows (t >> 4) + 16 j, j = 0..7 (zeros past the tensor's edge).  Keys of row pieces are complete within
+// a warp and written from here; everything that spans warps (tile key, quadrant keys, column keys, counts, the
+// tensor amax) is left per warp in the scratch `S` for the tail warp.  `dead`: a bounded wait has run out in this
+// warp -- its data are zeros and it writes no keys, but keeps its part in the hand-off.
+__device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 (&v)[8], AmaxShared& S)
 {
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    uint4 v[8];
     const int k = t & 15;
-    const long long first = row0 + (t >> 4);
-    const uint16_t* src = R.x + first * R.ld + col0 + 8 * k;
-    const long long step = 16 * R.ld;
-    if (!EDGE) {
-        // a tile inside the tensor: eight 16-byte loads, 16 rows apart
-#pragma unroll
-        for (int j = 0; j < 8; ++j, src += step) v[j] = *reinterpret_cast<const uint4*>(src);
-    } else {
-        const long long left = R.cols - col0 - 8 * k;       // elements of this thread's 16-byte chunk inside the tensor
-        const int nrows = (int)((R.rows - first + 15) >> 4); // this thread's rows (first, first + 16, ...) inside the tensor
-#pragma unroll
-        for (int j = 0; j < 8; ++j, src += step) {
-            v[j] = make_uint4(0u, 0u, 0u, 0u);
-            if (j < nrows) {
-                if (left >= 8) {
-                    v[j] = *reinterpret_cast<const uint4*>(src);
-                } else if (left > 0) {
-                    uint16_t e[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-                    for (int i = 0; i < (int)left; ++i) e[i] = src[i];
-                    v[j] = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
-                                      e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
-                }
-            }
-        }
-    }
-    const bool col_piece = R.col_keys != nullptr;            // blocks along the columns: one key per column piece of the tile
-    const bool per_piece = R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && R.col_keys != R.keys;
+    const uint32_t local = M.local;
+    const bool has_keys = (M.mode & kModeKeys) != 0u;
+    const bool col_piece = (M.mode & kModeColPiece) != 0u;
+    const bool per_piece = (M.mode & kModePerPiece) != 0u;
     uint32_t key[8], all = 0u, nf = 0u;
-    // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once.  The
-    // main kernel takes the tile's count from here and need not count while it converts.
+    // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once (on the
+    // words already masked for the keys).  The main kernel takes the tile's count from here and need not count while
+    // it converts.
     uint32_t nz2 = 0u;
-    if (R.keys != nullptr) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            nz2 += __vimin3_u16x2(v[j].x & 0x7FFF7FFFu, 0x00010001u, 0x00010001u) + __vimin3_u16x2(v[j].y & 0x7FFF7FFFu, 0x00010001u, 0x00010001u);
-            nz2 += __vimin3_u16x2(v[j].z & 0x7FFF7FFFu, 0x00010001u, 0x00010001u) + __vimin3_u16x2(v[j].w & 0x7FFF7FFFu, 0x00010001u, 0x00010001u);
-        }
-    }
-    uint32_t nz = (nz2 & 0xFFFFu) + (nz2 >> 16);
     if (per_piece) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { key[j] = key_of_chunk(v[j]); all = key_max(all, key[j]); }
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
+            nz2 += __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
+            nz2 += __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+            key[j] = key_of_masked(a0, a1, a2, a3);
+            all = key_max(all, key[j]);
+        }
     } else {
         // one key for the thread's 64 elements: packed halves are folded once at the end
         uint32_t mx = 0u, mn[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
+            if (has_keys) {
+                nz2 += __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
+                nz2 += __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+            }
             mx = __vimax3_u16x2(__vimax3_u16x2(mx, a0, a1), a2, a3);
             mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
             mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
@@ -182,6 +195,7 @@ __device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, lo
         const uint32_t m2 = __vimin3_u16x2(mn[0], mn[1], mn[1]);
         all = (max(mx & 0xFFFFu, mx >> 16) << 16) | (0xFFFFu - min(m2 & 0xFFFFu, m2 >> 16));
     }
+    uint32_t nz = (nz2 & 0xFFFFu) + (nz2 >> 16);
     // NaN or inf somewhere in the warp's data: redo the keys over finite elements and count the others
     const bool warp_nf = __any_sync(0xFFFFFFFFu, (all >> 16) >= kBf16Inf);
     uint32_t nf_piece = 0u;                                  // bit j: this thread saw NaN/inf in its chunk of piece j
@@ -199,7 +213,7 @@ __device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, lo
     if (per_piece) {
         // one key per row piece: combine the 16 lanes that share the piece
         const uint32_t half = (lane & 16) ? 0xFFFF0000u : 0x0000FFFFu;
-        uint32_t* kp = R.keys + (size_t)local * kRowKeyStride + (t >> 4);
+        uint32_t* kp = M.keys + (size_t)local * kRowKeyStride + (t >> 4);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             uint32_t kk = key[j];
@@ -212,7 +226,7 @@ __device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, lo
             if (k == 0) kp[16 * j] = kk;
         }
     }
-    if (R.keys != nullptr && R.kind == KIND_BLK64) {
+    if ((M.mode & kModeBlk64) != 0u) {
         // one key per 64x64 quadrant: this thread's chunk lies in column half (k >> 3); its first four rows
         // are in the upper half of the tile, the other four in the lower half
         uint32_t kq[2], nq[2] = {0u, 0u};
@@ -275,56 +289,202 @@ __device__ __forceinline__ void amax_tile(const TensorRec& R, uint32_t local, lo
             for (int i = 0; i < 4; ++i) { S.cm[warp][4 * lane + i] = cm[i]; S.cn[warp][4 * lane + i] = cn[i]; }
             S.cf[warp][lane] = cf;
         }
-        __syncthreads();
-        if (t < kTileCols) {
-            const int wd = t >> 1, sh = 16 * (t & 1);
-            uint32_t m = 0u, n = 0xFFFFu, f = 0u;
-            for (int wp = 0; wp < kThreads / 32; ++wp) {
-                m = max(m, (S.cm[wp][wd] >> sh) & 0xFFFFu);
-                n = min(n, (S.cn[wp][wd] >> sh) & 0xFFFFu);
-                f |= (S.cf[wp][t >> 3] >> (t & 7)) & 1u;
-            }
-            R.col_keys[(size_t)local * kRowKeyStride + t] = (m << 16) | (0xFFFFu - n) | (f << 31);
-        }
     }
     const uint32_t hi = __reduce_max_sync(0xFFFFFFFFu, all >> 16), lo = __reduce_max_sync(0xFFFFFFFFu, all & 0xFFFFu);
     nf = __reduce_add_sync(0xFFFFFFFFu, nf);
     nz = __reduce_add_sync(0xFFFFFFFFu, nz);
     if (lane == 0) { S.wkey[warp] = (hi << 16) | lo; S.wnf[warp] = nf; S.wnz[warp] = nz; }
-    __syncthreads();
-    if (t == 0) {
-        uint32_t kk = S.wkey[0];
+    if (t == 0) S.meta = M;
+}
+
+// The tail warp's work on one tile, from the scratch the compute warps left: keys of the columns (four per lane),
+// and by lane 0 the tile's key or quadrant keys, its count of finite non-zeros and the tensor amax.  `seen_ti`,
+// `seen_amax`: lane 0 remembers the largest amax it has sent for the tensor it is on, so that the atomic goes out
+// only when a tile raises it.
+__device__ __forceinline__ void amax_tail(const BatchParams& bp, const AmaxShared& S, int lane, int& seen_ti, uint32_t& seen_amax)
+{
+    const AmaxMeta M = S.meta;
+    const uint32_t local = M.local;
+    const bool has_keys = (M.mode & kModeKeys) != 0u;
+    const bool col_piece = (M.mode & kModeColPiece) != 0u;
+    const bool per_piece = (M.mode & kModePerPiece) != 0u;
+    if (col_piece) {
+        // columns 4 lane .. 4 lane + 3: two words of two columns each per warp, flags in byte lane >> 1
+        uint32_t m0 = 0u, m1 = 0u, n0 = 0xFFFFFFFFu, n1 = 0xFFFFFFFFu, f = 0u;
+#pragma unroll
+        for (int wp = 0; wp < kThreads / 32; ++wp) {
+            m0 = __vimax3_u16x2(m0, S.cm[wp][2 * lane], S.cm[wp][2 * lane]);
+            m1 = __vimax3_u16x2(m1, S.cm[wp][2 * lane + 1], S.cm[wp][2 * lane + 1]);
+            n0 = __vimin3_u16x2(n0, S.cn[wp][2 * lane], S.cn[wp][2 * lane]);
+            n1 = __vimin3_u16x2(n1, S.cn[wp][2 * lane + 1], S.cn[wp][2 * lane + 1]);
+            f |= S.cf[wp][lane >> 1];
+        }
+        f >>= 4 * (lane & 1);
+        uint4 kk;
+        kk.x = ((m0 & 0xFFFFu) << 16) | (0xFFFFu - (n0 & 0xFFFFu)) | ((f & 1u) << 31);
+        kk.y = ((m0 >> 16) << 16) | (0xFFFFu - (n0 >> 16)) | (((f >> 1) & 1u) << 31);
+        kk.z = ((m1 & 0xFFFFu) << 16) | (0xFFFFu - (n1 & 0xFFFFu)) | (((f >> 2) & 1u) << 31);
+        kk.w = ((m1 >> 16) << 16) | (0xFFFFu - (n1 >> 16)) | (((f >> 3) & 1u) << 31);
+        *reinterpret_cast<uint4*>(M.col_keys + (size_t)local * kRowKeyStride + 4 * lane) = kk;
+    }
+    if (lane == 0) {
+        uint32_t kk = S.wkey[0], nf = S.wnf[0], nz = S.wnz[0];
+#pragma unroll
         for (int i = 1; i < kThreads / 32; ++i) { kk = key_max(kk, S.wkey[i]); nf += S.wnf[i]; nz += S.wnz[i]; }
         // finite non-zero elements of the tile (NaN and inf are non-zero patterns: taken off)
-        if (R.keys != nullptr) R.keys[(size_t)local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)] = nz - nf;
-        if (R.col_keys != nullptr && R.col_keys != R.keys) R.col_keys[(size_t)local * kRowKeyStride + kTileRows] = nz - nf;
-        if (R.keys != nullptr && R.kind == KIND_BLK64) {
+        if (has_keys) M.keys[(size_t)local * M.key_stride + (M.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)] = nz - nf;
+        if ((M.mode & kModeColsApart) != 0u) M.col_keys[(size_t)local * kRowKeyStride + kTileRows] = nz - nf;
+        if ((M.mode & kModeBlk64) != 0u) {
             for (int q = 0; q < 4; ++q) {
                 uint32_t kq = S.qkey[0][q], nq = S.qnf[0][q];
                 for (int i = 1; i < kThreads / 32; ++i) { kq = key_max(kq, S.qkey[i][q]); nq |= S.qnf[i][q]; }
-                R.keys[(size_t)local * kTileKeyStride + q] = kq | (nq ? 0x80000000u : 0u);
+                M.keys[(size_t)local * kTileKeyStride + q] = kq | (nq ? 0x80000000u : 0u);
             }
-        } else if (R.keys != nullptr && !per_piece && !col_piece) {
-            R.keys[(size_t)local * R.key_stride] = kk | (nf ? 0x80000000u : 0u);
+        } else if (has_keys && !per_piece && !col_piece) {
+            M.keys[(size_t)local * M.key_stride] = kk | (nf ? 0x80000000u : 0u);
         }
         // non-negative binary32 patterns order like the values
-        // (atomics on one address are served one at a time: read first, most tiles end there)
-        unsigned int* slot = reinterpret_cast<unsigned int*>(R.amax_slot);
-        if (__ldcg(slot) < ((kk >> 16) << 16)) atomicMax(slot, (kk >> 16) << 16);
+        const uint32_t amax_bits = (kk >> 16) << 16;
+        if (M.ti != seen_ti) { seen_ti = M.ti; seen_amax = 0u; }
+        if (amax_bits > seen_amax) {
+            seen_amax = amax_bits;
+            atomicMax(reinterpret_cast<unsigned int*>(bp.t[M.ti].amax_slot), amax_bits);
+        }
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
-mor_amax_kernel(const __grid_constant__ BatchParams p)
+// The pre-pass kernel: persistent CTAs (two per SM) of 8 compute warps, a load warp and a tail warp.  One thread of
+// the load warp streams the CTA's tiles (tile numbers blockIdx.x, + gridDim.x, ...) through a ring of three 32 KiB
+// stages with TMA tile loads (zero fill past the tensor's edge), so that up to six tiles per SM are in flight
+// whatever the compute warps are doing; a compute thread copies its eight 16-byte chunks of a landed tile to
+// registers, the warp hands the stage back, reduces from the registers and leaves its results in one of two
+// scratch areas; the tail warp combines the eight warps' results, writes the keys that span warps and raises the
+// tensor amax, off the compute warps' path.  Every mbarrier wait is bounded; a wait that runs out sets the status
+// word that the finalise kernel reports, and from then on the tail warp writes nothing.
+constexpr int kAmaxStages = 3;
+constexpr int kAmaxThreads = kThreads + 64;            // 8 compute warps, the load warp, the tail warp
+constexpr int kAmaxStageBytes = kTileRows * kTileCols * 2;
+
+struct AmaxControl {
+    unsigned long long full[kAmaxStages];                // the tile has landed
+    unsigned long long empty[kAmaxStages];               // the compute warps have their copies (one arrival per warp)
+    AmaxMeta meta[kAmaxStages];                          // by the load warp, before the stage's copy is started
+    volatile uint32_t abort;
+    uint32_t issued;
+    AmaxShared S[2];
+};
+constexpr int kAmaxSmemBytes = 1024 + kAmaxStages * kAmaxStageBytes + (int)sizeof(AmaxControl);
+static_assert(2 * (kAmaxSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM must fit in shared memory");
+
+__global__ void __launch_bounds__(kAmaxThreads, 2)
+mor_amax_kernel(const __grid_constant__ MainParams p)
 {
-    __shared__ AmaxShared S;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* in = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    AmaxControl& C = *reinterpret_cast<AmaxControl*>(in + kAmaxStages * kAmaxStageBytes);
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    if (t == 0) {
+        for (int s = 0; s < kAmaxStages; ++s) { mbar_init(&C.full[s], 1); mbar_init(&C.empty[s], kThreads / 32); }
+        C.abort = 0u;
+        C.issued = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
     pdl_trigger();                                       // the main kernel may move in as this kernel's CTAs leave
-    uint32_t local;
-    const TensorRec& R = p.t[find_tensor(p, blockIdx.x, local)];
-    const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
-    const long long row0 = (long long)bi * kTileRows, col0 = (long long)bj * kTileCols;
-    if (row0 + kTileRows <= R.rows && col0 + kTileCols <= R.cols) amax_tile<false>(R, local, row0, col0, S);
-    else amax_tile<true>(R, local, row0, col0, S);
+    const uint32_t n_it = (p.total_tiles - blockIdx.x + gridDim.x - 1u) / gridDim.x;
+
+    if (warp == kThreads / 32) {
+        // ---- load warp: one thread issues, the others leave ----
+        if (lane != 0) return;
+        for (uint32_t it = 0; it < n_it; ++it) {
+            const uint32_t s = it % kAmaxStages, tile = blockIdx.x + it * gridDim.x;
+            if (it >= (uint32_t)kAmaxStages &&
+                !mbar_wait(&C.empty[s], (it / kAmaxStages - 1u) & 1u, &C.abort, p.wait_cycles)) {
+                C.abort = 1u;
+                atomicOr(p.device_status, 1u);
+                break;
+            }
+            uint32_t local;
+            const int ti = find_tensor(p.b, tile, local);
+            const TensorRec& R = p.b.t[ti];
+            const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
+            {
+                AmaxMeta m;
+                m.ti = ti; m.local = local; m.key_stride = R.key_stride; m.keys = R.keys; m.col_keys = R.col_keys;
+                const bool cols = R.col_keys != nullptr;
+                m.mode = (R.keys != nullptr ? kModeKeys : 0u) |
+                         (R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && R.col_keys != R.keys ? kModePerPiece : 0u) |
+                         (cols ? kModeColPiece : 0u) | (R.keys != nullptr && R.kind == KIND_BLK64 ? kModeBlk64 : 0u) |
+                         (cols && R.col_keys != R.keys ? kModeColsApart : 0u);
+                C.meta[s] = m;                           // (made visible by the arrival below)
+            }
+            // (test hook: the load of one chosen tile is left out, so that the waits for it run out)
+            if (tile != p.test_skip_tile) {
+                mbar_arrive_expect_tx(&C.full[s], (uint32_t)kAmaxStageBytes);
+                tma_load_tile(in + s * kAmaxStageBytes, &p.in_map[ti], (int)(bj * kTileCols), (int)(bi * kTileRows), &C.full[s]);
+            }
+            C.issued = it + 1u;
+        }
+        if (C.abort) {
+            // copies that may still be in flight must land (or be given up on) before the CTA goes
+            const uint32_t issued = C.issued;
+            for (uint32_t k = 0; k < (uint32_t)kAmaxStages && k < issued; ++k) {
+                const uint32_t it = issued - 1u - k;
+                mbar_wait(&C.full[it % kAmaxStages], (it / kAmaxStages) & 1u, nullptr, p.wait_cycles);
+            }
+        }
+        return;
+    }
+
+    if (warp == kThreads / 32 + 1) {
+        // ---- tail warp ----
+        int seen_ti = -1;
+        uint32_t seen_amax = 0u;
+#pragma unroll 1
+        for (uint32_t it = 0; it < n_it; ++it) {
+            const uint32_t b = it & 1u;
+            scratch_full_sync(b);
+            if (!C.abort) amax_tail(p.b, C.S[b], lane, seen_ti, seen_amax);
+            __syncwarp();
+            if (it + 2u < n_it) scratch_free_arrive(b);      // (the last two have no taker)
+        }
+        return;
+    }
+
+    // ---- compute warps ----
+    bool dead = false;
+    const uint32_t off = (uint32_t)((t >> 4) * 256 + (t & 15) * 16);
+    const uint32_t in_base = smem_addr(in);
+#pragma unroll 1
+    for (uint32_t it = 0; it < n_it; ++it) {
+        const uint32_t s = it % kAmaxStages, b = it & 1u;
+        if (!dead) {
+            bool ok = mbar_wait(&C.full[s], (it / kAmaxStages) & 1u, &C.abort, p.wait_cycles);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) {
+                dead = true;
+                if (lane == 0) { C.abort = 1u; atomicOr(p.device_status, 1u); }
+            }
+        }
+        uint4 v[8], m0, m1;
+        if (!dead) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = lds128(in_base + s * (uint32_t)kAmaxStageBytes + off + (uint32_t)(j * 16 * 256));
+            m0 = lds128(smem_addr(&C.meta[s]));
+            m1 = lds128(smem_addr(&C.meta[s]) + 16u);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&C.empty[s]);         // this warp's copies are in registers
+        if (it >= 2u) scratch_free_sync(b);              // the tail warp has read what tile it - 2 left in this scratch
+        if (!dead) {
+            AmaxMeta M;
+            M.ti = (int32_t)m0.x; M.local = m0.y; M.mode = m0.z; M.key_stride = m0.w;
+            M.keys = reinterpret_cast<uint32_t*>(((unsigned long long)m1.y << 32) | m1.x);
+            M.col_keys = reinterpret_cast<uint32_t*>(((unsigned long long)m1.w << 32) | m1.z);
+            amax_thread_part(M, v, C.S[b]);
+        }
+        scratch_full_arrive(b);
+    }
 }
 
 // Per-channel partition: a block is a whole row (a whole column), so its key is the combination of the keys of the
@@ -518,10 +678,28 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
 
 }  // namespace
 
-cudaError_t launch_amax(const BatchParams& p, uint32_t total_tiles, cudaStream_t s)
+cudaError_t launch_amax(const MainParams& p, cudaStream_t s)
 {
-    if (total_tiles == 0) return cudaSuccess;
-    mor_amax_kernel<<<total_tiles, kThreads, 0, s>>>(p);
+    if (p.total_tiles == 0) return cudaSuccess;
+    static std::atomic<int> sm_count[64];   // per device; 0 = not set up yet
+    static std::mutex setup;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int sms = sm_count[dev].load(std::memory_order_acquire);
+    if (sms == 0) {
+        std::lock_guard<std::mutex> lock(setup);         // host threads may make their first call together
+        e = cudaFuncSetAttribute(mor_amax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAmaxSmemBytes);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        if (sms <= 0) return cudaErrorInvalidDevice;
+        sm_count[dev].store(sms, std::memory_order_release);
+    }
+    const uint32_t resident = 2u * (uint32_t)sms;
+    const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
+    mor_amax_kernel<<<grid, kAmaxThreads, kAmaxSmemBytes, s>>>(p);
     return cudaGetLastError();
 }
 

@@ -40,6 +40,7 @@
 #include <mutex>
 
 #include "mor_internal.h"
+#include "mor_ptx.cuh"
 
 namespace mor {
 namespace {
@@ -106,70 +107,8 @@ static_assert(offsetof(Control, keys) % 16 == 0 && offsetof(Control, prep) % 16 
               offsetof(Control, prep2) % 16 == 0 && offsetof(Control, colscale) % 16 == 0 && offsetof(Control, wmax) % 16 == 0 &&
               offsetof(Control, meta) % 16 == 0, "16-byte shared-memory accesses");
 
-// ------------------------------------------------------------------ PTX helpers ----
+// (PTX helpers for mbarriers, TMA copies and shared-memory accesses: mor_ptx.cuh)
 
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(void* bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(void* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-// One try: the thread may be suspended by the hardware until the phase completes or a time limit of the
-// implementation's choosing (at most about `hint_ns`) has passed; true when the phase has completed.
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity, uint32_t hint_ns)
-{
-    uint32_t done;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(done) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
-    return done != 0;
-}
-// Keeps trying (a suspended thread takes no issue slots from the warps that compute); gives up after `limit` cycles.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const volatile uint32_t* abort_flag, long long limit)
-{
-    const long long t0 = clock64();
-    for (;;) {
-        if (mbar_try(bar, parity, 20000u)) return true;
-        if (abort_flag != nullptr && *abort_flag) return false;
-        if (clock64() - t0 > limit) return false;
-    }
-}
-// Bounded wait for the phase with the given parity; false when the limit ran out or (with a flag
-// given) another thread of the CTA has given up already.
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, const volatile uint32_t* abort_flag, long long limit)
-{
-    const uint32_t a = smem_addr(bar);
-    if (mbar_try(a, parity, 2000u)) return true;
-    return mbar_wait_slow(a, parity, abort_flag, limit);
-}
-__device__ __forceinline__ void tma_load_tile(void* dst, const CUtensorMap* map, int x, int y, void* bar)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(smem_addr(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar)) : "memory");
-}
-// plain bulk copy global -> shared (16-byte aligned, size a multiple of 16), completing on the same mbarrier
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, void* bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, int x, int y, const void* src)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(smem_addr(src)) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 // barrier over the compute threads that also ORs a predicate
 __device__ __forceinline__ bool compute_bar_or(bool v)
 {
@@ -196,27 +135,6 @@ __device__ __forceinline__ void out_full_arrive(uint32_t b)
 __device__ __forceinline__ void out_full_sync(uint32_t b)
 {
     asm volatile("barrier.cta.sync %0, %1;" ::"r"(kBarOutFull + b), "n"(kThreads + 32) : "memory");
-}
-
-__device__ __forceinline__ uint4 lds128(uint32_t a)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(uint32_t a)
-{
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t a, uint4 v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void sts64(uint32_t a, uint2 v)
-{
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(v.x), "r"(v.y) : "memory");
 }
 
 // {hi, lo} -> two FP8 codes, `lo` in the low byte (round to nearest even, saturate to the largest finite)

@@ -21,8 +21,8 @@ THREE = (mb.MOR_FMT_E4M3, mb.MOR_FMT_E5M2, mb.MOR_FMT_BF16)
 NONE = 0xFFFFFFFF
 
 
-def hook():
-    f = mb.load().mor_test_skip_tile_load
+def hook(name="mor_test_skip_tile_load"):
+    f = getattr(mb.load(), name)
     f.argtypes, f.restype = [C.c_uint32, C.c_longlong], None
     return f
 
@@ -87,3 +87,45 @@ def test_timeout_in_a_paired_rows_and_columns_launch():
     want = mb.analyze_quantize(x, rr)
     torch.cuda.synchronize()
     assert torch.equal(plan.outs[0].codes, want.codes) and torch.equal(plan.outs[0].sel, want.sel)
+
+
+@pytest.mark.parametrize("block,formats", [((128, 128), TWO), ((1, 128), THREE), ((128, 1), TWO), ((0, 1), TWO), ((64, 64), TWO)])
+@pytest.mark.parametrize("tile", [0, 7, 15])
+def test_timeout_in_the_amax_pre_pass(block, formats, tile):
+    """The pre-pass streams its tiles through a ring of stages with TMA loads and bounded waits of its own; the
+    second hook (``mor_test_skip_prepass_tile_load``) leaves one of its loads out.  Its CTA gives up on that tile, the
+    call returns with MOR_ERR_TIMEOUT (the main kernel still runs, on whatever keys there are), and the next call
+    is clean."""
+    import torch
+
+    bits = wl.gradient_like(512, 512, seed=99)
+    x = parity.to_device(bits)
+    crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block == (0, 1) else mb.MOR_CRIT_BLOCK_VS_E5M2
+    r = mb.Recipe(block, formats, crit)
+    set_hook = hook("mor_test_skip_prepass_tile_load")
+    set_hook(tile, 2_000_000)
+    try:
+        out = mb.analyze_quantize(x, r)
+        torch.cuda.synchronize()
+    finally:
+        set_hook(NONE, 0)
+    assert out.tensor_stats_dict()["status"] == mb.MOR_ERR_TIMEOUT
+    parity.run_and_compare(bits, r)
+
+
+def test_timeout_in_the_pre_pass_of_a_cta_with_several_tiles():
+    """More tiles than resident CTAs: the CTA that loses a tile has others before and after it in its ring."""
+    import torch
+
+    bits = wl.weight_like(2560, 2048, seed=100)                       # 320 tiles on at most 296 CTAs
+    x = parity.to_device(bits)
+    r = mb.Recipe((128, 128), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2)
+    set_hook = hook("mor_test_skip_prepass_tile_load")
+    set_hook(3, 2_000_000)
+    try:
+        out = mb.analyze_quantize(x, r)
+        torch.cuda.synchronize()
+    finally:
+        set_hook(NONE, 0)
+    assert out.tensor_stats_dict()["status"] == mb.MOR_ERR_TIMEOUT
+    parity.run_and_compare(bits, r)
