@@ -170,30 +170,34 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
-            nz2 += __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
-            nz2 += __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+            const uint32_t n01 = __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
+            const uint32_t n23 = __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+            nz2 += n01 + n23;
             key[j] = key_of_masked(a0, a1, a2, a3);
             all = key_max(all, key[j]);
         }
     } else {
-        // one key for the thread's 64 elements: packed halves are folded once at the end
-        uint32_t mx = 0u, mn[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+        // one key for the thread's 64 elements: packed halves are folded once at the end; two independent chains of
+        // every running value (even and odd chunks), so that a warp has something to issue while a result is on its way
+        uint32_t mx[2] = {0u, 0u}, mn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu}, nzc[2] = {0u, 0u};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
+            const int c = j & 1;
             const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
             if (has_keys) {
-                nz2 += __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
-                nz2 += __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+                const uint32_t n01 = __vimin3_u16x2(a0, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a1, 0x00010001u, 0x00010001u);
+                const uint32_t n23 = __vimin3_u16x2(a2, 0x00010001u, 0x00010001u) + __vimin3_u16x2(a3, 0x00010001u, 0x00010001u);
+                nzc[c] += n01 + n23;
             }
-            mx = __vimax3_u16x2(__vimax3_u16x2(mx, a0, a1), a2, a3);
-            mn[0] = __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[0]);
-            mn[1] = __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[1]);
-            mn[0] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, mn[0]);
-            mn[1] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, mn[1]);
+            mx[c] = __vimax3_u16x2(mx[c], __vimax3_u16x2(a0, a1, a2), a3);
+            mn[2 * c] = __viaddmin_u16x2(a2, 0xFFFFFFFFu, __viaddmin_u16x2(a0, 0xFFFFFFFFu, mn[2 * c]));
+            mn[2 * c + 1] = __viaddmin_u16x2(a3, 0xFFFFFFFFu, __viaddmin_u16x2(a1, 0xFFFFFFFFu, mn[2 * c + 1]));
             key[j] = 0u;
         }
-        const uint32_t m2 = __vimin3_u16x2(mn[0], mn[1], mn[1]);
-        all = (max(mx & 0xFFFFu, mx >> 16) << 16) | (0xFFFFu - min(m2 & 0xFFFFu, m2 >> 16));
+        nz2 = nzc[0] + nzc[1];
+        const uint32_t mxx = __vimax3_u16x2(mx[0], mx[1], mx[1]);
+        const uint32_t m2 = __vimin3_u16x2(__vimin3_u16x2(mn[0], mn[1], mn[2]), mn[3], mn[3]);
+        all = (max(mxx & 0xFFFFu, mxx >> 16) << 16) | (0xFFFFu - min(m2 & 0xFFFFu, m2 >> 16));
     }
     uint32_t nz = (nz2 & 0xFFFFu) + (nz2 >> 16);
     // NaN or inf somewhere in the warp's data: redo the keys over finite elements and count the others
@@ -396,28 +400,36 @@ mor_amax_kernel(const __grid_constant__ MainParams p)
     if (warp == kThreads / 32) {
         // ---- load warp: one thread issues, the others leave ----
         if (lane != 0) return;
+        // what changes only with the tensor is kept in registers: the CTA's tile numbers only grow, so the search for
+        // a tile's tensor goes forward from the last one (reads of the records in the parameter space are slow)
+        int ti = -1;
+        uint32_t begin = 0u, end = 0u, nbc = 1u;
+        AmaxMeta m;
+        m.ti = 0; m.local = 0u; m.mode = 0u; m.key_stride = 0u; m.keys = nullptr; m.col_keys = nullptr;
+#pragma unroll 1
         for (uint32_t it = 0; it < n_it; ++it) {
             const uint32_t s = it % kAmaxStages, tile = blockIdx.x + it * gridDim.x;
+            if (ti < 0 || (tile >= end && ti < p.b.n - 1)) {
+                if (ti < 0) { ti = 0; end = p.b.tile_end[0]; }
+                while (tile >= end && ti < p.b.n - 1) { begin = end; ++ti; end = p.b.tile_end[ti]; }
+                const TensorRec& R = p.b.t[ti];
+                nbc = R.nbc;
+                m.ti = ti; m.key_stride = R.key_stride; m.keys = R.keys; m.col_keys = R.col_keys;
+                const bool cols = m.col_keys != nullptr;
+                m.mode = (m.keys != nullptr ? kModeKeys : 0u) |
+                         (m.keys != nullptr && m.key_stride == (uint32_t)kRowKeyStride && m.col_keys != m.keys ? kModePerPiece : 0u) |
+                         (cols ? kModeColPiece : 0u) | (m.keys != nullptr && R.kind == KIND_BLK64 ? kModeBlk64 : 0u) |
+                         (cols && m.col_keys != m.keys ? kModeColsApart : 0u);
+            }
             if (it >= (uint32_t)kAmaxStages &&
                 !mbar_wait(&C.empty[s], (it / kAmaxStages - 1u) & 1u, &C.abort, p.wait_cycles)) {
                 C.abort = 1u;
                 atomicOr(p.device_status, 1u);
                 break;
             }
-            uint32_t local;
-            const int ti = find_tensor(p.b, tile, local);
-            const TensorRec& R = p.b.t[ti];
-            const uint32_t bi = local / R.nbc, bj = local - bi * R.nbc;
-            {
-                AmaxMeta m;
-                m.ti = ti; m.local = local; m.key_stride = R.key_stride; m.keys = R.keys; m.col_keys = R.col_keys;
-                const bool cols = R.col_keys != nullptr;
-                m.mode = (R.keys != nullptr ? kModeKeys : 0u) |
-                         (R.keys != nullptr && R.key_stride == (uint32_t)kRowKeyStride && R.col_keys != R.keys ? kModePerPiece : 0u) |
-                         (cols ? kModeColPiece : 0u) | (R.keys != nullptr && R.kind == KIND_BLK64 ? kModeBlk64 : 0u) |
-                         (cols && R.col_keys != R.keys ? kModeColsApart : 0u);
-                C.meta[s] = m;                           // (made visible by the arrival below)
-            }
+            m.local = tile - begin;
+            const uint32_t bi = m.local / nbc, bj = m.local - bi * nbc;
+            C.meta[s] = m;                               // (made visible by the arrival below)
             // (test hook: the load of one chosen tile is left out, so that the waits for it run out)
             if (tile != p.test_skip_tile) {
                 mbar_arrive_expect_tx(&C.full[s], (uint32_t)kAmaxStageBytes);
