@@ -277,7 +277,7 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--profile", default=None, metavar="RECIPE",
                     help="run only three calls of one recipe on --batch 4096x4096 tensors and exit (the small case that the "
-                         "profiler wraps): 128x128, 1x128, 64x64, 128x1, per-tensor, per-channel, each optionally followed by "
+                         "profiler wraps): 128x128, 1x128, 64x64, 128x1, per-tensor, per-channel, rows+cols, each optionally followed by "
                          "-supplied (group amax given: single read) or -three (three formats, gradient-like data)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -314,12 +314,19 @@ def main():
         name = args.profile
         three, supplied = name.endswith("-three"), name.endswith("-supplied")
         base = name.replace("-three", "").replace("-supplied", "")
-        block = {"128x128": (128, 128), "1x128": (1, 128), "64x64": (64, 64), "128x1": (128, 1), "per-tensor": (0, 0), "per-channel": (1, 0)}[base]
+        block = {"128x128": (128, 128), "1x128": (1, 128), "64x64": (64, 64), "128x1": (128, 1), "per-tensor": (0, 0), "per-channel": (1, 0), "rows+cols": (1, 128)}[base]
         crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) else E3
         gen = (lambda i: wl.gradient_like(ROWS, COLS, seed=3 + i)) if three else (lambda i: wl.weight_like(ROWS, COLS, seed=1 + 1000 * i))
         pxs = [torch.from_numpy(gen(i).view(np.int16)).view(torch.bfloat16).to(dev) for i in range(args.batch)]
         ga = mb.group_amax(pxs) if supplied else None
-        pplan = mb.BatchPlan(pxs, [mb.Recipe(block, T3 if three else T2, crit, 0.045)] * args.batch, group_amax=ga)
+        if base == "rows+cols":        # every tensor with 1x128 and with 128x1 blocks: one paired launch
+            pair_x, pair_r = [], []
+            for x in pxs:
+                pair_x += [x, x]
+                pair_r += [mb.Recipe((1, 128), T2, E3, 0.045), mb.Recipe((128, 1), T2, E3, 0.045)]
+            pplan = mb.BatchPlan(pair_x, pair_r)
+        else:
+            pplan = mb.BatchPlan(pxs, [mb.Recipe(block, T3 if three else T2, crit, 0.045)] * args.batch, group_amax=ga)
         for _ in range(3):
             pplan.run(torch.cuda.current_stream())
         torch.cuda.synchronize()

@@ -56,16 +56,6 @@ __device__ __forceinline__ void block_scale(float b_amax, uint32_t m_g, int scal
     s5_bits = (e5 << 23) | m;
 }
 
-__device__ __forceinline__ int find_tensor(const BatchParams& p, uint32_t tile, uint32_t& local)
-{
-    int ti = 0;
-    uint32_t begin = 0;
-#pragma unroll 1
-    while (ti < p.n - 1 && tile >= p.tile_end[ti]) { begin = p.tile_end[ti]; ++ti; }
-    local = tile - begin;
-    return ti;
-}
-
 __device__ __forceinline__ double warp_sum(double v)
 {
 #pragma unroll
@@ -110,13 +100,12 @@ __device__ __noinline__ uint2 key_of_chunk_finite(uint4 v)
 }
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
 
-// One 128 x 128 tile per CTA (the tiling of the main kernel); 16-byte loads straight to registers,
-// 16 lanes per 256-byte row piece.  Results: the tensor's amax (Algorithm 1, first step,
-// with the tensor as one group) by atomicMax and, when the tensor
-// record has a key array, the key of every row piece of the tile (1x128 partition: that is the
-// block's amax and smallest non-zero) or of the whole tile (other partitions), which lets the main
-// kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its elements (the key itself
-// covers the finite ones only).
+// The pre-pass works on the 128 x 128 tiles of the main kernel.  Results: the tensor's amax (Algorithm 1, first step,
+// with the tensor as one group) by atomicMax and, when the tensor record has a key array, per tile the key of every
+// row piece (1x128 partition: that is the block's amax and smallest non-zero), of every column piece (blocks along
+// the columns), of every 64x64 quadrant or of the whole tile (other partitions), and the tile's count of finite
+// non-zero elements, which let the main kernel skip its own scan.  Bit 31 of a key marks NaN/inf among its
+// elements (the key itself covers the finite ones only).
 // What the load warp tells the other warps about the tile in a stage (and, copied into the scratch, the tail warp).
 constexpr uint32_t kModeKeys = 1u;        // the record wants keys (and the tile's count of non-zeros)
 constexpr uint32_t kModePerPiece = 2u;    // ... one per row piece
