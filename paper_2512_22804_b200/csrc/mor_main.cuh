@@ -607,8 +607,8 @@ __device__ __forceinline__ void emit_e5m2_codes(const uint32_t (&w)[32], uint32_
 
 // Algorithm 2 for one block with the per-block metrics (M_1 = Eq. 3, M_2 = Eq. 4, or
 // Eq. 1-2 on the block alone).
-template <typename T>
-__device__ __forceinline__ uint32_t decide_block(const TensorRec& R, T e43, T e52, uint32_t nnz,
+template <typename T, typename REC>
+__device__ __forceinline__ uint32_t decide_block(const REC& R, T e43, T e52, uint32_t nnz,
                                                  uint32_t nonfinite, uint32_t amax_bits, uint32_t minm1_bits,
                                                  uint32_t n_elems)
 {
@@ -659,6 +659,61 @@ __device__ __forceinline__ TileId locate_tile(const BatchParams& b, uint32_t til
     t.vcols = (int)(cc < kTileCols ? cc : kTileCols);
     return t;
 }
+
+// The load warp and the store warp work once per tile, and what they need of the tensor's record sits in the
+// kernel's parameter space, where a read with a computed index is slow and a chain of them (pointer, test, branch,
+// next pointer) adds up to microseconds per tile.  They keep what they need in registers instead and reload it when
+// the CTA moves on to another tensor; a CTA's tile numbers only grow, so the search for a tile's tensor goes forward
+// from the last one.
+struct RecFacts {
+    uint8_t* sel;
+    uint8_t* scale_e8m0;
+    float* scale_f32;
+    mor_block_stats_t* block_stats;
+    uint32_t* keys;
+    uint32_t* row_keys;
+    long long cols;
+    uint32_t tile_begin, nbc, nbc_blk, key_stride, flags;
+    int32_t criterion, n_formats;
+    float threshold;
+    __device__ __forceinline__ void load(const TensorRec& R)
+    {
+        sel = R.sel; scale_e8m0 = R.scale_e8m0; scale_f32 = R.scale_f32; block_stats = R.block_stats;
+        keys = R.keys; row_keys = R.row_keys; cols = R.cols;
+        tile_begin = R.tile_begin; nbc = R.nbc; nbc_blk = R.nbc_blk; key_stride = R.key_stride; flags = R.flags;
+        criterion = R.criterion; n_formats = R.n_formats; threshold = R.threshold;
+    }
+};
+
+struct TileWalker {
+    int ti;
+    uint32_t begin, end, nbc;
+    long long rows, cols;
+    __device__ __forceinline__ TileWalker() : ti(-1), begin(0u), end(0u), nbc(1u), rows(0), cols(0) {}
+    // moves to the tensor of `tile`; true when that is another tensor than before (or the first call)
+    __device__ __forceinline__ bool seek(const BatchParams& b, uint32_t tile)
+    {
+        if (ti >= 0 && (tile < end || ti >= b.n - 1)) return false;
+        if (ti < 0) { ti = 0; begin = 0u; end = b.tile_end[0]; }
+#pragma unroll 1
+        while (ti < b.n - 1 && tile >= end) { begin = end; ++ti; end = b.tile_end[ti]; }
+        nbc = b.t[ti].nbc; rows = b.t[ti].rows; cols = b.t[ti].cols;
+        return true;
+    }
+    __device__ __forceinline__ TileId id(uint32_t tile) const
+    {
+        TileId t;
+        t.ti = ti;
+        t.local = tile - begin;
+        const uint32_t bi = t.local / nbc, bj = t.local - bi * nbc;
+        t.row0 = (int)(bi * kTileRows);
+        t.col0 = (int)(bj * kTileCols);
+        const long long rr = rows - t.row0, cc = cols - t.col0;
+        t.vrows = (int)(rr < kTileRows ? rr : kTileRows);
+        t.vcols = (int)(cc < kTileCols ? cc : kTileCols);
+        return t;
+    }
+};
 
 // tiles blockIdx.x, blockIdx.x + gridDim.x, ... below total_tiles (the grid never exceeds the tile count)
 __device__ __forceinline__ uint32_t my_tile_count(const MainParams& p)
@@ -720,15 +775,36 @@ __device__ __forceinline__ bool prepare_lines(const uint32_t* key_src, uint32_t 
     return all;
 }
 
+// What the load warp keeps about the tensor it is on.
+struct LoadState {
+    TileWalker walk;
+    RecFacts R;
+    const uint32_t* col_keys2;      // rows and columns from one read: the keys of the columns' record
+    uint32_t m_g, tensor_amax_bits;
+    int scale_mode;
+    __device__ __forceinline__ LoadState() : col_keys2(nullptr), m_g(0u), tensor_amax_bits(0u), scale_mode(0) {}
+};
+
 template <int KIND, bool PREP, bool COLFAST>
-__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it, int lane,
-                                                int& cur_ti, uint32_t& m_g, int& scale_mode, uint32_t& tensor_amax_bits)
+__device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C, unsigned char* in, uint32_t it, int lane, LoadState& L)
 {
     const uint32_t tile = blockIdx.x + it * gridDim.x;
     if (tile >= p.total_tiles) return;
     const uint32_t s = it % kStages;
-    const TileId t = locate_tile(p.b, tile);
-    const TensorRec& R = p.b.t[t.ti];
+    if (L.walk.seek(p.b, tile)) {
+        const TensorRec& T = p.b.t[L.walk.ti];
+        L.R.load(T);
+        if (PREP) {
+            L.scale_mode = T.scale_mode;
+            L.m_g = group_mantissa(*T.amax, L.scale_mode);
+            if (KIND == KIND_TENSOR) L.tensor_amax_bits = __float_as_uint(*T.amax_slot) >> 16;
+            if (KIND == KIND_DUAL) L.col_keys2 = p.b.t[L.walk.ti + 1].keys;
+        }
+    }
+    const TileId t = L.walk.id(tile);
+    const RecFacts& R = L.R;
+    const uint32_t m_g = L.m_g, tensor_amax_bits = L.tensor_amax_bits;
+    const int scale_mode = L.scale_mode;
     // (the full-width column paths need nothing but the prepared words: no copy of the keys)
     const uint32_t key_bytes = (R.keys == nullptr || COLFAST) ? 0u : ((KIND == KIND_CHANNEL || KIND == KIND_COLCH) ? (uint32_t)kTileRows * 4u : R.key_stride * 4u);
     const uint32_t* key_src = KIND == KIND_CHANNEL ? R.row_keys + t.row0 : KIND == KIND_COLCH ? R.row_keys + t.col0
@@ -742,18 +818,12 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
     }
     uint32_t tile_nnz = 0u;
     if (PREP) {
-        if (t.ti != cur_ti) {
-            cur_ti = t.ti;
-            scale_mode = R.scale_mode;
-            m_g = group_mantissa(*R.amax, scale_mode);
-            if (KIND == KIND_TENSOR) tensor_amax_bits = __float_as_uint(*R.amax_slot) >> 16;
-        }
         tile_nnz = R.keys[(size_t)t.local * R.key_stride + (R.key_stride == (uint32_t)kRowKeyStride ? (uint32_t)kTileRows : 4u)];
         if (KIND == KIND_ROW128 || KIND == KIND_CHANNEL || KIND == KIND_DUAL) {          // one key per row of the tile
             prepare_lines<0>(key_src, m_g, scale_mode, C.rtab, &C.prep[s][0], lane);
             if (KIND == KIND_DUAL) {
                 // ... and one per column, from the columns' record (same tiles, same group amax)
-                const bool any = prepare_lines<2>(p.b.t[t.ti + 1].keys + (size_t)t.local * kRowKeyStride, m_g, scale_mode, C.rtab, &C.prep2[s][0], lane);
+                const bool any = prepare_lines<2>(L.col_keys2 + (size_t)t.local * kRowKeyStride, m_g, scale_mode, C.rtab, &C.prep2[s][0], lane);
                 if (lane == 0) C.colflag[s] = any ? 1u : 0u;
             }
         } else if (KIND == KIND_COL128 || KIND == KIND_COLCH) {                            // one key per column of the tile
@@ -798,15 +868,14 @@ __device__ __forceinline__ void issue_tile_load(const MainParams& p, Control& C,
 template <int KIND, bool PREP, bool COLFAST>
 __device__ __forceinline__ void load_warp(const MainParams& p, Control& C, unsigned char* in, int lane)
 {
-    int cur_ti = -1, scale_mode = 0;
-    uint32_t m_g = 0u, tensor_amax_bits = 0u;
-    for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
+    LoadState L;
+    for (uint32_t it = 0; it < (uint32_t)kStages; ++it) issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it, lane, L);
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
         stage_free_sync(it % kStages);                  // sleeps until every compute thread has its copy
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u))
-            issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it + kStages, lane, cur_ti, m_g, scale_mode, tensor_amax_bits);
+            issue_tile_load<KIND, PREP, COLFAST>(p, C, in, it + kStages, lane, L);
     }
     if (lane == 0 && C.abort) {
         // copies that may still be in flight must land (or be given up on) before the CTA goes
@@ -827,6 +896,9 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
     constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128 || KIND == KIND_DUAL;   // 128 one-line blocks per tile
     constexpr int kEntries = kLineBlocks ? kTileRows : kThreads;
     bool stores_pending = false;
+    TileWalker walk;
+    RecFacts F0, F1;                                     // F1: the columns' record of a rows-and-columns pair
+    if (KIND == KIND_DUAL) F1 = RecFacts();
 #pragma unroll 1
     for (uint32_t it = 0;; ++it) {
         // both directions from one read: two conversions per tile, rows (record ti) then columns (record ti + 1)
@@ -834,9 +906,13 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         if (tile >= p.total_tiles) break;
         const uint32_t b = it & 1u, n = it >> 1;
         const bool columns = KIND == KIND_COL128 || KIND == KIND_COLCH || (KIND == KIND_DUAL && (it & 1u));
-        TileId t = locate_tile(p.b, tile);              // before the wait: off the critical path
+        if (walk.seek(p.b, tile)) {                      // (before the wait: off the critical path)
+            F0.load(p.b.t[walk.ti]);
+            if (KIND == KIND_DUAL) F1.load(p.b.t[walk.ti + 1]);
+        }
+        TileId t = walk.id(tile);
         if (KIND == KIND_DUAL && columns) t.ti += 1;
-        const TensorRec& R = p.b.t[t.ti];
+        const RecFacts R = (KIND == KIND_DUAL && columns) ? F1 : F0;     // (a copy: both stay in registers)
         constexpr bool kTileBlocks = KIND == KIND_BLK128 || KIND == KIND_BLK64;
         // the decision is handed back on every tile of a launch whose compute threads may need it (three formats:
         // E5M2 codes; EXTRA: a BF16 copy or a fake-quantised output for some tensor of the launch), whether this
@@ -1367,7 +1443,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                         if (R.sel) R.sel[blk] = (uint8_t)sel;
                         if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
                         if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
-                        if (R.block_stats) {
+                        if (EXTRA && R.block_stats) {
                             mor_block_stats_t bs;
                             bs.amax = __uint_as_float(amax_bits << 16);
                             bs.min_abs_nz = THREE ? minnz_value(minm1) : __uint_as_float(0x7F800000u);
@@ -1681,6 +1757,8 @@ __device__ __forceinline__ void compute_dual_fast(const MainParams& p, Control& 
     const uint32_t meta_base = smem_addr(&C.meta[0]), prep_base = smem_addr(&C.prep[0][0]), prep2_base = smem_addr(&C.prep2[0][0]);
     const uint32_t flag_base = smem_addr(&C.colflag[0]);
     bool dead = false;
+    RecFacts Q;              // what the rows' decision and metadata need of their record, reloaded per tensor
+    int q_ti = -1;
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
@@ -1700,7 +1778,8 @@ __device__ __forceinline__ void compute_dual_fast(const MainParams& p, Control& 
 
         // ---- rows (record ti): the streaming 1x128 path ----
         {
-            const TensorRec& R = p.b.t[m.ti];
+            if (m.ti != q_ti) { q_ti = m.ti; Q.load(p.b.t[m.ti]); }
+            const RecFacts& R = Q;
             uint32_t prep;
             asm volatile("ld.shared.u32 %0, [%1];" : "=r"(prep) : "r"(prep_base + s * (uint32_t)(kTileRows * 4) + (uint32_t)row * 4u));
             const uint32_t s4b = prep & 0x7FFFFFFFu;
