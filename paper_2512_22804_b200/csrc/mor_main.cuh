@@ -929,7 +929,44 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 stores_pending = true;
             }
 
-            if (COLFAST && (KIND != KIND_DUAL || columns)) {
+            if (COLFAST && KIND == KIND_ROW128) {
+                // 1x128 blocks whose compute threads hand over their sums and the row's scale (entry of thread
+                // 2 row + h: {E4M3 sum, E5M2 sum, non-zeros | non-finites << 16, scale bits}): this lane adds the two
+                // halves of rows lane, lane + 32, ..., decides their blocks and writes their metadata.
+                const uint32_t ea = smem_addr(&C.entry[b][0]) + (uint32_t)lane * 32u;
+                float f43 = 0.0f, f52 = 0.0f;
+                uint32_t n4 = 0, n5 = 0, nb = 0, tnnz = 0, tnonf = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint4 e0 = lds128(ea + (uint32_t)k * 1024u), e1 = lds128(ea + (uint32_t)k * 1024u + 16u);
+                    const float e43 = __uint_as_float(e0.x) + __uint_as_float(e1.x), e52 = __uint_as_float(e0.y) + __uint_as_float(e1.y);
+                    const uint32_t nz = e0.z + e1.z;
+                    f43 += e43; f52 += e52; tnnz += nz & 0xFFFFu; tnonf += nz >> 16;
+                    const int row = lane + 32 * k;
+                    if (row < t.vrows) {
+                        const uint32_t bsel = decide_block(R, e43, e52, 0u, nz >> 16, 0u, 0xFFFFu, (uint32_t)t.vcols);
+                        const uint32_t blk = (uint32_t)(t.row0 + row) * R.nbc + (uint32_t)(t.col0 / kTileCols);
+                        if (R.sel) R.sel[blk] = (uint8_t)bsel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(e0.w >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(e0.w);
+                        n4 += bsel == MOR_FMT_E4M3; n5 += bsel == MOR_FMT_E5M2; nb += bsel == MOR_FMT_BF16;
+                    }
+                }
+                double s43 = (double)f43, s52 = (double)f52;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { s43 += shfl_xor_f64(s43, o); s52 += shfl_xor_f64(s52, o); }
+                n4 = __reduce_add_sync(0xFFFFFFFFu, n4);
+                n5 = __reduce_add_sync(0xFFFFFFFFu, n5);
+                nb = __reduce_add_sync(0xFFFFFFFFu, nb);
+                tnnz = __reduce_add_sync(0xFFFFFFFFu, tnnz);
+                tnonf = __reduce_add_sync(0xFFFFFFFFu, tnonf);
+                if (lane == 0) {
+                    Partial P;
+                    P.sum43 = s43; P.sum52 = s52; P.nnz = tnnz; P.nonfinite = tnonf;
+                    P.n_e4m3 = n4; P.n_e5m2 = n5; P.n_bf16 = nb; P.min_nz_bits = 0xFFFFu;
+                    partials[R.tile_begin + t.local] = P;
+                }
+            } else if (COLFAST && (KIND != KIND_DUAL || columns)) {
                 // Blocks along the columns, handed over by cols_fast_tile: this lane takes columns 4 lane ..
                 // 4 lane + 3; a column's sums come in four parts (row groups), added in the order of the parts.
                 const uint32_t ea = smem_addr(&C.entry[b][0]) + (uint32_t)lane * 32u;
@@ -1419,7 +1456,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
             if (!kCount && tid == 0) nnz = m.nnz;       // the tile's count from the pre-pass, handed on in this thread's entry
 
-            if (kLineBlocks) {
+            constexpr bool kRowFast = KIND == KIND_ROW128 && !SCAN && !EXTRA && !THREE;
+            if (kRowFast) {
+                // the store warp adds the row's two halves, decides the block and writes its metadata
+                sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
+                       make_uint4(__float_as_uint(e43), __float_as_uint(e52), nnz | (nonf << 16), s4b));
+            } else if (kLineBlocks) {
                 // ---- block sums, decision, metadata ----
                 e43 += __shfl_xor_sync(0xFFFFFFFFu, e43, 1);
                 e52 += __shfl_xor_sync(0xFFFFFFFFu, e52, 1);
@@ -2022,6 +2064,8 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     // 128x1 blocks (alone, or beside the 1x128 blocks of the same tensor) with keys from the pre-pass, two formats,
     // plain outputs: the full-width column path
     constexpr bool kColFast = (KIND == KIND_COL128 || KIND == KIND_DUAL) && !SCAN && !EXTRA && !THREE;
+    // ... and the 1x128 blocks of the same recipe leave their decisions and metadata to the store warp as well
+    constexpr bool kRowFast = KIND == KIND_ROW128 && !SCAN && !EXTRA && !THREE;
     if (warp < kComputeWarps) {
         if constexpr (KIND == KIND_DUAL && kColFast) compute_dual_fast<YARD>(p, C, in, out, tid);
         else if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
@@ -2029,7 +2073,7 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
         else compute_warps<KIND, YARD, THREE, STORE, SCAN, EXTRA>(p, C, in, out, tid);
     }
     else if (warp == kLoadWarp) load_warp<KIND, !SCAN && (KIND != KIND_DUAL || kColFast), kColFast>(p, C, in, lane);
-    else store_warp<KIND, THREE, STORE, EXTRA, kColFast>(p, C, out, partials, lane);
+    else store_warp<KIND, THREE, STORE, EXTRA, kColFast || kRowFast>(p, C, out, partials, lane);
 }
 
 template <int KIND, bool YARD, bool THREE, bool STORE, bool SCAN, bool EXTRA>
