@@ -1255,6 +1255,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     int scale_mode = 0;
     bool has_fallback = false;
     bool has_fq = false, fq_e4m3 = false;   // fake-quantised output wanted; ... with E4M3 values whatever the block's selection
+    float* amax_slot = nullptr;              // scanning variants: where to gather the tensor amax (nullptr: nowhere)
     const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]), prep_base = smem_addr(&C.prep[0][0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
     const uint32_t n_it = my_tile_count(p);
@@ -1316,6 +1317,8 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             if (SCAN) {
                 scale_mode = R.scale_mode;
                 if (!dead) m_g = group_mantissa(*R.amax, scale_mode);
+                // no pre-pass ran and the caller gave no amax: the tensor amax that the summary reports is gathered here
+                amax_slot = (!(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot) ? R.amax_slot : nullptr;
             }
         }
         if (EXTRA || (!kCount && tid == 0)) {          // the tile's position (BF16 outputs) and its non-zero count
@@ -1345,9 +1348,9 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
             // patterns order like the values)
-            if (!(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot) {
+            if (amax_slot != nullptr) {
                 const uint32_t wamax = __reduce_max_sync(0xFFFFFFFFu, key >> 16);
-                raise_amax(R.amax_slot, wamax, lane == 0 && !dead);
+                raise_amax(amax_slot, wamax, lane == 0 && !dead);
             }
         } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
             key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
@@ -1382,7 +1385,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here
-            raise_amax(R.amax_slot, tile_amax, tid == 0 && !dead && !(R.flags & kFlagAmaxFinal) && R.amax == R.amax_slot);
+            if (amax_slot != nullptr) raise_amax(amax_slot, tile_amax, tid == 0 && !dead);
         } else {
             key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
@@ -1456,7 +1459,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
             if (!kCount && tid == 0) nnz = m.nnz;       // the tile's count from the pre-pass, handed on in this thread's entry
 
-            constexpr bool kRowFast = KIND == KIND_ROW128 && !SCAN && !EXTRA && !THREE;
+            constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
             if (kRowFast) {
                 // the store warp adds the row's two halves, decides the block and writes its metadata
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
@@ -2064,8 +2067,8 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     // 128x1 blocks (alone, or beside the 1x128 blocks of the same tensor) with keys from the pre-pass, two formats,
     // plain outputs: the full-width column path
     constexpr bool kColFast = (KIND == KIND_COL128 || KIND == KIND_DUAL) && !SCAN && !EXTRA && !THREE;
-    // ... and the 1x128 blocks of the same recipe leave their decisions and metadata to the store warp as well
-    constexpr bool kRowFast = KIND == KIND_ROW128 && !SCAN && !EXTRA && !THREE;
+    // ... and the 1x128 blocks of that recipe (scanning or not) leave their decisions and metadata to the store warp too
+    constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
     if (warp < kComputeWarps) {
         if constexpr (KIND == KIND_DUAL && kColFast) compute_dual_fast<YARD>(p, C, in, out, tid);
         else if constexpr (KIND == KIND_DUAL) compute_warps_dual<YARD, THREE, SCAN>(p, C, in, out, tid);
