@@ -170,3 +170,54 @@ def test_mixed_grid_128x128_three_way_full():
         out = mb.analyze_quantize(xs[0], rr)
         torch.cuda.synchronize()
         assert parity.compare(bits, rr, out, sub, ids=ids).n_exempt <= 4
+
+
+def test_rows_and_columns_full_size_plain_paired_call_sampled():
+    """8 configs[1]-sized tensors, each with 1x128 and with 128x1 blocks in one paired call of the plain two-format
+    recipe (the launch configuration bench.py times for that line): the streaming row path and the full-width
+    column path with keys of both directions from one pre-pass.  Sampled blocks of both directions against the
+    oracle, whole-tensor counts, and the codes of the column direction as the transpose of what the row direction
+    gives for the transposed tensor."""
+    import torch
+
+    hosts = [wl.weight_like(4096, 4096, seed=1 + 1000 * i) for i in range(3)]
+    hosts[1][17, 4000] = 0x7F80           # an inf: its tile takes the careful path in both directions
+    hosts[2][:, 77] = 0                   # a column of zeros
+    hosts[2][300:428, 1000:1128] = wl.gradient_like(128, 128, seed=5)     # a tile with tiny and large values side by side
+    xs = [parity.to_device(h) for h in hosts]
+    rr, rc = mb.Recipe((1, 128), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045), mb.Recipe((128, 1), TWO, mb.MOR_CRIT_BLOCK_VS_E5M2, 0.045)
+    px, pr = [], []
+    for x in xs:
+        px += [x, x]
+        pr += [rr, rc]
+    plan = mb.BatchPlan(px, pr)
+    plan.run()
+    plan.run()
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(17)
+    for i, h in enumerate(hosts):
+        for r, o in ((rr, plan.outs[2 * i]), (rc, plan.outs[2 * i + 1])):
+            grid = mb.grid_of(4096, 4096, r.block)
+            nb = grid[0] * grid[1]
+            ids = rng.choice(nb, 1024, replace=False)
+            if i == 1:      # the blocks around the inf
+                ids = np.concatenate([ids, [17 * 32 + 31] if r.block == (1, 128) else [0 * 4096 + 4000]])
+            if i == 2 and r.block == (128, 1):
+                ids = np.concatenate([ids, np.arange(32) * 4096 + 77, 2 * 4096 + 1000 + np.arange(128), 3 * 4096 + 1000 + np.arange(128)])
+            ids = np.unique(ids)
+            ref = orc.run(h, r.block, list(r.formats), r.criterion, r.threshold, ids=ids)
+            parity.compare(h, r, o, ref, ids=ids, check_block_stats=False)
+            ts = o.tensor_stats_dict()
+            assert ts["status"] == 0 and ts["n_blocks"] == nb == ts["n_e4m3"] + ts["n_e5m2"] + ts["n_bf16"]
+            assert ts["nnz"] == int(np.count_nonzero((h & 0x7FFF) != 0) - np.count_nonzero((h & 0x7FFF) >= 0x7F80))
+            assert ts["n_nonfinite"] == int(np.count_nonzero((h & 0x7FFF) >= 0x7F80))
+        # single calls give the same bytes
+        single = mb.analyze_quantize(xs[i], rc)
+        torch.cuda.synchronize()
+        assert torch.equal(single.codes, plan.outs[2 * i + 1].codes) and torch.equal(single.sel, plan.outs[2 * i + 1].sel)
+        xt = parity.to_device(np.ascontiguousarray(h.T))
+        tr = mb.analyze_quantize(xt, rr)
+        torch.cuda.synchronize()
+        assert torch.equal(tr.codes, plan.outs[2 * i + 1].codes)
+        assert torch.equal(tr.sel.t().contiguous(), plan.outs[2 * i + 1].sel)
+        assert torch.equal(tr.scale_e8m0.t().contiguous(), plan.outs[2 * i + 1].scale_e8m0)

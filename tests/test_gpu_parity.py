@@ -699,3 +699,23 @@ def test_invalid_arguments_launch_nothing():
     o = mb.alloc_outputs(128, 256, recipe((1, 128)), x.device)
     assert mb.mor_analyze_quantize(d, o.c_struct, 0, 0) == mb.MOR_ERR_WORKSPACE
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("shape", [(256, 256), (384, 200), (130, 520), (517, 72), (2560, 2048)])
+def test_full_width_column_path_edge_cases(shape):
+    """128x1 blocks, plain two-format recipe with the pre-pass (per-column scales prepared by the load warp, four
+    columns x 16 rows per thread): columns of zeros, a column piece whose amax is tiny (its scale exponent is beyond
+    what the fast conversion takes), NaN and infinities (their blocks stay in BF16, the tile takes the careful path),
+    ragged edges in both directions, and more tiles than resident CTAs."""
+    rows, cols = shape
+    g = wl.weight_like(rows, cols, seed=71)
+    g[:, 3] = 0                                   # zeros all the way down
+    g[: min(rows, 128), 9] = 0x0001               # smallest subnormal: the largest scale there is
+    g[5, 20] = 0x7FC0
+    if rows > 140:
+        g[140, 21] = 0xFF80
+        g[128:, 40] = wl.gradient_like(rows - 128, 1, seed=72)[:, 0]      # a wide spread of exponents down a column
+    ld = (cols + 7) // 8 * 8
+    for r in (recipe((128, 1), TWO), recipe((128, 1), TWO, mb.MOR_CRIT_TENSOR_MEAN_REL), recipe((128, 1), TWO, scale_mode=mb.MOR_SCALE_E8M0)):
+        rep = parity.run_and_compare(g, r, pad_to=ld if ld != cols else None, block_stats=False)
+        assert rep.n_exempt <= 2
