@@ -775,6 +775,14 @@ __device__ __forceinline__ bool prepare_lines(const uint32_t* key_src, uint32_t 
     return all;
 }
 
+// What a compute thread needs of the record to decide a block (Algorithm 2), kept in registers per tensor.
+struct DecideFacts {
+    int32_t criterion, n_formats;
+    uint32_t flags;
+    float threshold;
+    __device__ __forceinline__ void load(const TensorRec& R) { criterion = R.criterion; n_formats = R.n_formats; flags = R.flags; threshold = R.threshold; }
+};
+
 // What the load warp keeps about the tensor it is on.
 struct LoadState {
     TileWalker walk;
@@ -895,6 +903,9 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
 {
     constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128 || KIND == KIND_DUAL;   // 128 one-line blocks per tile
     constexpr int kEntries = kLineBlocks ? kTileRows : kThreads;
+    // 1x128 / 128x1 blocks without the optional outputs, where the compute threads decide (three formats, or the
+    // 16-bit column gather): the metadata is written here, from the entries
+    constexpr bool kMetaHere = (KIND == KIND_ROW128 || KIND == KIND_COL128) && !EXTRA && !COLFAST;
     bool stores_pending = false;
     TileWalker walk;
     RecFacts F0, F1;                                     // F1: the columns' record of a rows-and-columns pair
@@ -1024,6 +1035,15 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 if (kLineBlocks) {
                     const uint32_t sel = e.sel_min & 0xFFFFu;
                     n4 += sel == MOR_FMT_E4M3; n5 += sel == MOR_FMT_E5M2; nb += sel == MOR_FMT_BF16;
+                    if (kMetaHere && sel != kSelNone) {
+                        // the block's selection and scale, left by the line's first thread
+                        const uint32_t line = (uint32_t)(lane + 32 * k), sb = C.colscale[b][line];
+                        const uint32_t blk = KIND == KIND_COL128 ? (uint32_t)(t.row0 / kTileRows) * (uint32_t)R.cols + (uint32_t)t.col0 + line
+                                                                 : ((uint32_t)t.row0 + line) * R.nbc + (uint32_t)(t.col0 / kTileCols);
+                        if (R.sel) R.sel[blk] = (uint8_t)sel;
+                        if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(sb >> 23);
+                        if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(sb);
+                    }
                 }
                 mn = min(mn, e.sel_min >> 16);
             }
@@ -1258,6 +1278,12 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     float* amax_slot = nullptr;              // scanning variants: where to gather the tensor amax (nullptr: nowhere)
     const uint32_t meta_base = smem_addr(&C.meta[0]), keys_base = smem_addr(&C.keys[0][0]), prep_base = smem_addr(&C.prep[0][0]);
     bool dead = false;       // a wait has run out somewhere in the CTA: keep the arrivals, skip the rest
+    DecideFacts D;           // line blocks: what the block's decision needs of the record, reloaded per tensor
+    int d_ti = -1;
+    // line blocks without the optional outputs: the store warp writes the blocks' metadata (from the entries and the
+    // scale that the row's first thread leaves it); with them everything about a block is written from here
+    constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
+    constexpr bool kMetaInStore = kLineBlocks && !EXTRA && !kRowFast;
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
@@ -1309,6 +1335,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
         }
         const TensorRec& R = p.b.t[m.ti];
+        if (kLineBlocks && !kRowFast && m.ti != d_ti) { d_ti = m.ti; D.load(R); }
         if ((SCAN || EXTRA) && m.ti != cur_ti) {
             cur_ti = m.ti;
             has_fallback = EXTRA && STORE && R.fallback != nullptr;
@@ -1459,7 +1486,6 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
             if (!kCount && tid == 0) nnz = m.nnz;       // the tile's count from the pre-pass, handed on in this thread's entry
 
-            constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
             if (kRowFast) {
                 // the store warp adds the row's two halves, decides the block and writes its metadata
                 sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)tid * 16u,
@@ -1471,7 +1497,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 uint32_t nz = nnz | (nonf << 16);
                 nz += __shfl_xor_sync(0xFFFFFFFFu, nz, 1);
                 const bool valid = row < (KIND == KIND_COL128 ? m.vcols : m.vrows);
-                sel = decide_block(R, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
+                sel = decide_block(D, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
                 if (kStash) {
                     if (sel == MOR_FMT_E5M2) copy_stash(in_base + s * kInBytes + in_off, oa);
                     fence_async_smem();                  // the stage is written by the next TMA load: order the stash accesses before it
@@ -1482,7 +1508,9 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 if (h == 0) {
                     sts128(entry_base + b * (uint32_t)sizeof(C.entry[0]) + (uint32_t)row * 16u,
                            make_uint4(__float_as_uint(e43), __float_as_uint(e52), nz, (valid ? sel : kSelNone) | (minm1 << 16)));
-                    if (valid) {
+                    if (kMetaInStore) {
+                        C.colscale[b][row] = (sel == MOR_FMT_E5M2) ? s5b : s4b;
+                    } else if (valid) {
                         const uint32_t blk = m.blk_base + (uint32_t)row * (KIND == KIND_COL128 ? 1u : R.nbc);
                         const uint32_t sb = (sel == MOR_FMT_E5M2) ? s5b : s4b;
                         if (R.sel) R.sel[blk] = (uint8_t)sel;
