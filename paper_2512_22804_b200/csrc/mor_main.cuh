@@ -996,6 +996,16 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                 for (int c = 0; c < 4; ++c) {
                     if (4 * lane + c >= t.vcols) continue;
                     const uint32_t s4b = sc[c] & 0x7FFFFFFFu;
+                    if (KIND == KIND_COLCH) {
+                        // per-channel: a column is one block over all tile rows; its decision is the tensor's (finalise
+                        // kernel); the first tile row writes the column's scale
+                        if (t.row0 == 0) {
+                            const uint32_t blk = (uint32_t)t.col0 + 4u * (uint32_t)lane + (uint32_t)c;
+                            if (R.scale_e8m0) R.scale_e8m0[blk] = (uint8_t)(s4b >> 23);
+                            if (R.scale_f32) R.scale_f32[blk] = __uint_as_float(s4b);
+                        }
+                        continue;
+                    }
                     const uint32_t bsel = decide_block(R, e43[c], e52[c], 0u, sc[c] >> 31, 0u, 0xFFFFu, (uint32_t)t.vrows);
                     if (R.sel) R.sel[blk0 + c] = (uint8_t)bsel;
                     if (R.scale_e8m0) R.scale_e8m0[blk0 + c] = (uint8_t)(s4b >> 23);
@@ -2092,9 +2102,9 @@ mor_main_kernel(const __grid_constant__ MainParams p, Partial* __restrict__ part
     pdl_trigger();
     pdl_wait();
 
-    // 128x1 blocks (alone, or beside the 1x128 blocks of the same tensor) with keys from the pre-pass, two formats,
-    // plain outputs: the full-width column path
-    constexpr bool kColFast = (KIND == KIND_COL128 || KIND == KIND_DUAL) && !SCAN && !EXTRA && !THREE;
+    // 128x1 blocks (alone, or beside the 1x128 blocks of the same tensor) and per-channel columns with keys from the
+    // pre-pass, two formats, plain outputs: the full-width column path
+    constexpr bool kColFast = (KIND == KIND_COL128 || KIND == KIND_DUAL || KIND == KIND_COLCH) && !SCAN && !EXTRA && !THREE;
     // ... and the 1x128 blocks of that recipe (scanning or not) leave their decisions and metadata to the store warp too
     constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
     if (warp < kComputeWarps) {
