@@ -346,14 +346,23 @@ __device__ __forceinline__ uint32_t scan_words_finite(const uint32_t (&w)[32])
 
 __device__ __forceinline__ uint32_t key_max(uint32_t a, uint32_t b) { return __vimax3_u16x2(a, b, b); }
 
+// Where a streaming thread finds the j-th of its eight 16-byte chunks of the stage, and where the chunk's eight codes
+// go in the staging buffer.  Swizzled (a thread owns half a tile row: the chunks of its 128 bytes in an order that
+// keeps the lanes of a load or store phase on distinct banks) or LINEAR (partitions whose blocks are not made of
+// rows -- a thread then owns chunk tid & 15 of rows (tid >> 4) + 16 j, the lanes of a phase read neighbouring
+// chunks of one row, and every address is its base plus a constant).
+template <bool LINEAR> __device__ __forceinline__ uint32_t in_chunk(uint32_t a, int j) { return LINEAR ? a + (uint32_t)(j * 16 * 256) : a ^ (uint32_t)(j << 4); }
+template <bool LINEAR> __device__ __forceinline__ uint32_t out_chunk(uint32_t a, int j) { return LINEAR ? a + (uint32_t)(j * 16 * 128) : a ^ (uint32_t)(j << 3); }
+
 // The same two scans for a thread that has not copied its elements to registers: the eight 16-byte chunks are read
-// from the stage at a ^ (j << 4) (the conversion reads them a second time afterwards).
+// from the stage (the conversion reads them a second time afterwards).
+template <bool LINEAR = false>
 __device__ __forceinline__ uint32_t scan_stage(uint32_t a)
 {
     uint32_t mx[2] = {0u, 0u}, mn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint4 v = lds128(a ^ (j << 4));
+        const uint4 v = lds128(in_chunk<LINEAR>(a, j));
         const uint32_t a0 = v.x & 0x7FFF7FFFu, a1 = v.y & 0x7FFF7FFFu, a2 = v.z & 0x7FFF7FFFu, a3 = v.w & 0x7FFF7FFFu;
         mx[0] = __vimax3_u16x2(mx[0], a0, a1);
         mx[1] = __vimax3_u16x2(mx[1], a2, a3);
@@ -367,11 +376,12 @@ __device__ __forceinline__ uint32_t scan_stage(uint32_t a)
     const uint32_t amax = max(mxx & 0xFFFFu, mxx >> 16), minm1 = min(mnn & 0xFFFFu, mnn >> 16);
     return (amax << 16) | (0xFFFFu - minm1);
 }
+template <bool LINEAR = false>
 __device__ __noinline__ uint32_t scan_stage_finite(uint32_t a)
 {
     uint32_t m = 0u, n = 0xFFFFu;
 #pragma unroll 1
-    for (int j = 0; j < 8; ++j) scan_finite4(lds128(a ^ (j << 4)), m, n);
+    for (int j = 0; j < 8; ++j) scan_finite4(lds128(in_chunk<LINEAR>(a, j)), m, n);
     return (m << 16) | (0xFFFFu - n);
 }
 
@@ -515,7 +525,7 @@ __device__ __forceinline__ void conv_init(ConvAcc& c)
 // the staging buffer; a block that ends up in E5M2 has them replaced afterwards (emit_e5m2_codes).
 // With STASH the E5M2 codes are kept as well: chunk j0 + j's eight codes go to stash_addr ^ ((j0 + j) << 4), which
 // is the place of the chunk's own (already consumed) input in the stage.
-template <bool YARD, bool CAREFUL, bool STORE, int NCH, bool COUNT = true, bool STASH = false>
+template <bool YARD, bool CAREFUL, bool STORE, int NCH, bool COUNT = true, bool STASH = false, bool LINEAR = false>
 __device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uint32_t out_addr, int j0, uint32_t s4b, uint32_t s5b, ConvAcc& c,
                                                uint32_t stash_addr = 0u)
 {
@@ -527,15 +537,15 @@ __device__ __forceinline__ void convert_chunks(const uint32_t (&w)[4 * NCH], uin
             uint32_t a[4], b[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) convert_pair_careful<YARD>(w[4 * j + i], s4, s5, c.A, a[i], b[i]);
-            if (STORE) sts64(out_addr ^ ((j0 + j) << 3), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
-            if (STASH) sts64(stash_addr ^ ((j0 + j) << 4), make_uint2(__byte_perm(b[0], b[1], 0x5410), __byte_perm(b[2], b[3], 0x5410)));
+            if (STORE) sts64(out_chunk<LINEAR>(out_addr, j0 + j), make_uint2(__byte_perm(a[0], a[1], 0x5410), __byte_perm(a[2], a[3], 0x5410)));
+            if (STASH) sts64(in_chunk<LINEAR>(stash_addr, j0 + j), make_uint2(__byte_perm(b[0], b[1], 0x5410), __byte_perm(b[2], b[3], 0x5410)));
         } else {
             uint32_t c4[2], c5[2];
 #pragma unroll
             for (int k = 0; k < 2; ++k)
                 convert_quad_fast<YARD, COUNT>(w[4 * j + 2 * k], w[4 * j + 2 * k + 1], s4x2, tiny2, c.q43[k], c.q52[k], c.cnt2, c4[k], c5[k]);
-            if (STORE) sts64(out_addr ^ ((j0 + j) << 3), make_uint2(c4[0], c4[1]));
-            if (STASH) sts64(stash_addr ^ ((j0 + j) << 4), make_uint2(c5[0], c5[1]));
+            if (STORE) sts64(out_chunk<LINEAR>(out_addr, j0 + j), make_uint2(c4[0], c4[1]));
+            if (STASH) sts64(in_chunk<LINEAR>(stash_addr, j0 + j), make_uint2(c5[0], c5[1]));
         }
     }
 }
@@ -579,10 +589,11 @@ __device__ __forceinline__ void convert_words(const uint32_t (&w)[32], uint32_t 
 }
 
 // A block selected E5M2: the thread's 64 stashed E5M2 codes replace its E4M3 codes in the staging buffer.
+template <bool LINEAR = false>
 __device__ __forceinline__ void copy_stash(uint32_t stash_addr, uint32_t out_addr)
 {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) sts64(out_addr ^ (j << 3), lds64(stash_addr ^ (j << 4)));
+    for (int j = 0; j < 8; ++j) sts64(out_chunk<LINEAR>(out_addr, j), lds64(in_chunk<LINEAR>(stash_addr, j)));
 }
 
 // The E5M2 codes of a thread's 64 elements, for a block that selected E5M2 (such a block holds no
@@ -1275,8 +1286,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     const int swz = kColumns ? ((row >> 1) & 3) ^ (h << 2) : (row & 7) ^ (h << 2);
     constexpr bool kLineBlocks = KIND == KIND_ROW128 || KIND == KIND_COL128;
     const int q = KIND == KIND_BLK64 ? ((row >> 6) << 1) | h : 0;     // which of the tile's blocks this thread's elements belong to
-    const uint32_t in_off = (uint32_t)(row * 256 + h * 128 + (swz << 4));
-    const uint32_t out_off = (uint32_t)(row * 128 + h * 64 + (swz << 3));
+    // 128x128 blocks and the per-tensor block without BF16 outputs: any 64 elements of the tile will do for a thread,
+    // so it takes chunk tid & 15 of rows (tid >> 4) + 16 j and every address is a base plus a constant
+    constexpr bool kLinear = (KIND == KIND_BLK128 || KIND == KIND_TENSOR) && !EXTRA;
+    const uint32_t in_off = kLinear ? (uint32_t)((tid >> 4) * 256 + (tid & 15) * 16) : (uint32_t)(row * 256 + h * 128 + (swz << 4));
+    const uint32_t out_off = kLinear ? (uint32_t)((tid >> 4) * 128 + (tid & 15) * 8) : (uint32_t)(row * 128 + h * 64 + (swz << 3));
     const uint32_t in_base = smem_addr(in), out_base = smem_addr(out), entry_base = smem_addr(&C.entry[0][0]);
 
     // what changes only with the tensor, kept in registers
@@ -1376,11 +1390,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
         if (!SCAN) {
             key &= 0x7FFFFFFFu;                         // (the flag for NaN/inf is part of the prepared word)
         } else if (kLineBlocks) {
-            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
+            key = kStream ? scan_stage<kLinear>(in_base + s * kInBytes + in_off) : scan_words(w);
             key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);            // warp-uniform
             if (nonfin) {
-                key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
+                key = kStream ? scan_stage_finite<kLinear>(in_base + s * kInBytes + in_off) : scan_words_finite(w);
                 key = key_max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here (non-negative binary32
@@ -1390,7 +1404,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 raise_amax(amax_slot, wamax, lane == 0 && !dead);
             }
         } else if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
-            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
+            key = kStream ? scan_stage<kLinear>(in_base + s * kInBytes + in_off) : scan_words(w);
             uint32_t tile_amax = 0u;
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
@@ -1419,14 +1433,14 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 if (dead) { key = 0u; nonfin = false; }
                 tile_amax = any >> 16;
                 if (pass == 1 || !nonfin) break;
-                key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
+                key = kStream ? scan_stage_finite<kLinear>(in_base + s * kInBytes + in_off) : scan_words_finite(w);
             }
             // no pre-pass ran: the tensor amax that the summary reports is gathered here
             if (amax_slot != nullptr) raise_amax(amax_slot, tile_amax, tid == 0 && !dead);
         } else {
-            key = kStream ? scan_stage(in_base + s * kInBytes + in_off) : scan_words(w);
+            key = kStream ? scan_stage<kLinear>(in_base + s * kInBytes + in_off) : scan_words(w);
             nonfin = __any_sync(0xFFFFFFFFu, (key >> 16) >= kBf16Inf);
-            if (nonfin) key = kStream ? scan_stage_finite(in_base + s * kInBytes + in_off) : scan_words_finite(w);
+            if (nonfin) key = kStream ? scan_stage_finite<kLinear>(in_base + s * kInBytes + in_off) : scan_words_finite(w);
         }
         uint32_t amax_bits = key >> 16;
         const uint32_t minm1 = 0xFFFFu - (key & 0xFFFFu);
@@ -1468,11 +1482,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                         uint32_t wh[16];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const uint4 v = lds128(a ^ ((4 * half + j) << 4));
+                            const uint4 v = lds128(in_chunk<kLinear>(a, 4 * half + j));
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
                         if (half == 1 && !kStash) stage_free_arrive(s);
-                        convert_chunks<YARD, true, STORE, 4, kCount, kStash>(wh, oa, 4 * half, s4b, s5b, acc, a);
+                        convert_chunks<YARD, true, STORE, 4, kCount, kStash, kLinear>(wh, oa, 4 * half, s4b, s5b, acc, a);
                     }
                     conv_finish<YARD, true, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 } else {
@@ -1481,11 +1495,11 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                         uint32_t wh[16];
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const uint4 v = lds128(a ^ ((4 * half + j) << 4));
+                            const uint4 v = lds128(in_chunk<kLinear>(a, 4 * half + j));
                             wh[4 * j] = v.x; wh[4 * j + 1] = v.y; wh[4 * j + 2] = v.z; wh[4 * j + 3] = v.w;
                         }
                         if (half == 1 && !kStash) stage_free_arrive(s);
-                        convert_chunks<YARD, false, STORE, 4, kCount, kStash>(wh, oa, 4 * half, s4b, s5b, acc, a);
+                        convert_chunks<YARD, false, STORE, 4, kCount, kStash, kLinear>(wh, oa, 4 * half, s4b, s5b, acc, a);
                     }
                     conv_finish<YARD, false, kCount>(acc, s4b, s5b, e43, e52, nnz, nonf);
                 }
@@ -1509,7 +1523,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 const bool valid = row < (KIND == KIND_COL128 ? m.vcols : m.vrows);
                 sel = decide_block(D, e43, e52, nz & 0xFFFFu, nz >> 16, amax_bits, minm1, (uint32_t)(KIND == KIND_COL128 ? m.vrows : m.vcols));
                 if (kStash) {
-                    if (sel == MOR_FMT_E5M2) copy_stash(in_base + s * kInBytes + in_off, oa);
+                    if (sel == MOR_FMT_E5M2) copy_stash<kLinear>(in_base + s * kInBytes + in_off, oa);
                     fence_async_smem();                  // the stage is written by the next TMA load: order the stash accesses before it
                     stage_free_arrive(s);
                 } else if (THREE && STORE && sel == MOR_FMT_E5M2) {
@@ -1588,7 +1602,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 if (!dead) sel = C.dec_sel[b][q];
                 if (THREE && STORE) {
                     if (kStash) {
-                        if (!dead && sel == MOR_FMT_E5M2) copy_stash(in_base + s * kInBytes + in_off, oa);
+                        if (!dead && sel == MOR_FMT_E5M2) copy_stash<kLinear>(in_base + s * kInBytes + in_off, oa);
                     } else if (!dead && sel == MOR_FMT_E5M2) {
                         emit_e5m2_codes(w, oa, s5b);
                     }
