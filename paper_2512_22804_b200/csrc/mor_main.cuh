@@ -88,6 +88,7 @@ struct Control {
     uint32_t tile_scale[2][4][2];                        // scale bits (E4M3, E5M2) of the tile's blocks
     uint32_t tile_key[2][4];                             // amax bits << 16 | 0xFFFF - (min - 1)
     uint32_t dec_sel[2][4];
+    alignas(16) float wsum[2][3][kComputeWarps];         // 128x128 blocks, three formats: per warp the E4M3 sum, the E5M2 sum, NaN/inf count (as bits)
     uint32_t rtab[128];                                  // bits of fl32(448 / (1 + m/128))
     // blocks along the columns with prepared scales (compute_cols_fast): what the store warp needs per tile besides
     // the entries -- per column the scale bits (bit 31: the column piece holds NaN or inf), per warp the count of
@@ -939,8 +940,10 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
         // the decision is handed back on every tile of a launch whose compute threads may need it (three formats:
         // E5M2 codes; EXTRA: a BF16 copy or a fake-quantised output for some tensor of the launch), whether this
         // tensor's threads wait for it or not: the barrier's phase then follows the tile count
-        constexpr bool need_dec = kTileBlocks && (THREE || EXTRA);
-        const bool codes_wait = STORE && kTileBlocks && THREE;
+        // (128x128 blocks, three formats, plain outputs: the compute threads have decided and the codes are final)
+        constexpr bool kSelfDecided = KIND == KIND_BLK128 && THREE && STORE && !EXTRA;
+        constexpr bool need_dec = kTileBlocks && (THREE || EXTRA) && !kSelfDecided;
+        const bool codes_wait = STORE && kTileBlocks && THREE && !kSelfDecided;
         out_full_sync(b);                                // sleeps until every compute thread has arrived
         if (!__any_sync(0xFFFFFFFFu, C.abort != 0u)) {
             if (STORE && !codes_wait && lane == 0) {
@@ -1109,7 +1112,7 @@ __device__ __forceinline__ void store_warp(const MainParams& p, Control& C, unsi
                     if (vr > 0 && vc > 0) {
                         const uint32_t key = C.tile_key[b][q], s4b = C.tile_scale[b][q][0], s5b = C.tile_scale[b][q][1];
                         const uint32_t amax_bits = key >> 16, minm1 = 0xFFFFu - (key & 0xFFFFu);
-                        bsel = decide_block(R, s43[r], s52[r], nnz[r], nonf[r], amax_bits, minm1, (uint32_t)(vr * vc));
+                        bsel = kSelfDecided ? C.dec_sel[b][0] : decide_block(R, s43[r], s52[r], nnz[r], nonf[r], amax_bits, minm1, (uint32_t)(vr * vc));
                         const uint32_t blk = NR == 2 ? (uint32_t)(t.row0 / 64 + r) * R.nbc_blk + (uint32_t)(t.col0 / 64 + lane) : t.local;
                         const uint32_t sb = (bsel == MOR_FMT_E5M2) ? s5b : s4b;
                         if (R.sel) R.sel[blk] = (uint8_t)bsel;
@@ -1308,6 +1311,10 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
     // scale that the row's first thread leaves it); with them everything about a block is written from here
     constexpr bool kRowFast = KIND == KIND_ROW128 && !EXTRA && !THREE;
     constexpr bool kMetaInStore = kLineBlocks && !EXTRA && !kRowFast;
+    // 128x128 blocks, three formats, plain outputs: the compute threads settle the block's format among themselves
+    // (warp sums, one barrier, the same fixed-order total in every thread) and put the chosen codes in place before
+    // they hand the tile to the store warp -- no round trip through that warp
+    constexpr bool kSelfDecide = KIND == KIND_BLK128 && THREE && STORE && !EXTRA;
     const uint32_t n_it = my_tile_count(p);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
@@ -1359,7 +1366,7 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
             }
         }
         const TensorRec& R = p.b.t[m.ti];
-        if (kLineBlocks && !kRowFast && m.ti != d_ti) { d_ti = m.ti; D.load(R); }
+        if (((kLineBlocks && !kRowFast) || kSelfDecide) && m.ti != d_ti) { d_ti = m.ti; D.load(R); }
         if ((SCAN || EXTRA) && m.ti != cur_ti) {
             cur_ti = m.ti;
             has_fallback = EXTRA && STORE && R.fallback != nullptr;
@@ -1584,14 +1591,37 @@ __device__ __forceinline__ void compute_warps(const MainParams& p, Control& C, u
                 if ((KIND == KIND_BLK128 && tid == 0) || (KIND == KIND_BLK64 && (row & 63) == 0)) {
                     C.tile_scale[b][q][0] = s4b; C.tile_scale[b][q][1] = s5b; C.tile_key[b][q] = key;
                 }
+                if (kSelfDecide) {
+                    float w43 = e43, w52 = e52;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) { w43 += __shfl_xor_sync(0xFFFFFFFFu, w43, o); w52 += __shfl_xor_sync(0xFFFFFFFFu, w52, o); }
+                    const uint32_t wnf = __reduce_add_sync(0xFFFFFFFFu, nonf);
+                    if (lane == 0) { C.wsum[b][0][warp] = w43; C.wsum[b][1][warp] = w52; C.wsum[b][2][warp] = __uint_as_float(wnf); }
+                }
             }
             if (STORE) fence_async_smem();              // the codes must be visible to the TMA store
         } else if (kStream && !(kStash && !kLineBlocks)) {
             stage_free_arrive(s);                       // given up: the arrival that the conversion would have made
         }
+        if (kSelfDecide) {
+            dead = compute_bar_or(dead);                // every compute thread, whatever its state; spreads the word of a wait that ran out
+            if (!dead) {
+                const float4 a0 = *reinterpret_cast<const float4*>(&C.wsum[b][0][0]), a1 = *reinterpret_cast<const float4*>(&C.wsum[b][0][4]);
+                const float4 b0 = *reinterpret_cast<const float4*>(&C.wsum[b][1][0]), b1 = *reinterpret_cast<const float4*>(&C.wsum[b][1][4]);
+                const uint4 n0 = *reinterpret_cast<const uint4*>(&C.wsum[b][2][0]), n1 = *reinterpret_cast<const uint4*>(&C.wsum[b][2][4]);
+                const float t43 = ((a0.x + a0.y) + (a0.z + a0.w)) + ((a1.x + a1.y) + (a1.z + a1.w));
+                const float t52 = ((b0.x + b0.y) + (b0.z + b0.w)) + ((b1.x + b1.y) + (b1.z + b1.w));
+                const uint32_t tnf = (n0.x + n0.y + n0.z + n0.w) + (n1.x + n1.y + n1.z + n1.w);
+                sel = decide_block(D, t43, t52, 0u, tnf, amax_bits, minm1, (uint32_t)(m.vrows * m.vcols));
+                if (sel == MOR_FMT_E5M2) copy_stash<kLinear>(in_base + s * kInBytes + in_off, oa);
+                fence_async_smem();                      // stash accesses before the next TMA load; codes visible to the TMA store
+                if (tid == 0) C.dec_sel[b][0] = sel;     // for the store warp's metadata
+            }
+            stage_free_arrive(s);
+        }
         out_full_arrive(b);
 
-        if (KIND == KIND_BLK128 || KIND == KIND_BLK64) {
+        if (!kSelfDecide && (KIND == KIND_BLK128 || KIND == KIND_BLK64)) {
             const bool need_dec = THREE || (EXTRA && (has_fallback || has_fq));
             if ((THREE || EXTRA) && need_dec) {
                 if (!dead) {
