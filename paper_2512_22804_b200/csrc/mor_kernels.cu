@@ -149,7 +149,11 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
     const uint32_t local = M.local;
     const bool has_keys = (M.mode & kModeKeys) != 0u;
     const bool col_piece = (M.mode & kModeColPiece) != 0u;
-    const bool per_piece = (M.mode & kModePerPiece) != 0u;
+    // Keys of row pieces alone (1x128 blocks, per-channel rows): the thread holds half a row piece (see the kernel), so
+    // a piece's key is the thread's own key joined with its neighbour's.  With column keys wanted as well the thread
+    // holds chunks of eight row pieces and the 16 lanes of a piece are joined by shuffles.
+    const bool row_map = (M.mode & kModePerPiece) != 0u && !col_piece;
+    const bool per_piece = (M.mode & kModePerPiece) != 0u && col_piece;
     uint32_t key[8], all = 0u, nf = 0u;
     // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once (on the
     // words already masked for the keys).  The main kernel takes the tile's count from here and need not count while
@@ -202,6 +206,12 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
             nf += r.y;
             nf_piece |= (r.y ? 1u : 0u) << j;
         }
+    }
+    if (row_map) {
+        const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, all, 1);
+        uint32_t f = nf ? 1u : 0u;
+        f |= __shfl_xor_sync(0xFFFFFFFFu, f, 1);
+        if ((t & 1) == 0) M.keys[(size_t)local * kRowKeyStride + (t >> 1)] = key_max(all, other) | (f << 31);
     }
     if (per_piece) {
         // one key per row piece: combine the 16 lanes that share the piece
@@ -455,6 +465,7 @@ mor_amax_kernel(const __grid_constant__ MainParams p)
     // ---- compute warps ----
     bool dead = false;
     const uint32_t off = (uint32_t)((t >> 4) * 256 + (t & 15) * 16);
+    const uint32_t off_row = (uint32_t)((t >> 1) * 256 + (t & 1) * 128 + ((((t >> 1) & 7) ^ ((t & 1) << 2)) << 4));
     const uint32_t in_base = smem_addr(in);
 #pragma unroll 1
     for (uint32_t it = 0; it < n_it; ++it) {
@@ -469,10 +480,18 @@ mor_amax_kernel(const __grid_constant__ MainParams p)
         }
         uint4 v[8], m0, m1;
         if (!dead) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = lds128(in_base + s * (uint32_t)kAmaxStageBytes + off + (uint32_t)(j * 16 * 256));
             m0 = lds128(smem_addr(&C.meta[s]));
             m1 = lds128(smem_addr(&C.meta[s]) + 16u);
+            const uint32_t a = in_base + s * (uint32_t)kAmaxStageBytes;
+            if ((m0.z & (kModePerPiece | kModeColPiece)) == kModePerPiece) {
+                // row keys alone: thread (row t >> 1, half t & 1) takes the eight chunks of its 128 bytes, in an order
+                // that keeps the lanes of a load phase on distinct banks
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = lds128((a + off_row) ^ (uint32_t)(j << 4));
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = lds128(a + off + (uint32_t)(j * 16 * 256));
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&C.empty[s]);         // this warp's copies are in registers
