@@ -321,29 +321,36 @@ mor_status_t run(std::vector<Item>& items, void* workspace, size_t workspace_byt
         BatchParams& bp = pre.b;
         bp.n = 0;
         uint32_t t_end = 0;
+        bool rows_only = false;       // the launch being filled holds tensors that want row keys and nothing else
         auto flush = [&]() -> bool {
             if (bp.n == 0) return true;
             pre.total_tiles = t_end;
-            bool ok = launch_amax(pre, stream) == cudaSuccess;
+            bool ok = launch_amax(pre, rows_only, stream) == cudaSuccess;
             bool channel = false;
             for (int k = 0; k < bp.n; ++k) channel = channel || bp.t[k].kind == KIND_CHANNEL || bp.t[k].kind == KIND_COLCH;
             if (ok && channel) ok = launch_row_keys(bp, stream) == cudaSuccess;
             bp.n = 0; t_end = 0;
             return ok;
         };
-        for (int i = 0; i < n; ++i) {
-            const Item& it = items[i];
-            // a supplied group amax only fixes the shared mantissa; the per-tensor partition still
-            // needs its block amax, which is the tensor amax, from the data (Algorithm 1)
-            if (!it.prepass) continue;
-            TensorRec& r = bp.t[bp.n];
-            fill_rec(it, ws, l, r);
-            pre.in_map[bp.n] = in_maps[i];
-            t_end += r.n_tiles;
-            bp.tile_end[bp.n++] = t_end;
-            if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
+        // two rounds: the tensors that want row keys alone go through the pre-pass instantiation made for them
+        for (int round = 0; round < 2; ++round) {
+            rows_only = round == 0;
+            for (int i = 0; i < n; ++i) {
+                const Item& it = items[i];
+                // a supplied group amax only fixes the shared mantissa; the per-tensor partition still
+                // needs its block amax, which is the tensor amax, from the data (Algorithm 1)
+                if (!it.prepass) continue;
+                const bool wants_rows_only = (it.s.kind == KIND_ROW128 || it.s.kind == KIND_CHANNEL) && it.col_key_begin < 0;
+                if (wants_rows_only != rows_only) continue;
+                TensorRec& r = bp.t[bp.n];
+                fill_rec(it, ws, l, r);
+                pre.in_map[bp.n] = in_maps[i];
+                t_end += r.n_tiles;
+                bp.tile_end[bp.n++] = t_end;
+                if (bp.n == kMaxBatch && !flush()) return MOR_ERR_CUDA;
+            }
+            if (!flush()) return MOR_ERR_CUDA;
         }
-        if (!flush()) return MOR_ERR_CUDA;
     }
 
     // 2. main kernels, one launch per (variant, chunk of tensors); 3. their finalise kernels
@@ -581,7 +588,7 @@ mor_status_t mor_group_amax(const mor_tensor_desc_t* host_descs, int n, float* a
         }
         if (bp.n == kMaxBatch || (i == n - 1 && bp.n)) {
             pre.total_tiles = t_end;
-            if (launch_amax(pre, stream) != cudaSuccess) return MOR_ERR_CUDA;
+            if (launch_amax(pre, false, stream) != cudaSuccess) return MOR_ERR_CUDA;
             bp.n = 0; t_end = 0;
         }
     }

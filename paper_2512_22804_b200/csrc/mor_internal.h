@@ -148,7 +148,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 }
 #endif
 
-cudaError_t launch_amax(const MainParams& p, cudaStream_t s);   // records, input tensor maps, tile count, status word, wait limit
+cudaError_t launch_amax(const MainParams& p, bool rows_only, cudaStream_t s);   // records, input tensor maps, tile count, status word, wait limit
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s);      // per-channel: keys of whole rows / whole columns
 cudaError_t launch_row_decide(const BatchParams& p, Partial* partials, int kind, cudaStream_t s);
 cudaError_t launch_main(const MainVariant& v, const MainParams& p, Partial* partials, cudaStream_t s);

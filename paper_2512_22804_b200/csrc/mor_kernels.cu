@@ -142,6 +142,7 @@ __device__ __forceinline__ void scratch_free_sync(uint32_t b) { asm volatile("ba
 // a warp and written from here; everything that spans warps (tile key, quadrant keys, column keys, counts, the
 // tensor amax) is left per warp in the scratch `S` for the tail warp.  `dead`: a bounded wait has run out in this
 // warp -- its data are zeros and it writes no keys, but keeps its part in the hand-off.
+template <bool ROWS_ONLY>
 __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 (&v)[8], AmaxShared& S)
 {
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -150,10 +151,11 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
     const bool has_keys = (M.mode & kModeKeys) != 0u;
     const bool col_piece = (M.mode & kModeColPiece) != 0u;
     // Keys of row pieces alone (1x128 blocks, per-channel rows): the thread holds half a row piece (see the kernel), so
-    // a piece's key is the thread's own key joined with its neighbour's.  With column keys wanted as well the thread
+    // a piece's key is the thread's own key joined with its neighbour's.  In the general instantiation the thread
     // holds chunks of eight row pieces and the 16 lanes of a piece are joined by shuffles.
-    const bool row_map = (M.mode & kModePerPiece) != 0u && !col_piece;
-    const bool per_piece = (M.mode & kModePerPiece) != 0u && col_piece;
+    // (ROWS_ONLY: the instantiation for launches all of whose tensors want row keys and nothing else)
+    const bool row_map = ROWS_ONLY;
+    const bool per_piece = !ROWS_ONLY && (M.mode & kModePerPiece) != 0u;
     uint32_t key[8], all = 0u, nf = 0u;
     // non-zero elements of the thread's 64: per 16-bit half min(|x| bits, 1), summed in both halves at once (on the
     // words already masked for the keys).  The main kernel takes the tile's count from here and need not count while
@@ -379,6 +381,7 @@ struct AmaxControl {
 constexpr int kAmaxSmemBytes = 1024 + kAmaxStages * kAmaxStageBytes + (int)sizeof(AmaxControl);
 static_assert(2 * (kAmaxSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM must fit in shared memory");
 
+template <bool ROWS_ONLY>
 __global__ void __launch_bounds__(kAmaxThreads, 2)
 mor_amax_kernel(const __grid_constant__ MainParams p)
 {
@@ -483,7 +486,7 @@ mor_amax_kernel(const __grid_constant__ MainParams p)
             m0 = lds128(smem_addr(&C.meta[s]));
             m1 = lds128(smem_addr(&C.meta[s]) + 16u);
             const uint32_t a = in_base + s * (uint32_t)kAmaxStageBytes;
-            if ((m0.z & (kModePerPiece | kModeColPiece)) == kModePerPiece) {
+            if (ROWS_ONLY) {
                 // row keys alone: thread (row t >> 1, half t & 1) takes the eight chunks of its 128 bytes, in an order
                 // that keeps the lanes of a load phase on distinct banks
 #pragma unroll
@@ -501,7 +504,7 @@ mor_amax_kernel(const __grid_constant__ MainParams p)
             M.ti = (int32_t)m0.x; M.local = m0.y; M.mode = m0.z; M.key_stride = m0.w;
             M.keys = reinterpret_cast<uint32_t*>(((unsigned long long)m1.y << 32) | m1.x);
             M.col_keys = reinterpret_cast<uint32_t*>(((unsigned long long)m1.w << 32) | m1.z);
-            amax_thread_part(M, v, C.S[b]);
+            amax_thread_part<ROWS_ONLY>(M, v, C.S[b]);
         }
         scratch_full_arrive(b);
     }
@@ -698,10 +701,11 @@ mor_finalise_kernel(const __grid_constant__ BatchParams p, const Partial* __rest
 
 }  // namespace
 
-cudaError_t launch_amax(const MainParams& p, cudaStream_t s)
+template <bool ROWS_ONLY>
+cudaError_t launch_amax_t(const MainParams& p, cudaStream_t s)
 {
-    if (p.total_tiles == 0) return cudaSuccess;
-    static std::atomic<int> sm_count[64];   // per device; 0 = not set up yet
+    auto kfn = mor_amax_kernel<ROWS_ONLY>;
+    static std::atomic<int> sm_count[64];   // per instantiation and device; 0 = not set up yet
     static std::mutex setup;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -710,7 +714,7 @@ cudaError_t launch_amax(const MainParams& p, cudaStream_t s)
     int sms = sm_count[dev].load(std::memory_order_acquire);
     if (sms == 0) {
         std::lock_guard<std::mutex> lock(setup);         // host threads may make their first call together
-        e = cudaFuncSetAttribute(mor_amax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAmaxSmemBytes);
+        e = cudaFuncSetAttribute(kfn, cudaFuncAttributeMaxDynamicSharedMemorySize, kAmaxSmemBytes);
         if (e != cudaSuccess) return e;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
@@ -719,8 +723,16 @@ cudaError_t launch_amax(const MainParams& p, cudaStream_t s)
     }
     const uint32_t resident = 2u * (uint32_t)sms;
     const uint32_t grid = p.total_tiles < resident ? p.total_tiles : resident;
-    mor_amax_kernel<<<grid, kAmaxThreads, kAmaxSmemBytes, s>>>(p);
+    kfn<<<grid, kAmaxThreads, kAmaxSmemBytes, s>>>(p);
     return cudaGetLastError();
+}
+
+// rows_only: every tensor of the launch wants one key per row piece and nothing else (1x128 blocks or per-channel
+// rows, not paired with column blocks); the general instantiation serves every mix.
+cudaError_t launch_amax(const MainParams& p, bool rows_only, cudaStream_t s)
+{
+    if (p.total_tiles == 0) return cudaSuccess;
+    return rows_only ? launch_amax_t<true>(p, s) : launch_amax_t<false>(p, s);
 }
 
 cudaError_t launch_row_keys(const BatchParams& p, cudaStream_t s)
