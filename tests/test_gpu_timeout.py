@@ -31,6 +31,8 @@ CASES = [
     ("128x128 two-way, keys from the pre-pass (streaming)", (128, 128), TWO, {}, False),
     ("128x128 three-way (stash in the stage, decision round trip)", (128, 128), THREE, {}, False),
     ("1x128 three-way", (1, 128), THREE, {}, False),
+    ("1x128 two-way (decisions and metadata in the store warp)", (1, 128), TWO, {}, False),
+    ("per channel along the columns, tensor-level decision (full-width column path)", (0, 1), TWO, {}, False),
     ("64x64 with statistics and a fake-quantised output (register path)", (64, 64), THREE, dict(block_stats=True, fake_quant=True), False),
     ("128x128, group amax supplied (the kernel scans, CTA-wide exchange)", (128, 128), TWO, {}, True),
     ("1x128, group amax supplied", (1, 128), TWO, {}, True),
@@ -48,7 +50,7 @@ def test_timeout_is_reported_and_the_workspace_recovers(name, block, formats, kw
 
     bits = wl.gradient_like(512, 512, seed=97)                        # 16 tiles, one per thread block
     x = parity.to_device(bits)
-    crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) else mb.MOR_CRIT_BLOCK_VS_E5M2     # (0, 1): per column
+    crit = mb.MOR_CRIT_TENSOR_MEAN_REL if block in ((0, 0), (1, 0)) or (block == (0, 1) and not kw) else mb.MOR_CRIT_BLOCK_VS_E5M2
     r = mb.Recipe(block, formats, crit)
     ga = mb.group_amax([x]) if supplied else None
     torch.cuda.synchronize()
