@@ -10,17 +10,20 @@
 //                  two-stage ring of 32 KiB buffers to registers, then one thread starts the TMA
 //                  tile load (cp.async.bulk.tensor.2d, zero fill past the tensor's edge) of the
 //                  tile that uses the stage next; an mbarrier per stage tells when it has landed;
-//   compute warps  8 warps, two threads per tile row (per tile column with 128x1 blocks).  A thread
-//                  copies its 64 elements from the stage to registers, takes the block's amax and
-//                  smallest non-zero from the key that the amax pre-pass left for the block and
-//                  that arrived with the tile (or scans its registers for them where the caller
-//                  supplied the group amax and no pre-pass ran), derives the scale, converts and
-//                  accumulates the error terms from the registers, and writes its codes to a
-//                  16 KiB staging buffer;
+//   compute warps  8 warps.  A thread takes its 64 elements of the tile from the stage (two threads per tile row; with
+//                  128x128 blocks one 16-byte chunk of eight rows; with column blocks four columns over 16 rows,
+//                  or a column piece gathered by 16-bit loads), takes the block's scale as the load warp prepared
+//                  it from the key that the amax pre-pass left (or scans its elements for amax and smallest
+//                  non-zero where the caller supplied the group amax and no pre-pass ran), converts and
+//                  accumulates the error terms, and writes its codes to a 16 KiB staging buffer.  Without BF16
+//                  outputs it streams: 16 registers of data at a time, straight from the stage;
 //   store warp     sleeps on a hardware barrier until the staging buffer is complete, issues the
 //                  TMA tile store of the codes (clipped at the tensor's edge by the hardware, to 16-byte pieces of a row),
-//                  adds up the threads' sums in a fixed order, and writes the tile's partial and,
-//                  for 128x128 and 64x64 blocks, the blocks' decisions and metadata.
+//                  adds up the threads' sums in a fixed order, and writes the tile's partial and the blocks'
+//                  decisions and metadata (with the optional outputs, or three formats in line blocks, the
+//                  compute threads decide).
+// The load warp and the store warp keep what they need of a tensor's record in registers: reading the kernel's
+// parameter space once per tile with a computed index is slow enough to make them the pipeline's bottleneck.
 // Every wait on an mbarrier is bounded; a wait that runs out sets a status word that the
 // finalise kernel copies into mor_tensor_stats_t.status.  From then on the CTA's threads skip
 // the work and the waits but keep every barrier arrival, so that nobody is left waiting.
