@@ -161,7 +161,29 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
     // words already masked for the keys).  The main kernel takes the tile's count from here and need not count while
     // it converts.
     uint32_t nz2 = 0u;
-    if (per_piece) {
+    // per column of the thread's chunk (two columns to a word): the maximum and the wrapped minimum over its eight rows
+    uint32_t cm[4] = {0u, 0u, 0u, 0u}, cn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    bool have_cols = false;
+    if (col_piece && !per_piece) {
+        // column keys alone: the thread's own key is folded from its columns' (no second pass over the elements)
+        have_cols = true;
+#pragma unroll
+        for (int j = 0; j < 8; j += 2) {
+            const uint32_t a[4] = {v[j].x & 0x7FFF7FFFu, v[j].y & 0x7FFF7FFFu, v[j].z & 0x7FFF7FFFu, v[j].w & 0x7FFF7FFFu};
+            const uint32_t c[4] = {v[j + 1].x & 0x7FFF7FFFu, v[j + 1].y & 0x7FFF7FFFu, v[j + 1].z & 0x7FFF7FFFu, v[j + 1].w & 0x7FFF7FFFu};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                nz2 += __vimin3_u16x2(a[i], 0x00010001u, 0x00010001u) + __vimin3_u16x2(c[i], 0x00010001u, 0x00010001u);
+                cm[i] = __vimax3_u16x2(cm[i], a[i], c[i]);
+                cn[i] = __viaddmin_u16x2(c[i], 0xFFFFFFFFu, __viaddmin_u16x2(a[i], 0xFFFFFFFFu, cn[i]));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) key[j] = 0u;
+        const uint32_t mxx = __vimax3_u16x2(__vimax3_u16x2(cm[0], cm[1], cm[2]), cm[3], cm[3]);
+        const uint32_t m2 = __vimin3_u16x2(__vimin3_u16x2(cn[0], cn[1], cn[2]), cn[3], cn[3]);
+        all = (max(mxx & 0xFFFFu, mxx >> 16) << 16) | (0xFFFFu - min(m2 & 0xFFFFu, m2 >> 16));
+    } else if (per_piece) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t a0 = v[j].x & 0x7FFF7FFFu, a1 = v[j].y & 0x7FFF7FFFu, a2 = v[j].z & 0x7FFF7FFFu, a3 = v[j].w & 0x7FFF7FFFu;
@@ -258,9 +280,11 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
     if (col_piece) {
         // One key per column of the tile.  This thread holds 8 rows of 8 columns: per column the maximum and the
         // wrapped minimum over its rows, packed two columns to a word; lanes l and l ^ 16 hold the same columns of
-        // other rows; the warps' results meet in shared memory and 128 threads finish one column each.
-        uint32_t cm[4] = {0u, 0u, 0u, 0u}, cn[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu}, cf = 0u;
-        if (!warp_nf) {
+        // other rows; the warps' results meet in the scratch and the tail warp finishes four columns per lane.
+        uint32_t cf = 0u;
+        if (!warp_nf && have_cols) {
+            // (done above)
+        } else if (!warp_nf) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const uint32_t a[4] = {v[j].x & 0x7FFF7FFFu, v[j].y & 0x7FFF7FFFu, v[j].z & 0x7FFF7FFFu, v[j].w & 0x7FFF7FFFu};
@@ -269,6 +293,8 @@ __device__ __forceinline__ void amax_thread_part(const AmaxMeta& M, const uint4 
             }
         } else {
             // NaN or inf somewhere in the warp's data: element by element, finite ones only (rare path)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { cm[i] = 0u; cn[i] = 0xFFFFFFFFu; }
             for (int j = 0; j < 8; ++j) {
                 const uint32_t w4[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
                 for (int i = 0; i < 4; ++i)
